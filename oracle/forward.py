@@ -1,0 +1,113 @@
+"""Verify-forward oracle: q_i = M(x_<=t, x~_<i), i = 1..K+1 (Eq. 3 / Eq. 6).
+
+Test infrastructure only (see the package docstring).
+
+The paper treats the target model M as a black box; the model here is the
+Llama-style decoder the workloads name: RMSNorm, rotary position embedding
+(rotate-half pairing of feature i with i + head_dim/2), causal attention scaled by
+1/sqrt(head_dim), SwiGLU feed-forward, no biases, separate embedding and LM head.
+The pseudo-sequence is a chain, so the mask M_t is causal and the position ids
+P_t are consecutive: row i of a sequence with ctx cached tokens sits at position
+ctx + i and attends to the cache [0, ctx) and to rows 0..i of the same step.
+
+Arithmetic: everything in fp64 except what the data contract fixes - weights are
+bf16 values, and K and V are rounded to bf16 (round-to-nearest-even) when they
+enter the cache.  Logits come back as fp64; callers round to fp32 where the
+interface says fp32.
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Sequence
+
+import numpy as np
+import torch
+
+F64 = torch.float64
+
+
+class KVCache:
+    """Contiguous per-sequence cache: k, v bf16 [L, n_seqs, capacity, n_kv_heads, head_dim]."""
+
+    def __init__(self, cfg: Dict, n_seqs: int, capacity: int):
+        L, Hkv, dh = cfg["n_layers"], cfg["n_kv_heads"], cfg["head_dim"]
+        self.k = torch.zeros(L, n_seqs, capacity, Hkv, dh, dtype=torch.bfloat16)
+        self.v = torch.zeros(L, n_seqs, capacity, Hkv, dh, dtype=torch.bfloat16)
+        self.ctx = np.zeros(n_seqs, dtype=np.int64)
+        self.capacity = capacity
+
+    def clone(self) -> "KVCache":
+        c = object.__new__(KVCache)
+        c.k, c.v, c.ctx, c.capacity = self.k.clone(), self.v.clone(), self.ctx.copy(), self.capacity
+        return c
+
+
+def rmsnorm(x: torch.Tensor, gain: torch.Tensor, eps: float) -> torch.Tensor:
+    return x * torch.rsqrt((x * x).mean(dim=-1, keepdim=True) + eps) * gain
+
+
+def rope(x: torch.Tensor, pos: torch.Tensor, theta: float) -> torch.Tensor:
+    """x [R, H, dh]; rotate the pair (i, i + dh/2) by pos * theta^(-2i/dh)."""
+    dh = x.shape[-1]
+    half = dh // 2
+    inv_freq = theta ** (-(torch.arange(half, dtype=F64) * 2.0 / dh))
+    ang = pos.to(F64)[:, None] * inv_freq[None, :]
+    c, s = torch.cos(ang)[:, None, :], torch.sin(ang)[:, None, :]
+    x1, x2 = x[..., :half], x[..., half:]
+    return torch.cat([x1 * c - x2 * s, x2 * c + x1 * s], dim=-1)
+
+
+def _r(x: torch.Tensor, mirror: bool) -> torch.Tensor:
+    """Debug aid: round an activation to bf16 where a bf16 tensor-core path would."""
+    return x.to(torch.bfloat16).to(F64) if mirror else x
+
+
+def forward(W: Dict, cfg: Dict, kv: KVCache, seq_ids: Sequence[int],
+            tokens: Sequence[np.ndarray], mirror_bf16: bool = False) -> List[torch.Tensor]:
+    """One forward over the new rows of each listed sequence.
+
+    tokens[j] holds the rows of sequence seq_ids[j]: the pending token followed by its
+    drafts (or a prompt chunk).  K and V of every row are written to the cache at
+    positions ctx .. ctx + rows - 1; kv.ctx itself is not changed (committing is the
+    acceptance step's job).  Returns one fp64 logits tensor [rows, vocab] per sequence.
+    """
+    H, Hkv, dh = cfg["n_heads"], cfg["n_kv_heads"], cfg["head_dim"]
+    eps, theta = cfg["rms_eps"], cfg["rope_theta"]
+    rows = [len(t) for t in tokens]
+    starts = np.concatenate([[0], np.cumsum(rows)]).astype(int)
+    flat = torch.as_tensor(np.concatenate([np.asarray(t, dtype=np.int64) for t in tokens]))
+    pos = torch.cat([torch.arange(r, dtype=torch.int64) + int(kv.ctx[s])
+                     for s, r in zip(seq_ids, rows)])
+    for s, r in zip(seq_ids, rows):
+        if kv.ctx[s] + r > kv.capacity:
+            raise ValueError("KV capacity exceeded")
+    x = W["tok_emb"][flat].to(F64)
+    rep = H // Hkv
+    for l, lw in enumerate(W["layers"]):
+        h = _r(rmsnorm(x, lw["attn_norm"].to(F64), eps), mirror_bf16)
+        q = (h @ lw["wq"].to(F64).T).view(-1, H, dh)
+        k = (h @ lw["wk"].to(F64).T).view(-1, Hkv, dh)
+        v = (h @ lw["wv"].to(F64).T).view(-1, Hkv, dh)
+        q = _r(rope(q, pos, theta), mirror_bf16)
+        k = rope(k, pos, theta).to(torch.bfloat16)          # cache contract: bf16 K, V
+        v = v.to(torch.bfloat16)
+        att = torch.empty(x.shape[0], H, dh, dtype=F64)
+        for j, s in enumerate(seq_ids):
+            a, b, c = starts[j], starts[j + 1], int(kv.ctx[s])
+            kv.k[l, s, c:c + rows[j]] = k[a:b]
+            kv.v[l, s, c:c + rows[j]] = v[a:b]
+            for i in range(rows[j]):                          # row i sees cache + rows 0..i
+                n = c + i + 1
+                kk = kv.k[l, s, :n].to(F64).repeat_interleave(rep, dim=1)   # [n, H, dh]
+                vv = kv.v[l, s, :n].to(F64).repeat_interleave(rep, dim=1)
+                sc = torch.einsum("hd,nhd->hn", q[a + i], kk) / (dh ** 0.5)
+                pr = torch.softmax(sc, dim=-1)
+                att[a + i] = torch.einsum("hn,nhd->hd", pr, vv)
+        x = x + _r(att.reshape(-1, H * dh), mirror_bf16) @ lw["wo"].to(F64).T
+        h2 = _r(rmsnorm(x, lw["ffn_norm"].to(F64), eps), mirror_bf16)
+        gate = h2 @ lw["w_gate"].to(F64).T
+        up = h2 @ lw["w_up"].to(F64).T
+        act = _r(gate * torch.sigmoid(gate) * up, mirror_bf16)  # SwiGLU: silu(gate) * up
+        x = x + act @ lw["w_down"].to(F64).T
+    hn = _r(rmsnorm(x, W["final_norm"].to(F64), eps), mirror_bf16)
+    logits = hn @ W["lm_head"].to(F64).T
+    return [logits[starts[j]:starts[j + 1]] for j in range(len(rows))]
