@@ -1,0 +1,508 @@
+// Target model M and its paged KV cache; the verify forward q_i = M(x_<=t, x~_<i) of
+// Eq. 3 / Eq. 6 for a Llama-style decoder (RMSNorm, rotary embedding with rotate-half
+// pairing, causal attention, SwiGLU, no biases).
+//
+// One step processes R = B * (K+1) rows.  The residual stream, the norm statistics and the
+// softmax stay in fp32; GEMM operands, Q and the K/V cache are bf16.  K and V of all rows
+// are written to the pages before attention, so attention reads cache and new rows alike.
+#include <cmath>
+
+#include "model.cuh"
+
+namespace laser {
+namespace {
+
+using bf16 = __nv_bfloat16;
+
+// ---- row bookkeeping -------------------------------------------------------------------
+// One thread per row: position, cache slot, capacity check, rotary angles (fp64 -> fp32).
+__global__ void prep_rows_kernel(const int32_t* __restrict__ seq_ids, const int32_t* __restrict__ n_rows,
+                                 int B, int Rs, int R_pad, const int32_t* __restrict__ seq_len,
+                                 int max_seqs, int capacity, int half, double theta, int head_dim,
+                                 int32_t* __restrict__ row_pos, int32_t* __restrict__ row_seq,
+                                 int32_t* __restrict__ row_ctx, int32_t* __restrict__ row_n,
+                                 float* __restrict__ rope, int32_t* __restrict__ status) {
+  const int r = blockIdx.x;
+  const int b = r / Rs, i = r % Rs;
+  int pos = -1, seq = 0;
+  if (r < B * Rs) {
+    seq = seq_ids[b];
+    int nr = min(max(n_rows[b], 0), Rs);
+    int ctx = 0;
+    if (seq < 0 || seq >= max_seqs) {
+      nr = 0; seq = 0;
+      if (threadIdx.x == 0) atomicCAS(status, 0, LASER_ERR_INVALID_ARG);
+    } else {
+      ctx = seq_len[seq];
+      if (ctx + nr > capacity) {
+        nr = 0;
+        if (threadIdx.x == 0) atomicCAS(status, 0, LASER_ERR_CAPACITY);
+      }
+    }
+    if (i < nr) pos = ctx + i;
+    if (i == 0 && threadIdx.x == 0) { row_ctx[b] = ctx; row_n[b] = nr; }
+  }
+  if (threadIdx.x == 0) { row_pos[r] = pos; row_seq[r] = seq; }
+  for (int j = threadIdx.x; j < half; j += blockDim.x) {
+    const double inv_freq = pow(theta, -2.0 * double(j) / double(head_dim));
+    double s, c;
+    sincos(double(max(pos, 0)) * inv_freq, &s, &c);
+    rope[(size_t(r) * half + j) * 2] = float(c);
+    rope[(size_t(r) * half + j) * 2 + 1] = float(s);
+  }
+}
+
+__device__ __forceinline__ float block_sum(float v, float* red) {
+  for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  __syncthreads();
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float t = 0.f;
+  for (int w = 0; w < nw; ++w) t += red[w];
+  return t;
+}
+
+// Embedding gather, then RMSNorm with the first layer's gain.
+__global__ void __launch_bounds__(256)
+embed_norm_kernel(const int32_t* __restrict__ tokens, int R, int d, int vocab, const bf16* __restrict__ emb,
+                  const bf16* __restrict__ gain, float eps, float* __restrict__ resid, bf16* __restrict__ xn) {
+  __shared__ float red[8];
+  const int r = blockIdx.x;
+  const int tok = r < R ? tokens[r] : -1;
+  const bool ok = tok >= 0 && tok < vocab;
+  float ss = 0.f;
+  for (int j = threadIdx.x; j < d; j += blockDim.x) {
+    const float x = ok ? __bfloat162float(emb[size_t(tok) * d + j]) : 0.f;
+    resid[size_t(r) * d + j] = x;
+    ss += x * x;
+  }
+  ss = block_sum(ss, red);
+  const float scale = rsqrtf(ss / float(d) + eps);
+  for (int j = threadIdx.x; j < d; j += blockDim.x)
+    xn[size_t(r) * d + j] = __float2bfloat16(resid[size_t(r) * d + j] * scale * __bfloat162float(gain[j]));
+}
+
+// resid += sum of split-K planes; xn = RMSNorm(resid) * gain.
+__global__ void __launch_bounds__(256)
+residual_norm_kernel(const float* __restrict__ part, int splits, size_t split_stride, int ld, int d,
+                     const bf16* __restrict__ gain, float eps, float* __restrict__ resid, bf16* __restrict__ xn) {
+  __shared__ float red[8];
+  const int r = blockIdx.x;
+  float ss = 0.f;
+  for (int j = threadIdx.x; j < d; j += blockDim.x) {
+    float x = resid[size_t(r) * d + j];
+    for (int s = 0; s < splits; ++s) x += part[s * split_stride + size_t(r) * ld + j];
+    resid[size_t(r) * d + j] = x;
+    ss += x * x;
+  }
+  ss = block_sum(ss, red);
+  const float scale = rsqrtf(ss / float(d) + eps);
+  for (int j = threadIdx.x; j < d; j += blockDim.x)
+    xn[size_t(r) * d + j] = __float2bfloat16(resid[size_t(r) * d + j] * scale * __bfloat162float(gain[j]));
+}
+
+// act = silu(gate) * up from the split-K planes of the fused gate/up GEMM.
+__global__ void swiglu_kernel(const float* __restrict__ part, int splits, size_t split_stride, int f,
+                              bf16* __restrict__ act) {
+  const int r = blockIdx.y;
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= f) return;
+  float g = 0.f, u = 0.f;
+  for (int s = 0; s < splits; ++s) {
+    g += part[s * split_stride + size_t(r) * 2 * f + j];
+    u += part[s * split_stride + size_t(r) * 2 * f + f + j];
+  }
+  act[size_t(r) * f + j] = __float2bfloat16(g / (1.f + __expf(-g)) * u);
+}
+
+// Rotary embedding of Q and K, bf16 rounding, K/V page write.  grid (row, head slot) where
+// head slots are [0, H) for Q, [H, H+Hkv) for K, [H+Hkv, H+2Hkv) for V.
+__global__ void rope_kv_kernel(const float* __restrict__ part, int splits, size_t split_stride, int dqkv,
+                               int H, int Hkv, int dh, const float* __restrict__ rope,
+                               const int32_t* __restrict__ row_pos, const int32_t* __restrict__ row_seq,
+                               const int32_t* __restrict__ page_table, int pages_per_seq,
+                               bf16* __restrict__ pages_layer, size_t page_elems, bf16* __restrict__ q) {
+  const int r = blockIdx.x, slot = blockIdx.y, half = dh / 2;
+  const int pos = row_pos[r];
+  const float* src = part + size_t(r) * dqkv + size_t(slot) * dh;
+  for (int j = threadIdx.x; j < half; j += blockDim.x) {
+    float x1 = 0.f, x2 = 0.f;
+    for (int s = 0; s < splits; ++s) { x1 += src[s * split_stride + j]; x2 += src[s * split_stride + j + half]; }
+    float y1 = x1, y2 = x2;
+    if (slot < H + Hkv) {
+      const float c = rope[(size_t(r) * half + j) * 2], sn = rope[(size_t(r) * half + j) * 2 + 1];
+      y1 = x1 * c - x2 * sn;
+      y2 = x2 * c + x1 * sn;
+    }
+    if (slot < H) {
+      bf16* dst = q + size_t(r) * H * dh + size_t(slot) * dh;
+      dst[j] = __float2bfloat16(pos >= 0 ? y1 : 0.f);
+      dst[j + half] = __float2bfloat16(pos >= 0 ? y2 : 0.f);
+    } else if (pos >= 0) {
+      const int is_v = slot >= H + Hkv;
+      const int h = slot - H - (is_v ? Hkv : 0);
+      const int page = page_table[size_t(row_seq[r]) * pages_per_seq + pos / 16];
+      bf16* dst = pages_layer + size_t(page) * page_elems + (size_t(is_v) * Hkv + h) * 16 * dh + size_t(pos % 16) * dh;
+      dst[j] = __float2bfloat16(y1);
+      dst[j + half] = __float2bfloat16(y2);
+    }
+  }
+}
+
+// Causal attention of the step's rows over the paged cache: grid (sequence, head).
+// Scores of one row go to shared memory, softmax in fp32, then thread d accumulates
+// sum_j p_j V[j][d].
+__global__ void __launch_bounds__(128)
+attention_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ seq_ids,
+                 const int32_t* __restrict__ row_ctx, const int32_t* __restrict__ row_n, int Rs, int H,
+                 int Hkv, int dh, const int32_t* __restrict__ page_table, int pages_per_seq,
+                 const bf16* __restrict__ pages_layer, size_t page_elems, bf16* __restrict__ out) {
+  extern __shared__ float smem[];
+  float* s_q = smem;            // [dh]
+  float* s_sc = smem + dh;      // [ctx + rows]
+  __shared__ float red[4];
+  const int b = blockIdx.x, h = blockIdx.y, hk = h / (H / Hkv);
+  const int nr = row_n[b], ctx = row_ctx[b];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int32_t* pt = page_table + size_t(seq_ids[b]) * pages_per_seq;
+  const float scale = rsqrtf(float(dh));
+  for (int i = 0; i < Rs; ++i) {
+    const size_t r = size_t(b) * Rs + i;
+    bf16* o = out + r * H * dh + size_t(h) * dh;
+    if (i >= nr) {
+      for (int d = tid; d < dh; d += 128) o[d] = __float2bfloat16(0.f);
+      continue;
+    }
+    __syncthreads();
+    for (int d = tid; d < dh; d += 128) s_q[d] = __bfloat162float(q[r * H * dh + size_t(h) * dh + d]) * scale;
+    __syncthreads();
+    const int n = ctx + i + 1;
+    float mx = -INFINITY;
+    for (int j = tid; j < n; j += 128) {
+      const bf16* kp = pages_layer + size_t(pt[j / 16]) * page_elems + size_t(hk) * 16 * dh + size_t(j % 16) * dh;
+      float s = 0.f;
+      for (int d = 0; d < dh; d += 8) {
+        const uint4 u = *reinterpret_cast<const uint4*>(kp + d);
+        const bf16* e = reinterpret_cast<const bf16*>(&u);
+#pragma unroll
+        for (int x = 0; x < 8; ++x) s += s_q[d + x] * __bfloat162float(e[x]);
+      }
+      s_sc[j] = s;
+      mx = fmaxf(mx, s);
+    }
+    for (int o2 = 16; o2; o2 >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o2));
+    if (lane == 0) red[warp] = mx;
+    __syncthreads();
+    mx = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+    __syncthreads();
+    float sum = 0.f;
+    for (int j = tid; j < n; j += 128) {
+      const float e = __expf(s_sc[j] - mx);
+      s_sc[j] = e;
+      sum += e;
+    }
+    for (int o2 = 16; o2; o2 >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o2);
+    if (lane == 0) red[warp] = sum;
+    __syncthreads();
+    sum = red[0] + red[1] + red[2] + red[3];
+    for (int d = tid; d < dh; d += 128) {
+      float acc = 0.f;
+      for (int j = 0; j < n; ++j) {
+        const bf16* vp = pages_layer + size_t(pt[j / 16]) * page_elems + (size_t(Hkv) + hk) * 16 * dh + size_t(j % 16) * dh;
+        acc += s_sc[j] * __bfloat162float(vp[d]);
+      }
+      o[d] = __float2bfloat16(acc / sum);
+    }
+  }
+}
+
+// K/V copy between contiguous [n, Hkv*dh] arrays and the pages of one sequence and layer.
+__global__ void kv_copy_kernel(bf16* __restrict__ pages_layer, size_t page_elems, const int32_t* __restrict__ pt,
+                               int Hkv, int dh, int pos0, int n, bf16* __restrict__ k, bf16* __restrict__ v,
+                               int to_pages) {
+  const int w = Hkv * dh;
+  for (size_t idx = size_t(blockIdx.x) * blockDim.x + threadIdx.x; idx < size_t(n) * w;
+       idx += size_t(gridDim.x) * blockDim.x) {
+    const int t = int(idx / w), c = int(idx % w), h = c / dh, d = c % dh;
+    const int pos = pos0 + t;
+    bf16* kp = pages_layer + size_t(pt[pos / 16]) * page_elems + size_t(h) * 16 * dh + size_t(pos % 16) * dh + d;
+    bf16* vp = kp + size_t(Hkv) * 16 * dh;
+    if (to_pages) { *kp = k[idx]; *vp = v[idx]; } else { k[idx] = *kp; v[idx] = *vp; }
+  }
+}
+
+__global__ void set_len_kernel(int32_t* __restrict__ seq_len, const int32_t* __restrict__ src, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) seq_len[i] = src[i];
+}
+
+template <typename T>
+laser_status model_alloc(laser_model* m, T** p, size_t count) {
+  LASER_CUDA(cudaMalloc(reinterpret_cast<void**>(p), std::max<size_t>(count, 1) * sizeof(T)));
+  LASER_CUDA(cudaMemset(*p, 0, std::max<size_t>(count, 1) * sizeof(T)));
+  m->owned.push_back(*p);
+  return LASER_OK;
+}
+
+// Returns `first` if the pieces are adjacent in memory, else a fused device copy.
+laser_status fuse_rows(laser_model* m, const void* const* pieces, const size_t* elems, int n,
+                       const bf16** out) {
+  bool adjacent = true;
+  for (int i = 1; i < n; ++i)
+    adjacent = adjacent && (static_cast<const bf16*>(pieces[i]) == static_cast<const bf16*>(pieces[i - 1]) + elems[i - 1]);
+  if (adjacent) { *out = static_cast<const bf16*>(pieces[0]); return LASER_OK; }
+  size_t total = 0;
+  for (int i = 0; i < n; ++i) total += elems[i];
+  bf16* buf = nullptr;
+  LASER_TRY(model_alloc(m, &buf, total));
+  size_t off = 0;
+  for (int i = 0; i < n; ++i) {
+    LASER_CUDA(cudaMemcpy(buf + off, pieces[i], elems[i] * sizeof(bf16), cudaMemcpyDeviceToDevice));
+    off += elems[i];
+  }
+  *out = buf;
+  return LASER_OK;
+}
+
+}  // namespace
+}  // namespace laser
+
+using namespace laser;
+
+LASER_API laser_status laser_model_free(laser_model* m) {
+  if (!m) return LASER_OK;
+  gemm_state_free(m);
+  for (void* p : m->owned) cudaFree(p);
+  delete m;
+  return LASER_OK;
+}
+
+LASER_API laser_status laser_model_create(const laser_model_cfg* cfg, const laser_weights* w, laser_model** out) {
+  LASER_REQUIRE(cfg && w && out, "null argument");
+  LASER_REQUIRE(cfg->n_layers >= 0 && cfg->d_model >= 16 && cfg->n_heads >= 1 && cfg->n_kv_heads >= 1 &&
+                cfg->d_ffn >= 16 && cfg->vocab >= 8, "bad model shape");
+  LASER_REQUIRE(cfg->n_heads % cfg->n_kv_heads == 0, "n_heads must be a multiple of n_kv_heads");
+  LASER_REQUIRE(cfg->head_dim % 16 == 0 && cfg->head_dim >= 16 && cfg->head_dim <= 256, "head_dim = %d", cfg->head_dim);
+  LASER_REQUIRE(cfg->page_size == 16, "page_size must be 16");
+  LASER_REQUIRE(cfg->max_draft >= 0 && cfg->max_draft <= 63 && cfg->max_batch >= 1, "max_draft / max_batch");
+  LASER_REQUIRE(w->tok_emb && w->lm_head && w->final_norm, "null weight");
+  laser_model* m = new laser_model();
+  struct Guard { laser_model* p; ~Guard() { if (p) laser_model_free(p); } } guard{m};
+  m->cfg = *cfg;
+  m->rows_per_seq = cfg->max_draft + 1;
+  m->R = cfg->max_batch * m->rows_per_seq;
+  m->R_pad = ceil_div(m->R, 16) * 16;
+  const int d = cfg->d_model, f = cfg->d_ffn, L = cfg->n_layers;
+  m->dq = cfg->n_heads * cfg->head_dim;
+  m->dkv = cfg->n_kv_heads * cfg->head_dim;
+  m->dqkv = m->dq + 2 * m->dkv;
+  m->tok_emb = static_cast<const bf16*>(w->tok_emb);
+  m->lm_head = static_cast<const bf16*>(w->lm_head);
+  m->final_norm = static_cast<const bf16*>(w->final_norm);
+  for (int l = 0; l < L; ++l) {
+    LASER_REQUIRE(w->wq[l] && w->wk[l] && w->wv[l] && w->wo[l] && w->w_gate[l] && w->w_up[l] && w->w_down[l] &&
+                  w->attn_norm[l] && w->ffn_norm[l], "null weight in layer %d", l);
+    const void* qkv[3] = {w->wq[l], w->wk[l], w->wv[l]};
+    const size_t qkv_e[3] = {size_t(m->dq) * d, size_t(m->dkv) * d, size_t(m->dkv) * d};
+    const bf16* fused = nullptr;
+    LASER_TRY(fuse_rows(m, qkv, qkv_e, 3, &fused));
+    m->wqkv.push_back(fused);
+    const void* gu[2] = {w->w_gate[l], w->w_up[l]};
+    const size_t gu_e[2] = {size_t(f) * d, size_t(f) * d};
+    LASER_TRY(fuse_rows(m, gu, gu_e, 2, &fused));
+    m->wgu.push_back(fused);
+    m->wo.push_back(static_cast<const bf16*>(w->wo[l]));
+    m->wdown.push_back(static_cast<const bf16*>(w->w_down[l]));
+    m->attn_norm.push_back(static_cast<const bf16*>(w->attn_norm[l]));
+    m->ffn_norm.push_back(static_cast<const bf16*>(w->ffn_norm[l]));
+  }
+  const size_t Rp = size_t(m->R_pad);
+  LASER_TRY(model_alloc(m, &m->resid, Rp * d));
+  LASER_TRY(model_alloc(m, &m->xn, Rp * d));
+  LASER_TRY(model_alloc(m, &m->q, Rp * m->dq));
+  LASER_TRY(model_alloc(m, &m->attn, Rp * m->dq));
+  LASER_TRY(model_alloc(m, &m->act, Rp * f));
+  size_t part = 0;
+  const int shapes[4][2] = {{m->dqkv, d}, {d, m->dq}, {2 * f, d}, {d, f}};
+  for (auto& s : shapes) part = std::max(part, size_t(gemm_plan(m->R_pad, s[0], s[1]).splits) * Rp * s[0]);
+  m->part_floats = part;
+  LASER_TRY(model_alloc(m, &m->part, part));
+  LASER_TRY(model_alloc(m, &m->rope, Rp * (cfg->head_dim / 2) * 2));
+  LASER_TRY(model_alloc(m, &m->row_pos, Rp));
+  LASER_TRY(model_alloc(m, &m->row_seq, Rp));
+  LASER_TRY(model_alloc(m, &m->row_ctx, size_t(cfg->max_batch)));
+  LASER_TRY(model_alloc(m, &m->row_n, size_t(cfg->max_batch)));
+  LASER_TRY(model_alloc(m, &m->status, size_t(1)));
+  guard.p = nullptr;
+  *out = m;
+  return LASER_OK;
+}
+
+LASER_API laser_status laser_kv_free(laser_kv* kv) {
+  if (!kv) return LASER_OK;
+  cudaFree(kv->pages); cudaFree(kv->page_table); cudaFree(kv->seq_len);
+  delete kv;
+  return LASER_OK;
+}
+
+LASER_API laser_status laser_kv_create(const laser_model* m, int32_t max_seqs, int64_t n_pages, laser_kv** out) {
+  LASER_REQUIRE(m && out, "null argument");
+  LASER_REQUIRE(max_seqs >= 1 && n_pages >= max_seqs, "max_seqs = %d, n_pages = %lld", max_seqs, (long long)n_pages);
+  laser_kv* kv = new laser_kv();
+  struct Guard { laser_kv* p; ~Guard() { if (p) laser_kv_free(p); } } guard{kv};
+  kv->n_layers = m->cfg.n_layers; kv->n_kv_heads = m->cfg.n_kv_heads; kv->head_dim = m->cfg.head_dim;
+  kv->max_seqs = max_seqs; kv->n_pages = n_pages;
+  kv->pages_per_seq = int32_t(std::min<int64_t>(n_pages / max_seqs, 1 << 20));
+  const size_t elems = std::max<size_t>(1, size_t(kv->n_layers) * kv->layer_elems());
+  LASER_CUDA(cudaMalloc(reinterpret_cast<void**>(&kv->pages), elems * sizeof(__nv_bfloat16)));
+  LASER_CUDA(cudaMalloc(reinterpret_cast<void**>(&kv->page_table), size_t(max_seqs) * kv->pages_per_seq * 4));
+  LASER_CUDA(cudaMalloc(reinterpret_cast<void**>(&kv->seq_len), size_t(max_seqs) * 4));
+  LASER_CUDA(cudaMemset(kv->seq_len, 0, size_t(max_seqs) * 4));
+  std::vector<int32_t> table(size_t(max_seqs) * kv->pages_per_seq);
+  for (int s = 0; s < max_seqs; ++s)
+    for (int j = 0; j < kv->pages_per_seq; ++j) table[size_t(s) * kv->pages_per_seq + j] = j * max_seqs + s;
+  LASER_CUDA(cudaMemcpy(kv->page_table, table.data(), table.size() * 4, cudaMemcpyHostToDevice));
+  guard.p = nullptr;
+  *out = kv;
+  return LASER_OK;
+}
+
+LASER_API laser_status laser_kv_set_page_table(laser_kv* kv, const int32_t* table) {
+  LASER_REQUIRE(kv && table, "null argument");
+  const size_t n = size_t(kv->max_seqs) * kv->pages_per_seq;
+  std::vector<uint8_t> seen(size_t(kv->n_pages), 0);
+  for (size_t i = 0; i < n; ++i) {
+    LASER_REQUIRE(table[i] >= 0 && table[i] < kv->n_pages && !seen[table[i]], "page table entry %zu invalid or repeated", i);
+    seen[table[i]] = 1;
+  }
+  LASER_CUDA(cudaDeviceSynchronize());
+  LASER_CUDA(cudaMemcpy(kv->page_table, table, n * 4, cudaMemcpyHostToDevice));
+  return LASER_OK;
+}
+
+LASER_API laser_status laser_kv_set_len(laser_kv* kv, const int32_t* seq_ids, const int32_t* lens, int32_t n, void* stream) {
+  LASER_REQUIRE(kv && seq_ids && lens && n >= 0, "bad argument");
+  for (int i = 0; i < n; ++i) {
+    LASER_REQUIRE(seq_ids[i] >= 0 && seq_ids[i] < kv->max_seqs, "seq id %d out of range", seq_ids[i]);
+    LASER_REQUIRE(lens[i] >= 0 && lens[i] <= kv->capacity_tokens(), "length %d out of range", lens[i]);
+  }
+  for (int i = 0; i < n; ++i)
+    LASER_CUDA(cudaMemcpyAsync(kv->seq_len + seq_ids[i], lens + i, 4, cudaMemcpyHostToDevice, as_stream(stream)));
+  LASER_CUDA(cudaStreamSynchronize(as_stream(stream)));
+  return LASER_OK;
+}
+
+LASER_API laser_status laser_kv_set_len_dev(laser_kv* kv, const int32_t* lens_dev, int32_t n, void* stream) {
+  LASER_REQUIRE(kv && lens_dev && n >= 0 && n <= kv->max_seqs, "bad argument");
+  if (n == 0) return LASER_OK;
+  set_len_kernel<<<ceil_div(n, 256), 256, 0, as_stream(stream)>>>(kv->seq_len, lens_dev, n);
+  count_launch();
+  LASER_CUDA(cudaGetLastError());
+  return LASER_OK;
+}
+
+LASER_API laser_status laser_kv_get_len(const laser_kv* kv, const int32_t* seq_ids, int32_t* lens, int32_t n, void* stream) {
+  LASER_REQUIRE(kv && seq_ids && lens && n >= 0, "bad argument");
+  for (int i = 0; i < n; ++i) LASER_REQUIRE(seq_ids[i] >= 0 && seq_ids[i] < kv->max_seqs, "seq id %d out of range", seq_ids[i]);
+  for (int i = 0; i < n; ++i)
+    LASER_CUDA(cudaMemcpyAsync(lens + i, kv->seq_len + seq_ids[i], 4, cudaMemcpyDeviceToHost, as_stream(stream)));
+  LASER_CUDA(cudaStreamSynchronize(as_stream(stream)));
+  return LASER_OK;
+}
+
+static laser_status kv_copy(const laser_kv* kv, int32_t seq, int32_t layer, int32_t pos0, int32_t n,
+                            void* k, void* v, int to_pages, void* stream) {
+  LASER_REQUIRE(kv && k && v, "null argument");
+  LASER_REQUIRE(seq >= 0 && seq < kv->max_seqs && layer >= 0 && layer < kv->n_layers, "seq / layer out of range");
+  LASER_REQUIRE(pos0 >= 0 && n >= 0 && int64_t(pos0) + n <= kv->capacity_tokens(), "positions [%d, %d) outside the sequence's pages", pos0, pos0 + n);
+  if (n == 0) return LASER_OK;
+  const size_t total = size_t(n) * kv->n_kv_heads * kv->head_dim;
+  kv_copy_kernel<<<unsigned(std::min<size_t>(ceil_div<size_t>(total, 256), 4096)), 256, 0, as_stream(stream)>>>(
+      kv->pages + size_t(layer) * kv->layer_elems(), kv->page_elems(), kv->page_table + size_t(seq) * kv->pages_per_seq,
+      kv->n_kv_heads, kv->head_dim, pos0, n, static_cast<__nv_bfloat16*>(k), static_cast<__nv_bfloat16*>(v), to_pages);
+  count_launch();
+  LASER_CUDA(cudaGetLastError());
+  return LASER_OK;
+}
+
+LASER_API laser_status laser_kv_import(laser_kv* kv, int32_t seq, int32_t layer, int32_t pos0, int32_t n,
+                                       const void* k, const void* v, void* stream) {
+  return kv_copy(kv, seq, layer, pos0, n, const_cast<void*>(k), const_cast<void*>(v), 1, stream);
+}
+LASER_API laser_status laser_kv_export(const laser_kv* kv, int32_t seq, int32_t layer, int32_t pos0, int32_t n,
+                                       void* k, void* v, void* stream) {
+  return kv_copy(kv, seq, layer, pos0, n, k, v, 0, stream);
+}
+
+LASER_API laser_status laser_check(laser_model* m, void* stream) {
+  LASER_REQUIRE(m, "null model");
+  int32_t st = 0;
+  LASER_CUDA(cudaMemcpyAsync(&st, m->status, 4, cudaMemcpyDeviceToHost, as_stream(stream)));
+  LASER_CUDA(cudaStreamSynchronize(as_stream(stream)));
+  if (st != 0) {
+    LASER_CUDA(cudaMemsetAsync(m->status, 0, 4, as_stream(stream)));
+    set_error(st == LASER_ERR_CAPACITY ? "a sequence outgrew its KV pages"
+              : st == LASER_ERR_TIMEOUT ? "a device-side wait ran out" : "a step was given a bad sequence id");
+    return st;
+  }
+  return LASER_OK;
+}
+
+LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
+                                         const int32_t* n_rows, int32_t B, float* logits, void* stream_) {
+  LASER_REQUIRE(m && kv && seq_ids && tokens && n_rows && logits, "null argument");
+  LASER_REQUIRE(B >= 1 && B <= m->cfg.max_batch, "B = %d outside [1, max_batch = %d]", B, m->cfg.max_batch);
+  LASER_REQUIRE(kv->n_layers == m->cfg.n_layers && kv->n_kv_heads == m->cfg.n_kv_heads && kv->head_dim == m->cfg.head_dim,
+                "cache was created for another model shape");
+  cudaStream_t stream = as_stream(stream_);
+  const laser_model_cfg& c = m->cfg;
+  const int Rs = m->rows_per_seq, R = B * Rs, Rp = ceil_div(R, 16) * 16;
+  const int d = c.d_model, f = c.d_ffn, dh = c.head_dim, H = c.n_heads, Hkv = c.n_kv_heads;
+  const int capacity = int(std::min<int64_t>(kv->capacity_tokens(), INT32_MAX));
+
+  prep_rows_kernel<<<Rp, 64, 0, stream>>>(seq_ids, n_rows, B, Rs, Rp, kv->seq_len, kv->max_seqs, capacity, dh / 2,
+                                          double(c.rope_theta), dh, m->row_pos, m->row_seq, m->row_ctx, m->row_n,
+                                          m->rope, m->status);
+  const __nv_bfloat16* first_gain = c.n_layers > 0 ? m->attn_norm[0] : m->final_norm;
+  embed_norm_kernel<<<Rp, 256, 0, stream>>>(tokens, R, d, c.vocab, m->tok_emb, first_gain, c.rms_eps, m->resid, m->xn);
+  count_launch(2);
+  const size_t attn_smem = (size_t(dh) + size_t(capacity) + 8) * sizeof(float);
+  if (attn_smem > 48 * 1024) {
+    LASER_REQUIRE(attn_smem <= 200 * 1024, "KV capacity of %d tokens per sequence exceeds the attention kernel's limit", capacity);
+    LASER_CUDA(cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(attn_smem)));
+  }
+  for (int l = 0; l < c.n_layers; ++l) {
+    __nv_bfloat16* pages_l = kv->pages + size_t(l) * kv->layer_elems();
+    // QKV projection, rotary embedding, cache write
+    GemmPlan p1 = gemm_plan(Rp, m->dqkv, d);
+    size_t stride = size_t(Rp) * m->dqkv;
+    LASER_TRY(gemm_launch(m, m->xn, m->wqkv[l], m->part, Rp, Rp, m->dqkv, d, p1.splits, stride, m->dqkv, stream));
+    rope_kv_kernel<<<dim3(Rp, H + 2 * Hkv), 64, 0, stream>>>(m->part, p1.splits, stride, m->dqkv, H, Hkv, dh, m->rope,
+                                                             m->row_pos, m->row_seq, kv->page_table, kv->pages_per_seq,
+                                                             pages_l, kv->page_elems(), m->q);
+    attention_kernel<<<dim3(B, H), 128, attn_smem, stream>>>(m->q, seq_ids, m->row_ctx, m->row_n, Rs, H, Hkv, dh,
+                                                            kv->page_table, kv->pages_per_seq, pages_l,
+                                                            kv->page_elems(), m->attn);
+    // output projection, residual, norm
+    GemmPlan p2 = gemm_plan(Rp, d, m->dq);
+    stride = size_t(Rp) * d;
+    LASER_TRY(gemm_launch(m, m->attn, m->wo[l], m->part, Rp, Rp, d, m->dq, p2.splits, stride, d, stream));
+    residual_norm_kernel<<<Rp, 256, 0, stream>>>(m->part, p2.splits, stride, d, d, m->ffn_norm[l], c.rms_eps, m->resid, m->xn);
+    // SwiGLU feed-forward, residual, next norm
+    GemmPlan p3 = gemm_plan(Rp, 2 * f, d);
+    stride = size_t(Rp) * 2 * f;
+    LASER_TRY(gemm_launch(m, m->xn, m->wgu[l], m->part, Rp, Rp, 2 * f, d, p3.splits, stride, 2 * f, stream));
+    swiglu_kernel<<<dim3(ceil_div(f, 256), Rp), 256, 0, stream>>>(m->part, p3.splits, stride, f, m->act);
+    GemmPlan p4 = gemm_plan(Rp, d, f);
+    stride = size_t(Rp) * d;
+    LASER_TRY(gemm_launch(m, m->act, m->wdown[l], m->part, Rp, Rp, d, f, p4.splits, stride, d, stream));
+    const __nv_bfloat16* next_gain = l + 1 < c.n_layers ? m->attn_norm[l + 1] : m->final_norm;
+    residual_norm_kernel<<<Rp, 256, 0, stream>>>(m->part, p4.splits, stride, d, d, next_gain, c.rms_eps, m->resid, m->xn);
+    count_launch(5);
+  }
+  // LM head straight into the caller's logits (one plane, rows beyond R not stored)
+  LASER_TRY(gemm_launch(m, m->xn, m->lm_head, logits, Rp, R, c.vocab, d, 1, 0, c.vocab, stream));
+  LASER_CUDA(cudaGetLastError());
+  return LASER_OK;
+}
