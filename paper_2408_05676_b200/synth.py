@@ -215,7 +215,7 @@ def make_kv_layer(n_tokens: int, width: int, seed: int, layer: int, device: str 
                   ) -> Tuple[torch.Tensor, torch.Tensor]:
     """Synthetic cache contents of one layer: K, V ~ N(0,1) in bf16, [n_tokens, width]."""
     g = torch.Generator(device=device)
-    g.manual_seed(seed * 1000003 + layer)
+    g.manual_seed(int(seed) * 1000003 + int(layer))
     k = torch.randn(n_tokens, width, generator=g, device=device, dtype=torch.float32)
     v = torch.randn(n_tokens, width, generator=g, device=device, dtype=torch.float32)
     return k.to(torch.bfloat16), v.to(torch.bfloat16)
