@@ -32,8 +32,15 @@ def setup(L):
     # pool: the library's own greedy outputs on 12 other prompts, 3 per group
     pool_prompts = [synth.make_prompt(64, cfg["vocab"], 1000 + i) for i in range(12)]
     docs = L.generate(m, kv, None, pool_prompts, [0] * 12, L.make_params(K=8, max_new=200))["out"]
-    pool, offs = synth.pool_from_documents([docs[0:3], docs[3:6], docs[6:9], docs[9:12]])
     prompts = [synth.make_prompt(64, cfg["vocab"], 2000 + b) for b in range(4)]
+    # "old knowledge resembles new knowledge": each group also holds a corrupted copy of what
+    # its test prompt will generate, so drafts are found and are sometimes wrong
+    own = L.generate(m, kv, None, prompts, [0] * 4, L.make_params(K=8, max_new=64))["out"]
+    rng = np.random.default_rng(5)
+    for o in own:
+        for i in range(3, len(o), 11):
+            o[i] = int(rng.integers(0, cfg["vocab"]))
+    pool, offs = synth.pool_from_documents([docs[3 * g:3 * g + 3] + [own[g]] for g in range(4)])
     return cfg, Wc, m, kv, pool, offs, prompts
 
 
