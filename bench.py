@@ -1,0 +1,425 @@
+"""Benchmark of the Draft-Then-Verify hot path on the 7B-shape verify-step workload.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = draft retrieval (laser_draft) -> row assembly -> verify forward over
+[pending token + 8 drafts] for 16 sequences with 512 cached tokens each
+(laser_verify_step) -> acceptance + KV commit (laser_accept_commit), on seeded synthetic
+weights, cache and pool.  Prints one JSON line (rank 0).  `--impl reference` times the CPU
+oracle on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2408_05676_b200 import synth  # noqa: E402
+
+WORKLOAD = "verify-step-7b: batch 16, ctx 512 (16-token pages), 1+8 rows/seq, drafts 60% agreement"
+B, K, CTX, N_MAX = 16, 8, 512, 4
+POOL_TOKENS, POOL_GROUPS = 5_000_000, 1000
+SAMPLE_LAYERS = 4          # layers the CPU baseline really runs (time is extrapolated to all)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=float(d["hbm_gbs"]), source="measured")
+    return dict(hbm_gbs=6650.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.rows, self.proc, self.index = [], None, index
+
+    def __enter__(self):
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+
+
+# ---------------------------------------------------------------------------------------------
+def algorithmic_bytes(cfg, n_seqs, ctx, rows_per_seq):
+    d, f, V, Lr = cfg["d_model"], cfg["d_ffn"], cfg["vocab"], cfg["n_layers"]
+    dkv = cfg["n_kv_heads"] * cfg["head_dim"]
+    R = n_seqs * rows_per_seq
+    weights = 2 * (Lr * (2 * d * d + 2 * d * dkv + 3 * d * f) + d * V)
+    kv_read = n_seqs * ctx * Lr * 2 * dkv * 2
+    kv_write = R * Lr * 2 * dkv * 2
+    logits = 2 * R * V * 4
+    return dict(weights=weights, kv_read=kv_read, kv_write=kv_write, logits=logits,
+                total=weights + kv_read + kv_write + logits)
+
+
+def build_workload(L, dev, cfg):
+    """Weights, synthetic cache, greedy continuation, corrupted drafts, pool holding them."""
+    W = synth.make_weights(cfg, seed=0, device=dev)
+    model = L.model_create(cfg, W, max_batch=B)
+    pages_per_seq = (CTX + K + 1 + 15) // 16 + 1
+    kv = L.kv_create(model, B, B * pages_per_seq)
+    width = cfg["n_kv_heads"] * cfg["head_dim"]
+    for l in range(cfg["n_layers"]):
+        for s in range(B):
+            k, v = synth.make_kv_layer(CTX, width, 7 + 17 * s, l, device=dev)
+            L.kv_import(kv, s, l, 0, k, v)
+    seq_ids = torch.arange(B, dtype=torch.int32, device=dev)
+    lens = torch.full((B,), CTX, dtype=torch.int32, device=dev)
+    rng = np.random.default_rng(8)
+    last_np = rng.integers(0, cfg["vocab"], size=B).astype(np.int32)
+    # greedy continuation g_1..g_8 and the runner-up of each step, by 8 single-row steps
+    L.kv_set_len_dev(kv, lens)
+    tokens = torch.full((B, K + 1), -1, dtype=torch.int32, device=dev)
+    one = torch.ones(B, dtype=torch.int32, device=dev)
+    cur = torch.as_tensor(last_np, device=dev)
+    greedy, second = [], []
+    prm = L.make_params(K=K)
+    for _ in range(K):
+        tokens[:, 0] = cur
+        logits = L.verify_step(model, kv, seq_ids, tokens, one)
+        top2 = torch.topk(logits[:, 0], 2, dim=-1).indices
+        na, ot, no = L.accept_commit(kv, seq_ids, logits, tokens, one, prm)
+        cur = ot[:, 0].contiguous()
+        greedy.append(cur.cpu().numpy())
+        second.append(top2[:, 1].to(torch.int32).cpu().numpy())
+    L.check(model)
+    greedy, second = np.stack(greedy, 1), np.stack(second, 1)
+    drafts = synth.corrupt_drafts(greedy, second, cfg["vocab"], seed=8)
+    # pool: Zipf/template background; group of sequence b also holds "tail + drafts" as a document
+    pool, offs = synth.make_zipf_pool(POOL_TOKENS, POOL_GROUPS, vocab=cfg["vocab"], seed=42)
+    gid = (np.arange(B) * 61 % POOL_GROUPS).astype(np.int32)
+    tails = np.concatenate([rng.integers(0, cfg["vocab"], size=(B, N_MAX - 1)).astype(np.int32),
+                            last_np[:, None]], axis=1)
+    parts, new_offs = [], [0]
+    doc_of = {int(g): b for b, g in enumerate(gid)}
+    for g in range(POOL_GROUPS):
+        parts.append(pool[offs[g]:offs[g + 1]])
+        n = int(offs[g + 1] - offs[g])
+        if g in doc_of:
+            b = doc_of[g]
+            doc = np.concatenate([[synth.SENTINEL], tails[b], drafts[b]]).astype(np.int32)
+            parts.append(doc)
+            n += len(doc)
+        new_offs.append(new_offs[-1] + n)
+    pool = np.concatenate(parts)
+    offs = np.asarray(new_offs, dtype=np.int64)
+    return dict(cfg=cfg, W=W, model=model, kv=kv, seq_ids=seq_ids, lens=lens, last=last_np, tails=tails, gid=gid,
+                drafts=drafts, greedy=greedy, pool=pool, offs=offs)
+
+
+def run_ours(args):
+    from paper_2408_05676_b200 import binding as L
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = "cuda:%d" % local
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    cfg = synth.model_cfg("7b")
+    wl = build_workload(L, dev, cfg)
+    model, kv, seq_ids, lens = wl["model"], wl["kv"], wl["seq_ids"], wl["lens"]
+    t0 = time.time()
+    pool = L.pool_build(wl["pool"], wl["offs"], 1, N_MAX)
+    pool_build_s = time.time() - t0
+    V = cfg["vocab"]
+    d_tails = torch.as_tensor(wl["tails"], device=dev)
+    d_tl = torch.full((B,), N_MAX, dtype=torch.int32, device=dev)
+    d_gid = torch.as_tensor(wl["gid"], device=dev)
+    d_last = torch.as_tensor(wl["last"], device=dev)
+    draft = torch.empty(B, K, dtype=torch.int32, device=dev)
+    dlen = torch.empty(B, dtype=torch.int32, device=dev)
+    mn = torch.empty(B, dtype=torch.int32, device=dev)
+    tokens = torch.empty(B, K + 1, dtype=torch.int32, device=dev)
+    n_rows = torch.empty(B, dtype=torch.int32, device=dev)
+    logits = torch.empty(B, K + 1, V, dtype=torch.float32, device=dev)
+    outs = (torch.empty(B, dtype=torch.int32, device=dev), torch.empty(B, K + 1, dtype=torch.int32, device=dev),
+            torch.empty(B, dtype=torch.int32, device=dev))
+
+    def step(prm):
+        L.kv_set_len_dev(kv, lens)
+        L.draft(pool, d_tails, d_tl, d_gid, prm, draft, dlen, mn)
+        L.make_rows(d_last, draft, dlen, K, tokens, n_rows)
+        L.verify_step(model, kv, seq_ids, tokens, n_rows, logits)
+        L.accept_commit(kv, seq_ids, logits, tokens, n_rows, prm, out=outs)
+
+    strict = L.make_params(K=K, n_min=1, n_max=N_MAX, max_occ=64, mode=L.MODE_STRICT)
+    step(strict)
+    torch.cuda.synchronize()
+    L.check(model)
+    assert (draft.cpu().numpy() == wl["drafts"]).all(), "retrieved drafts differ from the planted ones"
+    # calibrated threshold: median runner-up probability on this step's logits
+    probs = torch.softmax(logits.reshape(-1, V), dim=-1)
+    p_cal = float(torch.topk(probs, 2, dim=-1).values[:, 1].median())
+    modes = dict(strict=strict,
+                 relaxed_paper=L.make_params(K=K, n_min=1, n_max=N_MAX, max_occ=64, mode=L.MODE_RELAXED, topk=2, p=0.1),
+                 relaxed_cal=L.make_params(K=K, n_min=1, n_max=N_MAX, max_occ=64, mode=L.MODE_RELAXED, topk=2, p=p_cal))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(prm, steps, warmup, sample_clocks=False):
+        for _ in range(warmup):
+            step(prm)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = L.launch_count()
+        sampler = ClockSampler(local) if sample_clocks else None
+        if sampler:
+            sampler.__enter__()
+        e0.record()
+        for _ in range(steps):
+            step(prm)
+        e1.record()
+        barrier()
+        if sampler:
+            sampler.__exit__()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t[0])
+        n_out = int(outs[2].sum())
+        n_acc = int(outs[0].sum())
+        return dict(ms=ms / steps, tokens=n_out, accepted=n_acc, launches=(L.launch_count() - l0) // steps,
+                    clocks=sampler.summary() if sampler else None)
+
+    res = {name: timed(prm, args.steps, args.warmup, sample_clocks=(name == "strict")) for name, prm in modes.items()}
+    main = res["strict"]
+    value = world * main["tokens"] / (main["ms"] * 1e-3)
+
+    # kernel-class profile: verify-step, dense-contraction and attention device time per step
+    L.profile_enable(model, True)
+    L.profile_read(model, 0), L.profile_read(model, 1)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * args.steps)]
+    for i in range(args.steps):
+        L.kv_set_len_dev(kv, lens)
+        L.draft(pool, d_tails, d_tl, d_gid, strict, draft, dlen, mn)
+        L.make_rows(d_last, draft, dlen, K, tokens, n_rows)
+        ev[2 * i].record()
+        L.verify_step(model, kv, seq_ids, tokens, n_rows, logits)
+        ev[2 * i + 1].record()
+        L.accept_commit(kv, seq_ids, logits, tokens, n_rows, strict, out=outs)
+    torch.cuda.synchronize()
+    gemm_ms, gemm_n = L.profile_read(model, 0)
+    attn_ms, attn_n = L.profile_read(model, 1)
+    L.profile_enable(model, False)
+    verify_ms = sum(ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(args.steps)) / args.steps
+    gemm_ms /= args.steps
+    attn_ms /= args.steps
+
+    # end to end: step inputs from pinned host memory, results back to the host, every step
+    h_in = [t.cpu().pin_memory() for t in (d_tails, d_tl, d_gid, d_last)]
+    h_out = [torch.empty_like(t, device="cpu").pin_memory() for t in outs]
+
+    def e2e_step():
+        for h, d in zip(h_in, (d_tails, d_tl, d_gid, d_last)):
+            d.copy_(h, non_blocking=True)
+        step(strict)
+        for h, d in zip(h_out, outs):
+            h.copy_(d, non_blocking=True)
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / args.steps
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t[0])
+    e2e_value = world * int(h_out[2].sum()) / (e2e_ms * 1e-3)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    peaks = measured_peaks()
+    ab = algorithmic_bytes(cfg, B, CTX, K + 1)
+    gemm_gbs = ab["weights"] / (gemm_ms * 1e-3) / 1e9
+    out = {
+        "metric": "generated_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": main["ms"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "model_shape": "llama-2-7b", "batch": B, "ctx": CTX, "draft_len": K,
+                   "pool_tokens": int(len(wl["pool"])), "pool_groups": POOL_GROUPS, "suffix_n": [1, N_MAX],
+                   "max_occ": 64, "l2": "inputs larger than L2 (13.2 GB of weights + 4.3 GB of KV per step)",
+                   "parallelism": "replicas x%d" % world},
+        "clocks": main["clocks"],
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in h_in)),
+                "d2h_bytes_per_step": int(sum(t.numel() * t.element_size() for t in h_out))},
+        "gpu_launches": int(main["launches"] * args.steps),
+        "roofline": {"kernel": "gemm_tc_kernel (all dense contractions of one verify step)", "bound": "hbm",
+                     "achieved": gemm_gbs, "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
+                     "frac": gemm_gbs / peaks["hbm_gbs"], "traffic": None,
+                     "algorithmic_bytes_per_step": ab["weights"], "ms_per_step": gemm_ms, "launches_per_step": gemm_n // args.steps},
+        "verify_step": {"ms": verify_ms, "algorithmic_bytes": ab["total"],
+                        "achieved_gbs": ab["total"] / (verify_ms * 1e-3) / 1e9,
+                        "frac_of_measured_hbm": ab["total"] / (verify_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                        "frac_of_nominal_8tbs": ab["total"] / (verify_ms * 1e-3) / 1e9 / 8000.0,
+                        "gemm_ms": gemm_ms, "attention_ms": attn_ms, "other_ms": verify_ms - gemm_ms - attn_ms},
+        "acceptance": {name: {"tokens_per_s": world * r["tokens"] / (r["ms"] * 1e-3), "ms_per_step": r["ms"],
+                              "accepted_drafts_per_step": r["accepted"] / B, "emitted_per_step": r["tokens"] / B}
+                       for name, r in res.items()},
+        "p_cal": p_cal, "pool_build_s": pool_build_s, "launches_per_step": int(main["launches"]),
+    }
+    out["cpu_baseline"] = cpu_baseline(wl, sample="1 of 16 sequences, %d of 32 layers run, time extrapolated" % SAMPLE_LAYERS)
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------------
+def oracle_sample(cfg, W_cpu, kv_rows, pool, offs, tail, gid, repeat=1):
+    """One sequence through the oracle: draft, forward over SAMPLE_LAYERS layers (timed apart from
+    the embedding/LM-head part so that the time can be scaled to all layers), acceptance."""
+    from oracle import accept as OA
+    from oracle import forward as OF
+    from oracle import retrieval as OR
+    cfg_s = dict(cfg, n_layers=SAMPLE_LAYERS)
+    cfg_0 = dict(cfg, n_layers=0)
+    W0 = dict(W_cpu, layers=[])
+    times = []
+    for _ in range(repeat):
+        t0 = time.perf_counter()
+        d, _ = OR.draft_one(pool, int(offs[gid]), int(offs[gid + 1]), tail, K, 1, N_MAX, 1, 64)
+        rows = np.asarray([tail[-1]] + d, np.int32)
+        t1 = time.perf_counter()
+        okv = OF.KVCache(cfg_s, 1, CTX + K + 2)
+        for l in range(SAMPLE_LAYERS):
+            okv.k[l, 0, :CTX] = kv_rows[l][0].view(CTX, cfg["n_kv_heads"], cfg["head_dim"])
+            okv.v[l, 0, :CTX] = kv_rows[l][1].view(CTX, cfg["n_kv_heads"], cfg["head_dim"])
+        okv.ctx[0] = CTX
+        t2 = time.perf_counter()
+        logits = OF.forward(W_cpu, cfg_s, okv, [0], [rows])[0]
+        t3 = time.perf_counter()
+        OF.forward(W0, cfg_0, OF.KVCache(cfg_0, 1, 16), [0], [rows])
+        t4 = time.perf_counter()
+        a, em = OA.accept_one(logits.float().numpy(), rows, len(rows), OA.STRICT, 2, 0.1)
+        t5 = time.perf_counter()
+        head = t4 - t3
+        per_layer = max((t3 - t2) - head, 0.0) / SAMPLE_LAYERS
+        total = (t1 - t0) + head + per_layer * cfg["n_layers"] + (t5 - t4)
+        times.append((total, len(em)))
+    return times
+
+
+def cpu_baseline(wl, sample):
+    cfg = wl["cfg"]
+    W = wl["W"]
+    W_cpu = dict(tok_emb=W["tok_emb"].cpu(), lm_head=W["lm_head"].cpu(), final_norm=W["final_norm"].cpu(),
+                 layers=[{k: v.cpu() for k, v in lw.items()} for lw in W["layers"][:SAMPLE_LAYERS]])
+    width = cfg["n_kv_heads"] * cfg["head_dim"]
+    kv_rows = [tuple(t.cpu() for t in synth.make_kv_layer(CTX, width, 7, l, device=str(W["tok_emb"].device)))
+               for l in range(SAMPLE_LAYERS)]
+    total, n_tok = oracle_sample(cfg, W_cpu, kv_rows, wl["pool"], wl["offs"], wl["tails"][0], int(wl["gid"][0]))[0]
+    return {"value": n_tok / total, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle",
+            "sample": sample, "seconds_extrapolated": total}
+
+
+def run_reference(args):
+    """CPU oracle on a bounded sample of the same workload; rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    cfg = synth.model_cfg("7b")
+    cfg_s = dict(cfg, n_layers=SAMPLE_LAYERS)
+    W_cpu = synth.make_weights(cfg_s, seed=0, device="cpu")
+    width = cfg["n_kv_heads"] * cfg["head_dim"]
+    kv_rows = [synth.make_kv_layer(CTX, width, 7, l) for l in range(SAMPLE_LAYERS)]
+    pool, offs = synth.make_zipf_pool(POOL_TOKENS // 10, POOL_GROUPS // 10, vocab=cfg["vocab"], seed=42)
+    rng = np.random.default_rng(8)
+    st = int(offs[3]) + 100
+    tail = pool[st:st + N_MAX].copy()          # a tail that occurs in its group, so a draft is found
+    times = oracle_sample(cfg, W_cpu, kv_rows, pool, offs, tail, 3, repeat=args.warmup + args.steps)[args.warmup:]
+    total = sum(t for t, _ in times)
+    toks = sum(n for _, n in times)
+    value = toks / total
+    sample = ("per step: 1 of 16 sequences, %d of 32 layers run and time extrapolated to 32; pool %d tokens"
+              % (SAMPLE_LAYERS, len(pool)))
+    print(json.dumps({
+        "impl": "reference", "metric": "generated_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "model_shape": "llama-2-7b", "batch": B, "ctx": CTX, "draft_len": K},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

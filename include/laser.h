@@ -201,6 +201,13 @@ laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int32_t* seq_
  * check (CAPACITY, TIMEOUT), clearing it. */
 laser_status laser_check(laser_model* m, void* stream);
 
+/* Measurement aid for the forward of Eq. 3: while enabled, every dense-contraction launch
+ * (class 0) and every attention launch (class 1) of laser_verify_step is bracketed by CUDA
+ * events on the call's stream.  laser_profile_read synchronises the device and returns the
+ * summed device time and the number of launches of one class since the previous read. */
+laser_status laser_profile_enable(laser_model* m, int32_t on);
+laser_status laser_profile_read(laser_model* m, int32_t cls, double* ms, int64_t* launches);
+
 /* ---- Acceptance and commit (Section 2.1, Section 3.4, Eq. 4 / Eq. 7 / Eq. 8) ------------
  * Drafts are verified in order against rows 0.. of the logits; n_accept[b] = drafts that
  * pass before the first failure; out_tokens[b] = those drafts followed by arg max of row

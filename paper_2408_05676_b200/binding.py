@@ -60,7 +60,7 @@ EXPORTS = ["laser_version", "laser_last_error", "laser_launch_count", "laser_poo
            "laser_pool_info", "laser_draft", "laser_make_rows", "laser_model_create", "laser_model_free",
            "laser_kv_create", "laser_kv_free", "laser_kv_set_page_table", "laser_kv_set_len",
            "laser_kv_get_len", "laser_kv_set_len_dev", "laser_kv_import", "laser_kv_export",
-           "laser_verify_step", "laser_check", "laser_accept_commit", "laser_generate"]
+           "laser_verify_step", "laser_check", "laser_profile_enable", "laser_profile_read", "laser_accept_commit", "laser_generate"]
 
 lib.laser_version.restype = C.c_char_p
 lib.laser_last_error.restype = C.c_char_p
@@ -275,6 +275,17 @@ def verify_step(model: Model, kv: KV, seq_ids, tokens, n_rows, logits=None, stre
                                _ptr(_dev(tokens, torch.int32)), _ptr(_dev(n_rows, torch.int32)),
                                C.c_int32(B), _ptr(_dev(logits, torch.float32)), _stream(stream)))
     return logits
+
+
+def profile_enable(model: Model, on: bool) -> None:
+    _chk(lib.laser_profile_enable(model.handle, C.c_int32(1 if on else 0)))
+
+
+def profile_read(model: Model, cls: int):
+    """Returns (device ms, launches) of class 0 (dense contractions) or 1 (attention)."""
+    ms, n = C.c_double(), C.c_int64()
+    _chk(lib.laser_profile_read(model.handle, C.c_int32(cls), C.byref(ms), C.byref(n)))
+    return ms.value, n.value
 
 
 def check(model: Model, stream=None) -> None:

@@ -265,14 +265,50 @@ laser_status fuse_rows(laser_model* m, const void* const* pieces, const size_t* 
   return LASER_OK;
 }
 
+// Brackets one launch with events when profiling is on.
+struct ProfScope {
+  laser_model* m; int cls; cudaStream_t st; bool on;
+  ProfScope(laser_model* m_, int cls_, cudaStream_t st_) : m(m_), cls(cls_), st(st_), on(m_->profile) { mark(); }
+  ~ProfScope() { mark(); }
+  void mark() {
+    if (!on) return;
+    auto& ev = m->prof_events[cls];
+    size_t& used = m->prof_used[cls];
+    if (used == ev.size()) { cudaEvent_t e; if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; } ev.push_back(e); }
+    cudaEventRecord(ev[used++], st);
+  }
+};
+
 }  // namespace
 }  // namespace laser
 
 using namespace laser;
 
+LASER_API laser_status laser_profile_enable(laser_model* m, int32_t on) {
+  LASER_REQUIRE(m, "null model");
+  m->profile = on != 0;
+  return LASER_OK;
+}
+
+LASER_API laser_status laser_profile_read(laser_model* m, int32_t cls, double* ms, int64_t* launches) {
+  LASER_REQUIRE(m && ms && launches && cls >= 0 && cls < 2, "bad argument");
+  LASER_CUDA(cudaDeviceSynchronize());
+  double total = 0;
+  const size_t n = m->prof_used[cls] / 2;
+  for (size_t i = 0; i < n; ++i) {
+    float t = 0;
+    LASER_CUDA(cudaEventElapsedTime(&t, m->prof_events[cls][2 * i], m->prof_events[cls][2 * i + 1]));
+    total += t;
+  }
+  m->prof_used[cls] = 0;
+  *ms = total; *launches = int64_t(n);
+  return LASER_OK;
+}
+
 LASER_API laser_status laser_model_free(laser_model* m) {
   if (!m) return LASER_OK;
   gemm_state_free(m);
+  for (auto& v : m->prof_events) for (cudaEvent_t e : v) cudaEventDestroy(e);
   for (void* p : m->owned) cudaFree(p);
   delete m;
   return LASER_OK;
@@ -477,32 +513,33 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
     // QKV projection, rotary embedding, cache write
     GemmPlan p1 = gemm_plan(Rp, m->dqkv, d);
     size_t stride = size_t(Rp) * m->dqkv;
-    LASER_TRY(gemm_launch(m, m->xn, m->wqkv[l], m->part, Rp, Rp, m->dqkv, d, p1.splits, stride, m->dqkv, stream));
+    { ProfScope ps(m, 0, stream); LASER_TRY(gemm_launch(m, m->xn, m->wqkv[l], m->part, Rp, Rp, m->dqkv, d, p1.splits, stride, m->dqkv, stream)); }
     rope_kv_kernel<<<dim3(Rp, H + 2 * Hkv), 64, 0, stream>>>(m->part, p1.splits, stride, m->dqkv, H, Hkv, dh, m->rope,
                                                              m->row_pos, m->row_seq, kv->page_table, kv->pages_per_seq,
                                                              pages_l, kv->page_elems(), m->q);
-    attention_kernel<<<dim3(B, H), 128, attn_smem, stream>>>(m->q, seq_ids, m->row_ctx, m->row_n, Rs, H, Hkv, dh,
-                                                            kv->page_table, kv->pages_per_seq, pages_l,
-                                                            kv->page_elems(), m->attn);
+    { ProfScope ps(m, 1, stream);
+      attention_kernel<<<dim3(B, H), 128, attn_smem, stream>>>(m->q, seq_ids, m->row_ctx, m->row_n, Rs, H, Hkv, dh,
+                                                              kv->page_table, kv->pages_per_seq, pages_l,
+                                                              kv->page_elems(), m->attn); }
     // output projection, residual, norm
     GemmPlan p2 = gemm_plan(Rp, d, m->dq);
     stride = size_t(Rp) * d;
-    LASER_TRY(gemm_launch(m, m->attn, m->wo[l], m->part, Rp, Rp, d, m->dq, p2.splits, stride, d, stream));
+    { ProfScope ps(m, 0, stream); LASER_TRY(gemm_launch(m, m->attn, m->wo[l], m->part, Rp, Rp, d, m->dq, p2.splits, stride, d, stream)); }
     residual_norm_kernel<<<Rp, 256, 0, stream>>>(m->part, p2.splits, stride, d, d, m->ffn_norm[l], c.rms_eps, m->resid, m->xn);
     // SwiGLU feed-forward, residual, next norm
     GemmPlan p3 = gemm_plan(Rp, 2 * f, d);
     stride = size_t(Rp) * 2 * f;
-    LASER_TRY(gemm_launch(m, m->xn, m->wgu[l], m->part, Rp, Rp, 2 * f, d, p3.splits, stride, 2 * f, stream));
+    { ProfScope ps(m, 0, stream); LASER_TRY(gemm_launch(m, m->xn, m->wgu[l], m->part, Rp, Rp, 2 * f, d, p3.splits, stride, 2 * f, stream)); }
     swiglu_kernel<<<dim3(ceil_div(f, 256), Rp), 256, 0, stream>>>(m->part, p3.splits, stride, f, m->act);
     GemmPlan p4 = gemm_plan(Rp, d, f);
     stride = size_t(Rp) * d;
-    LASER_TRY(gemm_launch(m, m->act, m->wdown[l], m->part, Rp, Rp, d, f, p4.splits, stride, d, stream));
+    { ProfScope ps(m, 0, stream); LASER_TRY(gemm_launch(m, m->act, m->wdown[l], m->part, Rp, Rp, d, f, p4.splits, stride, d, stream)); }
     const __nv_bfloat16* next_gain = l + 1 < c.n_layers ? m->attn_norm[l + 1] : m->final_norm;
     residual_norm_kernel<<<Rp, 256, 0, stream>>>(m->part, p4.splits, stride, d, d, next_gain, c.rms_eps, m->resid, m->xn);
     count_launch(5);
   }
   // LM head straight into the caller's logits (one plane, rows beyond R not stored)
-  LASER_TRY(gemm_launch(m, m->xn, m->lm_head, logits, Rp, R, c.vocab, d, 1, 0, c.vocab, stream));
+  { ProfScope ps(m, 0, stream); LASER_TRY(gemm_launch(m, m->xn, m->lm_head, logits, Rp, R, c.vocab, d, 1, 0, c.vocab, stream)); }
   LASER_CUDA(cudaGetLastError());
   return LASER_OK;
 }

@@ -28,6 +28,10 @@ struct laser_model {
   int32_t* row_n = nullptr;        // [max_batch] effective rows of each sequence
   int32_t* status = nullptr;       // first device-side error of the stream, 0 = none
   void* gemm_state = nullptr;      // tensor-map cache of the tensor-core GEMM
+  // optional per-class kernel timing (class 0 = GEMM, 1 = attention)
+  bool profile = false;
+  std::vector<cudaEvent_t> prof_events[2];  // begin/end pairs
+  size_t prof_used[2] = {0, 0};
 };
 
 namespace laser {
