@@ -1,0 +1,267 @@
+// Causal attention of the verify forward (Eq. 3 / Eq. 6, chain form of the mask): the K+1
+// rows of a sequence against its paged bf16 KV cache, which already holds the rows' own K/V.
+//
+// One CTA per (sequence, head, 16-row tile).  A producer warp walks the sequence's page table
+// and streams each 16-token page of K and V through TMA (128-byte swizzle) into a ring of
+// shared-memory stages; four consumer warps take pages round-robin, compute S = Q K^T and
+// O += P V with warp-level MMA (the rows are 16 at most, far below a tensor-memory tile),
+// keep an online softmax with warp-shuffle row reductions, and merge their partial
+// (max, sum, O) through shared memory at the end.  A page is read from HBM exactly once and
+// used by exactly one warp.  Every mbarrier wait is bounded.
+#include "model.cuh"
+#include "tma.cuh"
+
+namespace laser {
+namespace {
+
+using bf16 = __nv_bfloat16;
+constexpr int kConsumers = 4;
+constexpr int kAttnThreads = (kConsumers + 1) * 32;
+constexpr int kStages = 8;   // a multiple of kConsumers: stage s always serves warp s % 4
+
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int DH>
+__global__ void __launch_bounds__(kAttnThreads)
+attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restrict__ q,
+                  const int32_t* __restrict__ seq_ids, const int32_t* __restrict__ row_ctx,
+                  const int32_t* __restrict__ row_n, int Rs, int H, int Hkv,
+                  const int32_t* __restrict__ page_table, int pages_per_seq, int layer_row0,
+                  bf16* __restrict__ out, int32_t* __restrict__ status) {
+  constexpr int HALVES = DH / 64;                 // 64-element (128-byte) column blocks per row
+  constexpr int SUB = 16 * 128;                   // bytes of one 16-token x 64-element sub-tile
+  constexpr int STAGE = 2 * HALVES * SUB;         // K then V
+  constexpr int QLD = DH + 8;                     // padded row of the Q tile (elements)
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t full_bar[kStages], empty_bar[kStages];
+  __shared__ float s_m[kConsumers][16], s_l[kConsumers][16];
+  __shared__ int abort_flag;
+
+  const int b = blockIdx.x, h = blockIdx.y, mt = blockIdx.z;
+  const int hk = h / (H / Hkv);
+  const int nr = row_n[b], ctx = row_ctx[b];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int row0 = mt * 16;
+  bf16* obase = out + (size_t(b) * Rs + row0) * H * DH + size_t(h) * DH;
+  if (row0 >= nr) {  // nothing active in this tile: zero its rows
+    for (int idx = tid; idx < 16 * DH; idx += kAttnThreads) {
+      const int r = idx / DH, d = idx % DH;
+      if (row0 + r < Rs) obase[size_t(r) * H * DH + d] = __float2bfloat16(0.f);
+    }
+    return;
+  }
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;
+  uint8_t* tiles_ptr = smem_raw + (tiles - raw);
+  const uint32_t q_smem = tiles + kStages * STAGE;
+  bf16* q_ptr = reinterpret_cast<bf16*>(tiles_ptr + kStages * STAGE);
+  const int n_keys = ctx + nr;
+  const int n_pg = (n_keys + 15) >> 4;
+
+  if (tid == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
+    mbar_fence_init();
+    tma_prefetch_map(&kvmap);
+  }
+  // Q tile: rows of this sequence, zero beyond the active ones
+  for (int idx = tid; idx < 16 * (DH / 8); idx += kAttnThreads) {
+    const int r = idx / (DH / 8), c = idx % (DH / 8);
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (row0 + r < nr) v = *reinterpret_cast<const uint4*>(q + (size_t(b) * Rs + row0 + r) * H * DH + size_t(h) * DH + c * 8);
+    *reinterpret_cast<uint4*>(q_ptr + r * QLD + c * 8) = v;
+  }
+  __syncthreads();
+
+  if (warp == kConsumers) {  // producer
+    if (lane == 0) {
+      const int32_t* pt = page_table + size_t(seq_ids[b]) * pages_per_seq;
+      bool ok = true;
+      int issued = 0;
+      for (int p = 0; p < n_pg && ok; ++p) {
+        const int s = p % kStages;
+        if (p >= kStages) ok = mbar_wait(smem_u32(&empty_bar[s]), ((p / kStages) - 1) & 1, &abort_flag);
+        if (!ok) break;
+        const uint32_t bar = smem_u32(&full_bar[s]);
+        const uint32_t dst = tiles + uint32_t(s) * STAGE;
+        mbar_expect_tx(bar, STAGE);
+        const int phys = pt[p];
+        const int rowk = layer_row0 + ((phys * 2) * Hkv + hk) * 16;
+        const int rowv = layer_row0 + ((phys * 2 + 1) * Hkv + hk) * 16;
+#pragma unroll
+        for (int hf = 0; hf < HALVES; ++hf) {
+          tma_load_2d(dst + hf * SUB, &kvmap, hf * 64, rowk, bar);
+          tma_load_2d(dst + (HALVES + hf) * SUB, &kvmap, hf * 64, rowv, bar);
+        }
+        issued = p + 1;
+      }
+      if (!ok)
+        for (int p = max(0, issued - kStages); p < issued; ++p) mbar_drain(smem_u32(&full_bar[p % kStages]), (p / kStages) & 1);
+    }
+    return;
+  }
+
+  // ---- consumers ----
+  const int g = lane >> 2, qd = lane & 3;
+  const float sl2 = rsqrtf(float(DH)) * 1.4426950408889634f;
+  uint32_t qf[DH / 16][4];
+  {
+    const int mat = lane >> 3, r = (lane & 7) + (mat & 1) * 8;
+#pragma unroll
+    for (int ks = 0; ks < DH / 16; ++ks) ldsm_x4(qf[ks], q_smem + uint32_t(r * QLD + ks * 16 + (mat >> 1) * 8) * 2);
+  }
+  float o[DH / 8][4];
+#pragma unroll
+  for (int t = 0; t < DH / 8; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+  // last key each of this lane's two rows may see; inactive rows copy the last active row
+  const int lim0 = ctx + min(row0 + g, nr - 1), lim1 = ctx + min(row0 + g + 8, nr - 1);
+
+  for (int p = warp; p < n_pg; p += kConsumers) {
+    const int s = p % kStages;
+    if (!mbar_wait(smem_u32(&full_bar[s]), (p / kStages) & 1, &abort_flag)) break;
+    const uint32_t kbase = tiles + uint32_t(s) * STAGE, vbase = kbase + HALVES * SUB;
+    float sc[2][4];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) sc[t][0] = sc[t][1] = sc[t][2] = sc[t][3] = 0.f;
+    {
+      const int mat = lane >> 3, key = (lane & 7) + (mat >> 1) * 8;
+#pragma unroll
+      for (int ks = 0; ks < DH / 16; ++ks) {
+        const int c = (ks & 3) * 2 + (mat & 1);
+        uint32_t kb[4];
+        ldsm_x4(kb, kbase + (ks >> 2) * SUB + key * 128 + ((c ^ (key & 7)) << 4));
+        mma16816(sc[0], qf[ks], kb[0], kb[1]);
+        mma16816(sc[1], qf[ks], kb[2], kb[3]);
+      }
+    }
+    // causal mask, online softmax (rows g and g+8 of the tile)
+    const int key0 = p * 16 + 2 * qd;
+    float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+    for (int t = 0; t < 2; ++t)
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        const int key = key0 + t * 8 + c;
+        if (key > lim0) sc[t][c] = -INFINITY;
+        if (key > lim1) sc[t][2 + c] = -INFINITY;
+        mx0 = fmaxf(mx0, sc[t][c]);
+        mx1 = fmaxf(mx1, sc[t][2 + c]);
+      }
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+    const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
+    const float mu0 = mn0 == -INFINITY ? 0.f : mn0, mu1 = mn1 == -INFINITY ? 0.f : mn1;
+    const float al0 = exp2f((m_run[0] - mu0) * sl2), al1 = exp2f((m_run[1] - mu1) * sl2);
+    m_run[0] = mn0; m_run[1] = mn1;
+    uint32_t pf[4];
+    float ps0 = 0.f, ps1 = 0.f;
+    {
+      const float p00 = exp2f((sc[0][0] - mu0) * sl2), p01 = exp2f((sc[0][1] - mu0) * sl2);
+      const float p02 = exp2f((sc[0][2] - mu1) * sl2), p03 = exp2f((sc[0][3] - mu1) * sl2);
+      const float p10 = exp2f((sc[1][0] - mu0) * sl2), p11 = exp2f((sc[1][1] - mu0) * sl2);
+      const float p12 = exp2f((sc[1][2] - mu1) * sl2), p13 = exp2f((sc[1][3] - mu1) * sl2);
+      ps0 = p00 + p01 + p10 + p11;
+      ps1 = p02 + p03 + p12 + p13;
+      pf[0] = pack_bf16(p00, p01);   // row g,   keys 2q..   (k low)
+      pf[1] = pack_bf16(p02, p03);   // row g+8, keys 2q..
+      pf[2] = pack_bf16(p10, p11);   // row g,   keys 8+2q.. (k high)
+      pf[3] = pack_bf16(p12, p13);   // row g+8, keys 8+2q..
+    }
+    l_run[0] = l_run[0] * al0 + ps0;
+    l_run[1] = l_run[1] * al1 + ps1;
+#pragma unroll
+    for (int t = 0; t < DH / 8; ++t) { o[t][0] *= al0; o[t][1] *= al0; o[t][2] *= al1; o[t][3] *= al1; }
+    {
+      const int mat = lane >> 3, key = (lane & 7) + (mat & 1) * 8;
+#pragma unroll
+      for (int j = 0; j < DH / 16; ++j) {
+        const int c = (j & 3) * 2 + (mat >> 1);
+        uint32_t vb[4];
+        ldsm_x4_t(vb, vbase + (j >> 2) * SUB + key * 128 + ((c ^ (key & 7)) << 4));
+        mma16816(o[2 * j], pf, vb[0], vb[1]);
+        mma16816(o[2 * j + 1], pf, vb[2], vb[3]);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&empty_bar[s]));
+  }
+
+  // ---- merge the four partial results ----
+  l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1); l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
+  l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 1); l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 2);
+  asm volatile("bar.sync 1, 128;" ::: "memory");   // every page consumed: the stages are free
+  float* s_o = reinterpret_cast<float*>(tiles_ptr);  // [consumer][16][DH]
+  if (qd == 0) { s_m[warp][g] = m_run[0]; s_m[warp][g + 8] = m_run[1]; s_l[warp][g] = l_run[0]; s_l[warp][g + 8] = l_run[1]; }
+#pragma unroll
+  for (int t = 0; t < DH / 8; ++t) {
+    *reinterpret_cast<float2*>(s_o + (warp * 16 + g) * DH + t * 8 + 2 * qd) = make_float2(o[t][0], o[t][1]);
+    *reinterpret_cast<float2*>(s_o + (warp * 16 + g + 8) * DH + t * 8 + 2 * qd) = make_float2(o[t][2], o[t][3]);
+  }
+  asm volatile("bar.sync 1, 128;" ::: "memory");
+  for (int idx = tid; idx < 16 * DH; idx += kConsumers * 32) {
+    const int r = idx / DH, d = idx % DH;
+    if (row0 + r >= Rs) continue;
+    float mt_ = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kConsumers; ++w) mt_ = fmaxf(mt_, s_m[w][r]);
+    float num = 0.f, den = 0.f;
+#pragma unroll
+    for (int w = 0; w < kConsumers; ++w) {
+      const float e = s_m[w][r] == -INFINITY ? 0.f : exp2f((s_m[w][r] - mt_) * sl2);
+      num += e * s_o[(w * 16 + r) * DH + d];
+      den += e * s_l[w][r];
+    }
+    const bool live = row0 + r < nr && den > 0.f && !abort_flag;
+    obase[size_t(r) * H * DH + d] = __float2bfloat16(live ? num / den : 0.f);
+  }
+  if (tid == 0 && abort_flag) atomicCAS(status, 0, LASER_ERR_TIMEOUT);
+}
+
+}  // namespace
+
+bool attention_tma_supported(const laser_model* m, const laser_kv* kv) {
+  return kv->has_pages_map && (m->cfg.head_dim == 64 || m->cfg.head_dim == 128);
+}
+
+laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const int32_t* seq_ids, int B,
+                                  cudaStream_t stream) {
+  const int dh = m->cfg.head_dim, H = m->cfg.n_heads, Hkv = m->cfg.n_kv_heads, Rs = m->rows_per_seq;
+  const int64_t rows_per_layer = int64_t(kv->n_pages) * 2 * Hkv * 16;
+  const int layer_row0 = int(rows_per_layer * layer);
+  const size_t smem = 1024 + size_t(kStages) * (2 * (dh / 64) * 16 * 128) + size_t(16) * (dh + 8) * 2;
+  dim3 grid(B, H, ceil_div(Rs, 16));
+  if (dh == 128) {
+    LASER_CUDA(cudaFuncSetAttribute(attn_paged_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+    attn_paged_kernel<128><<<grid, kAttnThreads, smem, stream>>>(kv->pages_map, m->q, seq_ids, m->row_ctx, m->row_n, Rs, H,
+                                                                 Hkv, kv->page_table, kv->pages_per_seq, layer_row0,
+                                                                 m->attn, m->status);
+  } else {
+    LASER_CUDA(cudaFuncSetAttribute(attn_paged_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+    attn_paged_kernel<64><<<grid, kAttnThreads, smem, stream>>>(kv->pages_map, m->q, seq_ids, m->row_ctx, m->row_n, Rs, H,
+                                                                Hkv, kv->page_table, kv->pages_per_seq, layer_row0,
+                                                                m->attn, m->status);
+  }
+  count_launch();
+  LASER_CUDA(cudaGetLastError());
+  return LASER_OK;
+}
+
+}  // namespace laser

@@ -14,12 +14,11 @@
 // stages with tcgen05.commit; warps 2-5 read the accumulator with tcgen05.ld and store it
 // transposed (token-major).  Every wait is bounded: on expiry the CTA records
 // LASER_ERR_TIMEOUT, drains its copies, frees its TMEM and exits.
-#include <cuda.h>
-
 #include <map>
 #include <tuple>
 
 #include "model.cuh"
+#include "tma.cuh"
 
 namespace laser {
 namespace {
@@ -90,41 +89,6 @@ constexpr int kBM = 128;          // weight rows per tile (MMA M)
 constexpr int kBK = 64;           // K elements per stage = one 128-byte swizzle span of bf16
 constexpr int kMaxStages = 6;
 constexpr int kMaxNT = 256;
-constexpr long long kWaitCycles = 2000000000LL;  // ~1 s: far beyond any healthy wait
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false when the limit ran out or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; return false; }
-  }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-
 // Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows 128 B apart, groups
 // of 8 rows 1024 B apart.
 __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
@@ -167,9 +131,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     abort_flag = 0;
     for (int s = 0; s < stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
     mbar_init(smem_u32(&acc_bar), 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+    mbar_fence_init();
+    tma_prefetch_map(&tmW);
+    tma_prefetch_map(&tmA);
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(tmem_cols) : "memory");
@@ -196,10 +160,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         issued = kb + 1;
       }
       if (!ok) {  // drain copies still in flight before the CTA may exit
-        for (int kb = max(0, issued - stages); kb < issued; ++kb) {
-          const long long t0 = clock64();
-          while (!mbar_try(smem_u32(&full_bar[kb % stages]), (kb / stages) & 1) && clock64() - t0 < kWaitCycles) {}
-        }
+        for (int kb = max(0, issued - stages); kb < issued; ++kb)
+          mbar_drain(smem_u32(&full_bar[kb % stages]), (kb / stages) & 1);
       }
     }
   } else if (warp == 1) {
@@ -255,51 +217,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 }
 
 // ---- host side --------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
 struct GemmState {
-  EncodeTiledFn encode = nullptr;
   // (pointer, rows, cols, box rows) -> tensor map
   std::map<std::tuple<const void*, int, int, int>, CUtensorMap> maps;
 };
 
 laser_status get_state(laser_model* m, GemmState** out) {
-  if (!m->gemm_state) {
-    GemmState* st = new GemmState();
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
-      delete st;
-      set_error("cuTensorMapEncodeTiled is not available from the driver");
-      return LASER_ERR_UNSUPPORTED;
-    }
-    st->encode = reinterpret_cast<EncodeTiledFn>(fn);
-    m->gemm_state = st;
-  }
+  if (!m->gemm_state) m->gemm_state = new GemmState();
   *out = static_cast<GemmState*>(m->gemm_state);
   return LASER_OK;
 }
 
-// bf16 row-major [rows, cols] matrix, box = box_rows x 64 elements, 128-byte swizzle.
 laser_status tensor_map(GemmState* st, const void* ptr, int rows, int cols, int box_rows, const CUtensorMap** out) {
   auto key = std::make_tuple(ptr, rows, cols, box_rows);
   auto it = st->maps.find(key);
   if (it == st->maps.end()) {
     CUtensorMap tm;
-    const cuuint64_t dims[2] = {cuuint64_t(cols), cuuint64_t(rows)};
-    const cuuint64_t strides[1] = {cuuint64_t(cols) * 2};
-    const cuuint32_t box[2] = {cuuint32_t(kBK), cuuint32_t(box_rows)};
-    const cuuint32_t estr[2] = {1, 1};
-    CUresult r = st->encode(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) {
-      set_error("cuTensorMapEncodeTiled failed (%d) for a %d x %d matrix, box %d x %d", int(r), rows, cols, box_rows, kBK);
-      return LASER_ERR_CUDA;
-    }
+    LASER_TRY(encode_bf16_2d(&tm, ptr, uint64_t(rows), uint64_t(cols), uint32_t(box_rows)));
     it = st->maps.emplace(key, tm).first;
   }
   *out = &it->second;

@@ -8,6 +8,7 @@
 #include <cmath>
 
 #include "model.cuh"
+#include "tma.cuh"
 
 namespace laser {
 namespace {
@@ -392,6 +393,8 @@ LASER_API laser_status laser_kv_create(const laser_model* m, int32_t max_seqs, i
   kv->pages_per_seq = int32_t(std::min<int64_t>(n_pages / max_seqs, 1 << 20));
   const size_t elems = std::max<size_t>(1, size_t(kv->n_layers) * kv->layer_elems());
   LASER_CUDA(cudaMalloc(reinterpret_cast<void**>(&kv->pages), elems * sizeof(__nv_bfloat16)));
+  // masked keys still enter P*V with weight 0, so the pages must never hold NaN/Inf patterns
+  LASER_CUDA(cudaMemset(kv->pages, 0, elems * sizeof(__nv_bfloat16)));
   LASER_CUDA(cudaMalloc(reinterpret_cast<void**>(&kv->page_table), size_t(max_seqs) * kv->pages_per_seq * 4));
   LASER_CUDA(cudaMalloc(reinterpret_cast<void**>(&kv->seq_len), size_t(max_seqs) * 4));
   LASER_CUDA(cudaMemset(kv->seq_len, 0, size_t(max_seqs) * 4));
@@ -399,6 +402,11 @@ LASER_API laser_status laser_kv_create(const laser_model* m, int32_t max_seqs, i
   for (int s = 0; s < max_seqs; ++s)
     for (int j = 0; j < kv->pages_per_seq; ++j) table[size_t(s) * kv->pages_per_seq + j] = j * max_seqs + s;
   LASER_CUDA(cudaMemcpy(kv->page_table, table.data(), table.size() * 4, cudaMemcpyHostToDevice));
+  const uint64_t map_rows = uint64_t(kv->n_layers) * uint64_t(n_pages) * 2 * kv->n_kv_heads * 16;
+  if (kv->head_dim % 64 == 0 && map_rows > 0 && map_rows < (uint64_t(1) << 31)) {
+    LASER_TRY(encode_bf16_2d(&kv->pages_map, kv->pages, map_rows, uint64_t(kv->head_dim), 16));
+    kv->has_pages_map = true;
+  }
   guard.p = nullptr;
   *out = kv;
   return LASER_OK;
@@ -503,8 +511,9 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
   const __nv_bfloat16* first_gain = c.n_layers > 0 ? m->attn_norm[0] : m->final_norm;
   embed_norm_kernel<<<Rp, 256, 0, stream>>>(tokens, R, d, c.vocab, m->tok_emb, first_gain, c.rms_eps, m->resid, m->xn);
   count_launch(2);
+  const bool use_tma_attn = attention_tma_supported(m, kv);
   const size_t attn_smem = (size_t(dh) + size_t(capacity) + 8) * sizeof(float);
-  if (attn_smem > 48 * 1024) {
+  if (!use_tma_attn && attn_smem > 48 * 1024) {
     LASER_REQUIRE(attn_smem <= 200 * 1024, "KV capacity of %d tokens per sequence exceeds the attention kernel's limit", capacity);
     LASER_CUDA(cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(attn_smem)));
   }
@@ -517,10 +526,17 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
     rope_kv_kernel<<<dim3(Rp, H + 2 * Hkv), 64, 0, stream>>>(m->part, p1.splits, stride, m->dqkv, H, Hkv, dh, m->rope,
                                                              m->row_pos, m->row_seq, kv->page_table, kv->pages_per_seq,
                                                              pages_l, kv->page_elems(), m->q);
-    { ProfScope ps(m, 1, stream);
-      attention_kernel<<<dim3(B, H), 128, attn_smem, stream>>>(m->q, seq_ids, m->row_ctx, m->row_n, Rs, H, Hkv, dh,
-                                                              kv->page_table, kv->pages_per_seq, pages_l,
-                                                              kv->page_elems(), m->attn); }
+    {
+      ProfScope ps(m, 1, stream);
+      if (use_tma_attn) {
+        LASER_TRY(attention_tma_launch(m, kv, l, seq_ids, B, stream));
+      } else {
+        attention_kernel<<<dim3(B, H), 128, attn_smem, stream>>>(m->q, seq_ids, m->row_ctx, m->row_n, Rs, H, Hkv, dh,
+                                                                kv->page_table, kv->pages_per_seq, pages_l,
+                                                                kv->page_elems(), m->attn);
+        count_launch();
+      }
+    }
     // output projection, residual, norm
     GemmPlan p2 = gemm_plan(Rp, d, m->dq);
     stride = size_t(Rp) * d;
@@ -536,7 +552,7 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
     { ProfScope ps(m, 0, stream); LASER_TRY(gemm_launch(m, m->act, m->wdown[l], m->part, Rp, Rp, d, f, p4.splits, stride, d, stream)); }
     const __nv_bfloat16* next_gain = l + 1 < c.n_layers ? m->attn_norm[l + 1] : m->final_norm;
     residual_norm_kernel<<<Rp, 256, 0, stream>>>(m->part, p4.splits, stride, d, d, next_gain, c.rms_eps, m->resid, m->xn);
-    count_launch(5);
+    count_launch(4);
   }
   // LM head straight into the caller's logits (one plane, rows beyond R not stored)
   { ProfScope ps(m, 0, stream); LASER_TRY(gemm_launch(m, m->xn, m->lm_head, logits, Rp, R, c.vocab, d, 1, 0, c.vocab, stream)); }

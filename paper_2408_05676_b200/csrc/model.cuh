@@ -47,4 +47,10 @@ laser_status gemm_launch(laser_model* m, const __nv_bfloat16* A, const __nv_bflo
                          cudaStream_t stream);
 void gemm_state_free(laser_model* m);
 
+// TMA-fed paged attention (head_dim 64 or 128 and a cache small enough for 32-bit row
+// coordinates); the verify forward falls back to a plain kernel otherwise.
+bool attention_tma_supported(const laser_model* m, const laser_kv* kv);
+laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const int32_t* seq_ids, int B,
+                                  cudaStream_t stream);
+
 }  // namespace laser

@@ -70,7 +70,7 @@ def _check_new_kv(L, kv, okv, cfg, seq, n_new):
 
 @pytest.mark.parametrize("name,over,B,ctx", [
     ("tiny", dict(n_layers=0, d_model=320, vocab=2000), 2, [0, 0]),     # embedding -> norm -> LM head only
-    ("tiny", dict(), 4, [37, 0, 64, 5]),
+    ("tiny", dict(), 4, [150, 0, 170, 5]),
     ("tiny", dict(n_layers=3, d_model=512, n_heads=4, n_kv_heads=4, head_dim=128, d_ffn=1376, vocab=8192), 3, [130, 16, 1]),
     ("tiny", dict(n_layers=2, d_model=256, n_heads=8, n_kv_heads=2, head_dim=32, d_ffn=256, vocab=1000, max_draft=3), 5, [9, 33, 2, 0, 17]),
 ])
