@@ -167,7 +167,7 @@ def run_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(dev))
-    cfg = synth.model_cfg("7b")
+    cfg = synth.model_cfg("7b", n_layers=args.layers)
     wl = build_workload(L, dev, cfg)
     model, kv, seq_ids, lens = wl["model"], wl["kv"], wl["seq_ids"], wl["lens"]
     t0 = time.time()
@@ -301,7 +301,8 @@ def run_ours(args):
         "metric": "generated_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": main["ms"], "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "model_shape": "llama-2-7b", "batch": B, "ctx": CTX, "draft_len": K,
+        "config": {"workload": WORKLOAD if args.layers == 32 else WORKLOAD + " [REDUCED to %d layers: profiler capture only]" % args.layers,
+                   "model_shape": "llama-2-7b", "layers": args.layers, "batch": B, "ctx": CTX, "draft_len": K,
                    "pool_tokens": int(len(wl["pool"])), "pool_groups": POOL_GROUPS, "suffix_n": [1, N_MAX],
                    "max_occ": 64, "l2": "inputs larger than L2 (13.2 GB of weights + 4.3 GB of KV per step)",
                    "parallelism": "replicas x%d" % world},
@@ -324,7 +325,8 @@ def run_ours(args):
                        for name, r in res.items()},
         "p_cal": p_cal, "pool_build_s": pool_build_s, "launches_per_step": int(main["launches"]),
     }
-    out["cpu_baseline"] = cpu_baseline(wl, sample="1 of 16 sequences, %d of 32 layers run, time extrapolated" % SAMPLE_LAYERS)
+    if args.layers >= SAMPLE_LAYERS:
+        out["cpu_baseline"] = cpu_baseline(wl, sample="1 of 16 sequences, %d of 32 layers run, time extrapolated" % SAMPLE_LAYERS)
     print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
@@ -413,6 +415,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=32,
+                    help="decoder layers of the 7B shape (fewer only for small profiler captures; the line says so)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
