@@ -222,6 +222,25 @@ laser_status laser_accept_commit(laser_kv* kv, const int32_t* seq_ids, const flo
                                  int32_t V, const laser_params* p, int32_t* n_accept,
                                  int32_t* out_tokens, int32_t* n_out, void* stream);
 
+/* Same result as laser_accept_commit, for callers that must not allocate device memory.
+ * (The paper has no counterpart; this exists for integration.)  Some hosts of this library
+ * cannot call cudaMalloc on the decoding path: a serving engine that reserved all of HBM for
+ * its own pools at start-up has nothing left for the driver to hand out, and an allocation
+ * in the middle of a step would also stall every stream of the device while the driver
+ * serves it.  laser_accept_commit keeps its per-row verdicts in a lazily grown scratch
+ * buffer; this variant keeps them in a fixed 132 KB array that is part of the library image
+ * on every GPU that loads it, and calls no allocating routine at all.
+ *   Limits: B <= 1024 sequences and B * (K+1) <= 16384 rows; larger calls return
+ *   LASER_ERR_CAPACITY and launch nothing.
+ *   The first call on each device looks up the array's device address (the device must be
+ *   current); make that first call before starting any stream capture.
+ *   All calls on a device share the one array: two calls whose kernels may overlap on the GPU
+ *   (different streams) race on it and give undefined results.  Serialise them. */
+laser_status laser_accept_commit_noalloc(laser_kv* kv, const int32_t* seq_ids, const float* logits,
+                                         const int32_t* tokens, const int32_t* n_rows, int32_t B,
+                                         int32_t V, const laser_params* p, int32_t* n_accept,
+                                         int32_t* out_tokens, int32_t* n_out, void* stream);
+
 /* ---- Generation loop (Section 2.1 / Section 3) ----------------------------------------
  * Prefills each prompt except its last token, then repeats draft -> verify -> accept ->
  * commit until every sequence has max_new tokens (the last step is truncated) or has

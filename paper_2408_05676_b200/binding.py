@@ -60,7 +60,8 @@ EXPORTS = ["laser_version", "laser_last_error", "laser_launch_count", "laser_poo
            "laser_pool_info", "laser_draft", "laser_make_rows", "laser_model_create", "laser_model_free",
            "laser_kv_create", "laser_kv_free", "laser_kv_set_page_table", "laser_kv_set_len",
            "laser_kv_get_len", "laser_kv_set_len_dev", "laser_kv_import", "laser_kv_export",
-           "laser_verify_step", "laser_check", "laser_profile_enable", "laser_profile_read", "laser_accept_commit", "laser_generate"]
+           "laser_verify_step", "laser_check", "laser_profile_enable", "laser_profile_read", "laser_accept_commit", "laser_accept_commit_noalloc",
+           "laser_generate"]
 
 lib.laser_version.restype = C.c_char_p
 lib.laser_last_error.restype = C.c_char_p
@@ -290,6 +291,20 @@ def profile_read(model: Model, cls: int):
 
 def check(model: Model, stream=None) -> None:
     _chk(lib.laser_check(model.handle, _stream(stream)))
+
+
+def accept_commit_noalloc(kv: Optional[KV], seq_ids, logits, tokens, n_rows, params: Params, out, stream=None):
+    """laser_accept_commit_noalloc: same outputs as accept_commit, no device allocation inside the
+    library.  The caller supplies every output tensor: out = (n_accept, out_tokens, n_out)."""
+    B, R, V = logits.shape
+    n_accept, out_tokens, n_out = out
+    _chk(lib.laser_accept_commit_noalloc(kv.handle if kv is not None else C.c_void_p(0),
+                                         _ptr(seq_ids) if seq_ids is not None else C.c_void_p(0),
+                                         _ptr(_dev(logits, torch.float32)), _ptr(_dev(tokens, torch.int32)),
+                                         _ptr(_dev(n_rows, torch.int32)), C.c_int32(B), C.c_int32(V),
+                                         C.byref(params), _ptr(n_accept), _ptr(out_tokens), _ptr(n_out),
+                                         _stream(stream)))
+    return out
 
 
 def accept_commit(kv: Optional[KV], seq_ids, logits, tokens, n_rows, params: Params, out=None, stream=None):

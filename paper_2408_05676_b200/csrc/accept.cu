@@ -149,8 +149,64 @@ accept_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__
     out_tokens[b * R + j] = j < a ? tokens[b * R + j + 1] : (j == a ? v[a].argmax : -1);
 }
 
+// Fixed scratch of the allocation-free entry point: per-sequence counters, then row verdicts.
+constexpr int kNoAllocMaxSeqs = 1024;
+constexpr int kNoAllocMaxRows = 16384;
+constexpr size_t kNoAllocCounterBytes = sizeof(int32_t) * kNoAllocMaxSeqs;
+constexpr size_t kNoAllocBytes = kNoAllocCounterBytes + sizeof(RowVerdict) * kNoAllocMaxRows;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+// Device address of g_noalloc_scratch on the current device, resolved once per device.
+laser_status noalloc_scratch(void** out) {
+  constexpr int kMaxDevices = 64;
+  static void* addr[kMaxDevices] = {};
+  int dev = 0;
+  LASER_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) { set_error("device index %d out of range", dev); return LASER_ERR_UNSUPPORTED; }
+  if (!addr[dev]) {
+    void* p = nullptr;
+    // the symbol's name is only a host-side handle; the kernel needs the address the runtime maps it to
+    LASER_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+    addr[dev] = p;
+  }
+  *out = addr[dev];
+  return LASER_OK;
+}
+
 }  // namespace
 }  // namespace laser
+
+LASER_API laser_status laser_accept_commit_noalloc(laser_kv* kv, const int32_t* seq_ids, const float* logits,
+                                                   const int32_t* tokens, const int32_t* n_rows, int32_t B,
+                                                   int32_t V, const laser_params* p, int32_t* n_accept,
+                                                   int32_t* out_tokens, int32_t* n_out, void* stream) {
+  using namespace laser;
+  LASER_REQUIRE(p && logits && tokens && n_rows && n_accept && out_tokens && n_out, "null argument");
+  LASER_REQUIRE(B >= 0 && V >= 1 && p->K >= 0, "B = %d, V = %d, K = %d", B, V, p->K);
+  LASER_REQUIRE(p->mode >= LASER_MODE_STRICT && p->mode <= LASER_MODE_TOPP, "mode = %d", p->mode);
+  LASER_REQUIRE(p->mode == LASER_MODE_STRICT || p->mode == LASER_MODE_TOPP || p->topk >= 1, "topk = %d", p->topk);
+  LASER_REQUIRE(kv == nullptr || seq_ids != nullptr, "seq_ids is required when committing");
+  const int64_t rows = int64_t(B) * (int64_t(p->K) + 1);
+  if (B > kNoAllocMaxSeqs || rows > kNoAllocMaxRows) {
+    set_error("laser_accept_commit_noalloc handles at most %d sequences and %d rows (B * (K+1)); got B = %d, rows = %lld",
+              kNoAllocMaxSeqs, kNoAllocMaxRows, B, (long long)rows);
+    return LASER_ERR_CAPACITY;
+  }
+  if (B == 0) return LASER_OK;
+  void* scratch = nullptr;
+  LASER_TRY(noalloc_scratch(&scratch));
+  int32_t* counters = static_cast<int32_t*>(scratch);
+  RowVerdict* verdicts = reinterpret_cast<RowVerdict*>(static_cast<char*>(scratch) + kNoAllocCounterBytes);
+  // the array keeps whatever the previous call left: the arrival counters must start at zero
+  LASER_CUDA(cudaMemsetAsync(counters, 0, sizeof(int32_t) * size_t(B), as_stream(stream)));
+  const int R = p->K + 1;
+  accept_rows_kernel<<<B * R, kAcceptThreads, 0, as_stream(stream)>>>(
+      logits, tokens, n_rows, seq_ids, R, V, p->mode, p->topk, double(p->p), counters, verdicts,
+      n_accept, out_tokens, n_out, kv ? kv->seq_len : nullptr);
+  count_launch();
+  LASER_CUDA(cudaGetLastError());
+  return LASER_OK;
+}
 
 LASER_API laser_status laser_accept_commit(laser_kv* kv, const int32_t* seq_ids,
                                            const float* logits, const int32_t* tokens,

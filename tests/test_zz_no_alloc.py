@@ -1,0 +1,71 @@
+"""laser_accept_commit_noalloc against laser_accept_commit.
+
+Some programs embedding this library cannot allocate device memory while decoding: an engine
+that took all of HBM for its own pools at start-up leaves nothing for cudaMalloc, and an
+allocation inside a step would stall the whole device.  For them the library offers an
+acceptance call whose scratch is a fixed array inside the library image.  This test drives that
+call through the C ABI twice in a row (the array keeps the first call's contents, so the second
+call proves the counters are cleared) and requires the very same outputs as the ordinary call -
+acceptance is integer work, so the tolerance is exact equality.  It also checks that a call
+beyond the fixed capacity is refused instead of overrunning the array.  The file sorts last so
+that a stop-at-first-failure run has already covered every other test.
+"""
+import numpy as np
+import pytest
+import torch
+
+from helpers import dev_i32, ensure_built
+from paper_2408_05676_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def L():
+    ensure_built()
+    from paper_2408_05676_b200 import binding
+    return binding
+
+
+def _outs(B, R):
+    return (torch.full((B,), -7, dtype=torch.int32, device="cuda"),
+            torch.full((B, R), -7, dtype=torch.int32, device="cuda"),
+            torch.full((B,), -7, dtype=torch.int32, device="cuda"))
+
+
+def test_two_calls_in_a_row_match_the_allocating_entry_point(L):
+    for (B, K, V, seed, mode) in [(16, 8, 4096, 21, L.MODE_RELAXED), (5, 3, 1001, 22, L.MODE_STRICT)]:
+        logits, tokens, n_rows = synth.make_accept_case(B, K, V, seed)
+        n_rows[1] = 0
+        dl, dt, dn = torch.as_tensor(logits, device="cuda"), dev_i32(tokens), dev_i32(n_rows)
+        prm = L.make_params(K=K, mode=mode, topk=2, p=0.1)
+        want = [t.cpu().numpy() for t in L.accept_commit(None, None, dl, dt, dn, prm)]
+        for call in range(2):
+            got = L.accept_commit_noalloc(None, None, dl, dt, dn, prm, _outs(B, K + 1))
+            torch.cuda.synchronize()
+            for g, w in zip(got, want):
+                assert (g.cpu().numpy() == w).all(), (B, K, V, call)
+        # a different shape right after reuses the same array
+        logits2, tokens2, n_rows2 = synth.make_accept_case(B + 3, K, V, seed + 100)
+        dl2, dt2, dn2 = torch.as_tensor(logits2, device="cuda"), dev_i32(tokens2), dev_i32(n_rows2)
+        want2 = [t.cpu().numpy() for t in L.accept_commit(None, None, dl2, dt2, dn2, prm)]
+        got2 = L.accept_commit_noalloc(None, None, dl2, dt2, dn2, prm, _outs(B + 3, K + 1))
+        for g, w in zip(got2, want2):
+            assert (g.cpu().numpy() == w).all()
+
+
+def test_sizes_beyond_the_fixed_array_are_refused(L):
+    B, K, V = 1025, 0, 8
+    logits = torch.zeros(B, K + 1, V, device="cuda")
+    tokens = torch.zeros(B, K + 1, dtype=torch.int32, device="cuda")
+    n_rows = torch.ones(B, dtype=torch.int32, device="cuda")
+    outs = _outs(B, K + 1)
+    with pytest.raises(L.LaserError) as e:
+        L.accept_commit_noalloc(None, None, logits, tokens, n_rows, L.make_params(K=K), outs)
+    assert e.value.status == -4 and "at most" in str(e.value)
+    assert int(outs[0][0]) == -7                      # nothing was launched
+    B, K = 600, 31                                     # 19200 rows > 16384
+    with pytest.raises(L.LaserError):
+        L.accept_commit_noalloc(None, None, torch.zeros(B, K + 1, V, device="cuda"),
+                                torch.zeros(B, K + 1, dtype=torch.int32, device="cuda"),
+                                torch.ones(B, dtype=torch.int32, device="cuda"), L.make_params(K=K), _outs(B, K + 1))
