@@ -1,19 +1,23 @@
-// Dense contractions of the verify forward (QKV, O, gate/up, down, LM head):
-// out[r][n] = sum_k A[r][k] * W[n][k], bf16 operands, fp32 accumulation.
+// Dense contractions of the verify forward (QKV, O, gate/up, down, LM head) with their
+// element-wise neighbours fused in: acc[r][n] = sum_k A[r][k] * W[n][k], bf16 operands, fp32
+// accumulation, followed by RMSNorm scaling / rotary embedding + cache write / residual add /
+// SwiGLU in the epilogue.
 //
-// The token rows are few (batch x (K+1)) and the weight matrices are large, so the weight
-// rows take the 128-wide M side of the MMA and the token rows the N side: a 128 x NT
-// accumulator in tensor memory, NT <= 256 token rows, no padding of the rows to 128.
-// Split-K partial sums go to separate planes that the consumer kernel adds in a fixed
-// order, which keeps the result independent of scheduling.
+// Shape of the problem: few token rows (batch x (K+1), e.g. 144) against large weight
+// matrices, so the step is bound by streaming the weights from HBM.  The weight rows take the
+// 128-wide M side of tcgen05.mma and the token rows the N side (NT <= 192, no padding of the
+// rows to 128); the accumulator is a 128 x NT fp32 tile in tensor memory.
 //
-// Tensor-memory kernel (tcgen05): one CTA per (token tile, weight tile, K range), two CTAs
-// resident per SM.  Warp 0 streams 128x64 weight tiles and NTx64 activation tiles with TMA
-// (128-byte swizzle) through a ring of shared-memory stages; warp 1 issues tcgen05.mma
-// (M=128, N=NT, K=16) from shared-memory descriptors into a TMEM accumulator and releases
-// stages with tcgen05.commit; warps 2-5 read the accumulator with tcgen05.ld and store it
-// transposed (token-major).  Every wait is bounded: on expiry the CTA records
-// LASER_ERR_TIMEOUT, drains its copies, frees its TMEM and exits.
+// One CTA per (token tile, weight tile, K range); the CTAs that share an output tile form a
+// thread-block cluster along K.  Warp 0 streams weight and activation tiles with TMA
+// (128-byte swizzle) through a ring of shared-memory stages, warp 1 issues the MMAs and frees
+// stages with tcgen05.commit, warps 2-5 move the finished accumulator from tensor memory to
+// shared memory.  The partial tiles of a cluster are then summed through distributed shared
+// memory in a fixed order (run-to-run identical results, no partial sums in global memory);
+// each CTA reduces and finishes its own slice of the token columns with the fused epilogue.
+// Two CTAs fit on an SM, so one CTA's epilogue overlaps another's main loop.
+// Every mbarrier wait is bounded: on expiry the CTA records LASER_ERR_TIMEOUT, drains its
+// copies, still joins the cluster barriers, frees its tensor memory and exits.
 #include <map>
 #include <tuple>
 
@@ -23,84 +27,24 @@
 namespace laser {
 namespace {
 
-// ---------------------------------------------------------------------------------------
-// Warp-level MMA kernel (mma.sync m16n8k16).  Serves shapes the tensor-memory kernel does
-// not cover.  Each warp owns 8 weight rows and walks all token rows in groups of MT tiles
-// of 16; operands are read straight from global memory / L1 in fragment layout.
-// ---------------------------------------------------------------------------------------
-constexpr int kMmaWarps = 4;
-
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
-                                               uint32_t a3, uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-template <int MT>
-__global__ void __launch_bounds__(kMmaWarps * 32)
-gemm_mma_kernel(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ W,
-                float* __restrict__ out, int R_pad, int R_store, int N, int K, int k_per_split,
-                size_t split_stride, int ldo) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = (blockIdx.x * kMmaWarps + warp) * 8;
-  if (n0 >= N) return;
-  const int g = lane >> 2, t2 = (lane & 3) * 2;
-  const int kb = blockIdx.y * k_per_split, ke = min(K, kb + k_per_split);
-  const __nv_bfloat16* wrow = W + size_t(n0 + g) * K + t2;
-  float* o = out + size_t(blockIdx.y) * split_stride;
-  for (int m0 = 0; m0 < R_pad; m0 += MT * 16) {
-    float acc[MT][4];
-#pragma unroll
-    for (int t = 0; t < MT; ++t) acc[t][0] = acc[t][1] = acc[t][2] = acc[t][3] = 0.f;
-    for (int k = kb; k < ke; k += 16) {
-      const uint32_t b0 = *reinterpret_cast<const uint32_t*>(wrow + k);
-      const uint32_t b1 = *reinterpret_cast<const uint32_t*>(wrow + k + 8);
-#pragma unroll
-      for (int t = 0; t < MT; ++t) {
-        const int r = m0 + t * 16 + g;
-        if (m0 + t * 16 < R_pad) {
-          const __nv_bfloat16* a = A + size_t(r) * K + k + t2;
-          const uint32_t a0 = *reinterpret_cast<const uint32_t*>(a);
-          const uint32_t a1 = *reinterpret_cast<const uint32_t*>(a + size_t(8) * K);
-          const uint32_t a2 = *reinterpret_cast<const uint32_t*>(a + 8);
-          const uint32_t a3 = *reinterpret_cast<const uint32_t*>(a + size_t(8) * K + 8);
-          mma_bf16_16816(acc[t], a0, a1, a2, a3, b0, b1);
-        }
-      }
-    }
-#pragma unroll
-    for (int t = 0; t < MT; ++t) {
-      const int r = m0 + t * 16 + g;
-      if (m0 + t * 16 < R_pad) {
-        if (r < R_store) *reinterpret_cast<float2*>(o + size_t(r) * ldo + n0 + t2) = make_float2(acc[t][0], acc[t][1]);
-        if (r + 8 < R_store) *reinterpret_cast<float2*>(o + size_t(r + 8) * ldo + n0 + t2) = make_float2(acc[t][2], acc[t][3]);
-      }
-    }
-  }
-}
-
-// ---------------------------------------------------------------------------------------
-// Tensor-memory kernel
-// ---------------------------------------------------------------------------------------
+using bf16 = __nv_bfloat16;
 constexpr int kTcThreads = 192;
 constexpr int kBM = 128;          // weight rows per tile (MMA M)
 constexpr int kBK = 64;           // K elements per stage = one 128-byte swizzle span of bf16
 constexpr int kMaxStages = 6;
-constexpr int kMaxNT = 256;
+constexpr int kMaxNT = 192;       // token rows per tile: accumulator staging must fit shared memory
+constexpr int kSmemBudget = 110 * 1024;
+
 // Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows 128 B apart, groups
 // of 8 rows 1024 B apart.
 __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
   uint64_t d = 0;
   d |= uint64_t((smem_addr & 0x3FFFF) >> 4);        // start address
-  d |= uint64_t(0) << 16;                           // leading byte offset: unused for swizzled K-major
   d |= uint64_t(1024 >> 4) << 32;                   // stride byte offset between 8-row groups
   d |= uint64_t(1) << 46;                           // descriptor version of this architecture
   d |= uint64_t(2) << 61;                           // 128-byte swizzle
   return d;
 }
-
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
@@ -110,22 +54,126 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t local_addr, uint32_t rank) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  return make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+}
 
+// ---- fused epilogues: one warp finishes one token row r of a 128-feature tile; lane l holds
+//      features n0 + 4l .. 4l+3 in v ----------------------------------------------------------
+__device__ __forceinline__ void epi_plain(const GemmEpilogue& e, int r, int n0, int lane, float4 v, float rstd, int N) {
+  if (r >= e.R_store) return;
+  const int n = n0 + 4 * lane;
+  float* o = e.out + size_t(r) * e.ldo + n;
+  v.x *= rstd; v.y *= rstd; v.z *= rstd; v.w *= rstd;
+  if (n + 3 < N && (e.ldo & 3) == 0) {
+    *reinterpret_cast<float4*>(o) = v;
+  } else {
+    if (n < N) o[0] = v.x;
+    if (n + 1 < N) o[1] = v.y;
+    if (n + 2 < N) o[2] = v.z;
+    if (n + 3 < N) o[3] = v.w;
+  }
+}
+
+// resid += acc; xb = bf16(resid * gain of the next norm); per-tile sum of squares for that norm
+__device__ __forceinline__ void epi_resid(const GemmEpilogue& e, int r, int n0, int lane, float4 v, int N, int tile) {
+  const int n = n0 + 4 * lane;
+  float ss = 0.f;
+  if (n < N) {  // N is a multiple of 8 (checked on the host), so the four features are all valid
+    float4 x = *reinterpret_cast<float4*>(e.resid + size_t(r) * N + n);
+    x.x += v.x; x.y += v.y; x.z += v.z; x.w += v.w;
+    *reinterpret_cast<float4*>(e.resid + size_t(r) * N + n) = x;
+    const uint2 g2 = *reinterpret_cast<const uint2*>(e.gain_next + n);
+    const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&g2.x), g23 = *reinterpret_cast<const __nv_bfloat162*>(&g2.y);
+    *reinterpret_cast<uint2*>(e.xb + size_t(r) * N + n) =
+        pack4_bf16(x.x * __low2float(g01), x.y * __high2float(g01), x.z * __low2float(g23), x.w * __high2float(g23));
+    ss = x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+  }
+  for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if (lane == 0) e.sumsq_out[size_t(tile) * e.sumsq_ld + r] = ss;
+}
+
+// tile rows 0..63 = gate features f0.., rows 64..127 = up features f0..; act = silu(g) * u
+__device__ __forceinline__ void epi_swiglu(const GemmEpilogue& e, int r, int f0, int lane, float4 v, float rstd) {
+  float4 u;
+  u.x = __shfl_xor_sync(0xffffffffu, v.x, 16); u.y = __shfl_xor_sync(0xffffffffu, v.y, 16);
+  u.z = __shfl_xor_sync(0xffffffffu, v.z, 16); u.w = __shfl_xor_sync(0xffffffffu, v.w, 16);
+  const int fidx = f0 + 4 * lane;
+  if (lane < 16 && fidx < e.f) {  // f is a multiple of 8 (checked on the host)
+    auto act = [rstd](float g, float up) { g *= rstd; up *= rstd; return g / (1.f + __expf(-g)) * up; };
+    *reinterpret_cast<uint2*>(e.act + size_t(r) * e.f + fidx) =
+        pack4_bf16(act(v.x, u.x), act(v.y, u.y), act(v.z, u.z), act(v.w, u.w));
+  }
+}
+
+// rotary embedding of Q and K (pair i, i + dh/2), bf16 rounding, Q store, K/V page write
+__device__ __forceinline__ void epi_qkv(const GemmEpilogue& e, int r, int n0, int lane, float4 v, float rstd, int N) {
+  v.x *= rstd; v.y *= rstd; v.z *= rstd; v.w *= rstd;
+  const int dh = e.dh, half = dh >> 1, dq = e.H * dh, dkv = e.Hkv * dh;
+  const int shift = dh >> 3;  // lanes between a feature and its rotation partner
+  float4 pv;
+  pv.x = __shfl_xor_sync(0xffffffffu, v.x, shift); pv.y = __shfl_xor_sync(0xffffffffu, v.y, shift);
+  pv.z = __shfl_xor_sync(0xffffffffu, v.z, shift); pv.w = __shfl_xor_sync(0xffffffffu, v.w, shift);
+  const int n = n0 + 4 * lane;
+  if (n >= N) return;
+  const int pos = e.row_pos[r];
+  const int idx = n % dh;          // four consecutive features stay inside one half of one head
+  float4 y = v;
+  if (n < dq + dkv) {
+    const int j = idx % half;
+    const float4 cs01 = *reinterpret_cast<const float4*>(e.rope + (size_t(r) * half + j) * 2);      // c0 s0 c1 s1
+    const float4 cs23 = *reinterpret_cast<const float4*>(e.rope + (size_t(r) * half + j + 2) * 2);  // c2 s2 c3 s3
+    const float sg = idx < half ? -1.f : 1.f;
+    y.x = v.x * cs01.x + sg * pv.x * cs01.y;
+    y.y = v.y * cs01.z + sg * pv.y * cs01.w;
+    y.z = v.z * cs23.x + sg * pv.z * cs23.y;
+    y.w = v.w * cs23.z + sg * pv.w * cs23.w;
+  }
+  if (n < dq) {
+    if (pos < 0) y = make_float4(0.f, 0.f, 0.f, 0.f);
+    *reinterpret_cast<uint2*>(e.q + size_t(r) * dq + n) = pack4_bf16(y.x, y.y, y.z, y.w);
+  } else if (pos >= 0) {
+    const int is_v = n >= dq + dkv;
+    const int h = (n - dq - is_v * dkv) / dh;
+    const int page = e.page_table[size_t(e.row_seq[r]) * e.pages_per_seq + (pos >> 4)];
+    bf16* dst = e.pages_layer + size_t(page) * e.page_elems + (size_t(is_v) * e.Hkv + h) * 16 * dh + size_t(pos & 15) * dh + idx;
+    *reinterpret_cast<uint2*>(dst) = pack4_bf16(y.x, y.y, y.z, y.w);
+  }
+}
+
+template <int EPI>
 __global__ void __launch_bounds__(kTcThreads)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA,
-               float* __restrict__ out, int N, int R_store, int NT, int total_kb, int kb_per_split, int stages,
-               size_t split_stride, int ldo, int tmem_cols, int32_t* __restrict__ status) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, const GemmEpilogue e,
+               int N, int NT, int total_kb, int kb_per_split, int splits, int stages, int tmem_cols,
+               int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_bar;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
+  __shared__ float s_rstd[kMaxNT];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
+  float* stage_acc = reinterpret_cast<float*>(smem_raw + (tiles - raw));  // [NT][128] after the main loop
   const uint32_t w_bytes = kBM * 128, a_bytes = uint32_t(NT) * 128, stage_bytes = w_bytes + a_bytes;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int r0 = blockIdx.x * NT, n0 = blockIdx.y * kBM;
-  const int kb0 = blockIdx.z * kb_per_split;
-  const int nkb = min(kb_per_split, total_kb - kb0);
+  const int krank = blockIdx.x % splits, ttile = blockIdx.x / splits, wtile = blockIdx.y;
+  const int r0 = ttile * NT, n0 = wtile * kBM;
+  const int kb0 = krank * kb_per_split;
+  const int nkb = max(0, min(kb_per_split, total_kb - kb0));
+  // rows of the weight matrix behind the two 64-row halves of the tile
+  const int wrow0 = EPI == EPI_SWIGLU ? wtile * 64 : n0;
+  const int wrow1 = EPI == EPI_SWIGLU ? e.f + wtile * 64 : n0 + 64;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -155,14 +203,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const uint32_t bar = smem_u32(&full_bar[s]);
         const uint32_t dst = tiles + uint32_t(s) * stage_bytes;
         mbar_expect_tx(bar, stage_bytes);
-        tma_load_2d(dst, &tmW, (kb0 + kb) * kBK, n0, bar);
-        tma_load_2d(dst + w_bytes, &tmA, (kb0 + kb) * kBK, r0, bar);
+        const int k = (kb0 + kb) * kBK;
+        tma_load_2d(dst, &tmW, k, wrow0, bar);
+        tma_load_2d(dst + w_bytes / 2, &tmW, k, wrow1, bar);
+        tma_load_2d(dst + w_bytes, &tmA, k, r0, bar);
         issued = kb + 1;
       }
-      if (!ok) {  // drain copies still in flight before the CTA may exit
-        for (int kb = max(0, issued - stages); kb < issued; ++kb)
-          mbar_drain(smem_u32(&full_bar[kb % stages]), (kb / stages) & 1);
-      }
+      if (!ok)  // drain copies still in flight before the CTA may exit
+        for (int kb = max(0, issued - stages); kb < issued; ++kb) mbar_drain(smem_u32(&full_bar[kb % stages]), (kb / stages) & 1);
     }
   } else if (warp == 1) {
     if (lane == 0) {  // MMA issuer
@@ -182,15 +230,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       }
       umma_commit(smem_u32(&acc_bar));  // arrives when every MMA issued so far has finished
     }
-  } else {  // epilogue warps: TMEM lane quarter = warp id modulo 4
-    const int quarter = warp & 3;
+  } else {
+    // RMSNorm scale of each token row of this tile, from the producer's per-tile sums of squares
+    for (int j = threadIdx.x - 64; j < NT; j += 128) {
+      float rstd = 1.f;
+      if (e.sumsq_in && r0 + j < e.R_rows) {
+        float ss = 0.f;
+        for (int t = 0; t < e.sumsq_in_tiles; ++t) ss += e.sumsq_in[size_t(t) * e.sumsq_ld + r0 + j];
+        rstd = rsqrtf(ss * e.inv_d + e.eps);
+      }
+      s_rstd[j] = rstd;
+    }
+    // accumulator: tensor memory -> shared memory, token-major [NT][128]
+    const int quarter = warp & 3;  // a warp may only touch its own 32 TMEM lanes
     const bool ok = mbar_wait(smem_u32(&acc_bar), 0, &abort_flag);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (ok && nkb > 0) {
-      const int n = n0 + quarter * 32 + lane;
-      float* o = out + size_t(blockIdx.z) * split_stride + n;
-      for (int c = 0; c < NT; c += 16) {
-        uint32_t v[16];
+    for (int c = 0; c < NT; c += 16) {
+      uint32_t v[16];
+      if (ok && nkb > 0) {
         const uint32_t taddr = tmem_acc + (uint32_t(quarter * 32) << 16) + uint32_t(c);
         asm volatile(
             "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
@@ -198,17 +255,44 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
               "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
             : "r"(taddr) : "memory");
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (n < N) {
+      } else {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int r = r0 + c + i;
-            if (r < R_store) o[size_t(r) * ldo] = __uint_as_float(v[i]);
-          }
-        }
+        for (int i = 0; i < 16; ++i) v[i] = 0u;
       }
+#pragma unroll
+      for (int i = 0; i < 16; ++i) stage_acc[(c + i) * kBM + quarter * 32 + lane] = __uint_as_float(v[i]);
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (splits > 1) cluster_sync_all();  // every partial tile of the cluster is staged
+
+  // each CTA sums and finishes its slice of the token columns; ranks are added in order 0..splits-1
+  {
+    const int slice = (NT + splits - 1) / splits;
+    const int j_lo = krank * slice, j_hi = min(NT, j_lo + slice);
+    const uint32_t stage_addr = tiles;
+    for (int j = j_lo + warp; j < j_hi; j += kTcThreads / 32) {
+      float4 v;
+      if (splits > 1) {
+        v = ld_cluster_f4(stage_addr + uint32_t(j * kBM + 4 * lane) * 4, 0);
+        for (int rk = 1; rk < splits; ++rk) {
+          const float4 w = ld_cluster_f4(stage_addr + uint32_t(j * kBM + 4 * lane) * 4, uint32_t(rk));
+          v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+        }
+      } else {
+        v = *reinterpret_cast<const float4*>(stage_acc + j * kBM + 4 * lane);
+      }
+      const int r = r0 + j;
+      if (r >= e.R_rows) continue;   // the last token tile may overhang the buffers
+      const float rstd = s_rstd[j];
+      if (EPI == EPI_PLAIN) epi_plain(e, r, n0, lane, v, rstd, N);
+      else if (EPI == EPI_RESID) epi_resid(e, r, n0, lane, v, N, wtile);
+      else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, wtile * 64, lane, v, rstd);
+      else epi_qkv(e, r, n0, lane, v, rstd, N);
+    }
+  }
+  if (splits > 1) cluster_sync_all();  // peers may still be reading this CTA's staged tile
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(tmem_cols) : "memory");
@@ -220,12 +304,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 struct GemmState {
   // (pointer, rows, cols, box rows) -> tensor map
   std::map<std::tuple<const void*, int, int, int>, CUtensorMap> maps;
+  bool attrs_set = false;
 };
 
-laser_status get_state(laser_model* m, GemmState** out) {
+GemmState* get_state(laser_model* m) {
   if (!m->gemm_state) m->gemm_state = new GemmState();
-  *out = static_cast<GemmState*>(m->gemm_state);
-  return LASER_OK;
+  return static_cast<GemmState*>(m->gemm_state);
 }
 
 laser_status tensor_map(GemmState* st, const void* ptr, int rows, int cols, int box_rows, const CUtensorMap** out) {
@@ -247,69 +331,80 @@ TcShape tc_shape(int R_pad) {
   s.n_tiles = ceil_div(R_pad, kMaxNT);
   s.NT = ceil_div(ceil_div(R_pad, s.n_tiles), 16) * 16;
   const int stage_bytes = kBM * 128 + s.NT * 128;
-  s.stages = std::max(2, std::min(kMaxStages, (110 * 1024) / stage_bytes));
+  s.stages = std::max(2, std::min(kMaxStages, kSmemBudget / stage_bytes));
   s.tmem_cols = 32;
   while (s.tmem_cols < s.NT) s.tmem_cols <<= 1;
-  s.smem = size_t(s.stages) * stage_bytes + 1024;
+  s.smem = std::max(size_t(s.stages) * stage_bytes, size_t(s.NT) * kBM * 4) + 1024;
   return s;
 }
 
-bool tc_ok(int N, int K) { return K % 8 == 0 && N >= 1 && K >= 8; }
+template <int EPI>
+laser_status launch_epi(const CUtensorMap& tw, const CUtensorMap& ta, const GemmEpilogue& e, int N, const TcShape& sh,
+                        int w_tiles, int total_kb, int kbps, int splits, int32_t* status, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(sh.n_tiles * splits), unsigned(w_tiles), 1);
+  cfg.blockDim = dim3(kTcThreads, 1, 1);
+  cfg.dynamicSmemBytes = sh.smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = unsigned(splits);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  LASER_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI>, tw, ta, e, N, sh.NT, total_kb, kbps, splits, sh.stages,
+                                sh.tmem_cols, status));
+  return LASER_OK;
+}
 
 }  // namespace
 
-GemmPlan gemm_plan(int R_pad, int N, int K) {
-  if (!tc_ok(N, K)) {
-    const int blocks = ceil_div(N, 8 * kMmaWarps);
-    int splits = std::max(1, std::min(8, ceil_div(296, blocks)));
-    while (splits > 1 && ceil_div(ceil_div(K, splits), 16) * 16 * (splits - 1) >= K) --splits;
-    return GemmPlan{splits};
-  }
-  // Pick the split count with the least modelled time: CTAs are spread over 148 SMs, each
-  // costs its K blocks plus a fixed prologue/epilogue share, each extra plane costs a little.
+int gemm_splits(int R_pad, int N, int K, int epi) {
+  // Modelled time: CTAs are spread over 148 SMs (two resident per SM); each costs its K blocks
+  // plus a fixed prologue/epilogue share; the cluster reduction grows with the split count.
   const TcShape sh = tc_shape(R_pad);
-  const int tiles = ceil_div(N, kBM) * sh.n_tiles, total_kb = ceil_div(K, kBK);
+  const int w_tiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
+  const int tiles = w_tiles * sh.n_tiles, total_kb = ceil_div(K, kBK);
   int best = 1;
   double best_cost = 1e30;
-  for (int s = 1; s <= std::min(total_kb, 16); ++s) {
+  for (int s = 1; s <= std::min(total_kb, 8); ++s) {
     const int kbps = ceil_div(total_kb, s);
-    if (kbps * (s - 1) >= total_kb) continue;  // a split would be empty
-    const double cost = double(ceil_div(tiles * s, 148)) * (kbps + 3.0) + 0.4 * s;
+    if (kbps * (s - 1) >= total_kb) continue;  // a rank would have no K blocks
+    const double cost = double(ceil_div(tiles * s, 148)) * (kbps + 4.0) + 0.5 * s;
     if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
   }
-  return GemmPlan{best};
+  return best;
 }
 
-laser_status gemm_launch(laser_model* m, const __nv_bfloat16* A, const __nv_bfloat16* W, float* out,
-                         int R_pad, int R_store, int N, int K, int splits, size_t split_stride, int ldo,
-                         cudaStream_t stream) {
-  if (R_pad % 16 != 0) { set_error("GEMM rows %d not a multiple of 16", R_pad); return LASER_ERR_UNSUPPORTED; }
-  if (tc_ok(N, K) && (reinterpret_cast<uintptr_t>(A) & 15) == 0 && (reinterpret_cast<uintptr_t>(W) & 15) == 0) {
-    GemmState* st = nullptr;
-    LASER_TRY(get_state(m, &st));
-    const TcShape sh = tc_shape(R_pad);
-    const CUtensorMap *tw = nullptr, *ta = nullptr;
-    LASER_TRY(tensor_map(st, W, N, K, kBM, &tw));
-    LASER_TRY(tensor_map(st, A, m->R_pad, K, sh.NT, &ta));
-    const int total_kb = ceil_div(K, kBK), kbps = ceil_div(total_kb, splits);
-    LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024));
-    dim3 grid(sh.n_tiles, ceil_div(N, kBM), splits);
-    gemm_tc_kernel<<<grid, kTcThreads, sh.smem, stream>>>(*tw, *ta, out, N, R_store, sh.NT, total_kb, kbps, sh.stages,
-                                                           split_stride, ldo, sh.tmem_cols, m->status);
-    count_launch();
-    LASER_CUDA(cudaGetLastError());
-    return LASER_OK;
-  }
-  if (N % 8 != 0 || K % 16 != 0) {
-    set_error("GEMM shape N=%d K=%d unsupported (need K%%8==0 and 16-byte aligned operands, or N%%8==0 and K%%16==0)", N, K);
+laser_status gemm_fused(laser_model* m, const __nv_bfloat16* A, const __nv_bfloat16* W, int R_pad, int N, int K, int epi,
+                        const GemmEpilogue& e, cudaStream_t stream) {
+  if (R_pad % 16 != 0 || K % 8 != 0 || N % 8 != 0 || (reinterpret_cast<uintptr_t>(A) & 15) || (reinterpret_cast<uintptr_t>(W) & 15)) {
+    set_error("GEMM shape N=%d K=%d rows=%d unsupported (N, K multiples of 8, rows of 16, 16-byte aligned operands)", N, K, R_pad);
     return LASER_ERR_UNSUPPORTED;
   }
-  const int k_per_split = ceil_div(ceil_div(K, splits), 16) * 16;
-  dim3 grid(ceil_div(N, 8 * kMmaWarps), splits);
-  gemm_mma_kernel<9><<<grid, kMmaWarps * 32, 0, stream>>>(A, W, out, R_pad, R_store, N, K, k_per_split,
-                                                           split_stride, ldo);
+  GemmState* st = get_state(m);
+  if (!st->attrs_set) {
+    LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048));
+    LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048));
+    LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048));
+    LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048));
+    st->attrs_set = true;
+  }
+  const TcShape sh = tc_shape(R_pad);
+  const CUtensorMap *tw = nullptr, *ta = nullptr;
+  LASER_TRY(tensor_map(st, W, N, K, 64, &tw));
+  LASER_TRY(tensor_map(st, A, m->R_pad, K, sh.NT, &ta));
+  const int splits = gemm_splits(R_pad, N, K, epi);
+  const int total_kb = ceil_div(K, kBK), kbps = ceil_div(total_kb, splits);
+  const int w_tiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
+  switch (epi) {
+    case EPI_PLAIN: LASER_TRY(launch_epi<EPI_PLAIN>(*tw, *ta, e, N, sh, w_tiles, total_kb, kbps, splits, m->status, stream)); break;
+    case EPI_RESID: LASER_TRY(launch_epi<EPI_RESID>(*tw, *ta, e, N, sh, w_tiles, total_kb, kbps, splits, m->status, stream)); break;
+    case EPI_SWIGLU: LASER_TRY(launch_epi<EPI_SWIGLU>(*tw, *ta, e, N, sh, w_tiles, total_kb, kbps, splits, m->status, stream)); break;
+    default: LASER_TRY(launch_epi<EPI_QKV>(*tw, *ta, e, N, sh, w_tiles, total_kb, kbps, splits, m->status, stream)); break;
+  }
   count_launch();
-  LASER_CUDA(cudaGetLastError());
   return LASER_OK;
 }
 

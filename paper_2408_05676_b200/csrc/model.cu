@@ -64,10 +64,12 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return t;
 }
 
-// Embedding gather, then RMSNorm with the first layer's gain.
+// Embedding gather: resid = emb[token]; xb = bf16(resid * gain of the first norm); the sum of
+// squares of the row goes to tile plane 0 (the consumer GEMM turns it into the RMSNorm scale).
 __global__ void __launch_bounds__(256)
-embed_norm_kernel(const int32_t* __restrict__ tokens, int R, int d, int vocab, const bf16* __restrict__ emb,
-                  const bf16* __restrict__ gain, float eps, float* __restrict__ resid, bf16* __restrict__ xn) {
+embed_kernel(const int32_t* __restrict__ tokens, int R, int d, int vocab, const bf16* __restrict__ emb,
+             const bf16* __restrict__ gain, float* __restrict__ resid, bf16* __restrict__ xb,
+             float* __restrict__ sumsq) {
   __shared__ float red[8];
   const int r = blockIdx.x;
   const int tok = r < R ? tokens[r] : -1;
@@ -76,79 +78,11 @@ embed_norm_kernel(const int32_t* __restrict__ tokens, int R, int d, int vocab, c
   for (int j = threadIdx.x; j < d; j += blockDim.x) {
     const float x = ok ? __bfloat162float(emb[size_t(tok) * d + j]) : 0.f;
     resid[size_t(r) * d + j] = x;
+    xb[size_t(r) * d + j] = __float2bfloat16(x * __bfloat162float(gain[j]));
     ss += x * x;
   }
   ss = block_sum(ss, red);
-  const float scale = rsqrtf(ss / float(d) + eps);
-  for (int j = threadIdx.x; j < d; j += blockDim.x)
-    xn[size_t(r) * d + j] = __float2bfloat16(resid[size_t(r) * d + j] * scale * __bfloat162float(gain[j]));
-}
-
-// resid += sum of split-K planes; xn = RMSNorm(resid) * gain.
-__global__ void __launch_bounds__(256)
-residual_norm_kernel(const float* __restrict__ part, int splits, size_t split_stride, int ld, int d,
-                     const bf16* __restrict__ gain, float eps, float* __restrict__ resid, bf16* __restrict__ xn) {
-  __shared__ float red[8];
-  const int r = blockIdx.x;
-  float ss = 0.f;
-  for (int j = threadIdx.x; j < d; j += blockDim.x) {
-    float x = resid[size_t(r) * d + j];
-    for (int s = 0; s < splits; ++s) x += part[s * split_stride + size_t(r) * ld + j];
-    resid[size_t(r) * d + j] = x;
-    ss += x * x;
-  }
-  ss = block_sum(ss, red);
-  const float scale = rsqrtf(ss / float(d) + eps);
-  for (int j = threadIdx.x; j < d; j += blockDim.x)
-    xn[size_t(r) * d + j] = __float2bfloat16(resid[size_t(r) * d + j] * scale * __bfloat162float(gain[j]));
-}
-
-// act = silu(gate) * up from the split-K planes of the fused gate/up GEMM.
-__global__ void swiglu_kernel(const float* __restrict__ part, int splits, size_t split_stride, int f,
-                              bf16* __restrict__ act) {
-  const int r = blockIdx.y;
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= f) return;
-  float g = 0.f, u = 0.f;
-  for (int s = 0; s < splits; ++s) {
-    g += part[s * split_stride + size_t(r) * 2 * f + j];
-    u += part[s * split_stride + size_t(r) * 2 * f + f + j];
-  }
-  act[size_t(r) * f + j] = __float2bfloat16(g / (1.f + __expf(-g)) * u);
-}
-
-// Rotary embedding of Q and K, bf16 rounding, K/V page write.  grid (row, head slot) where
-// head slots are [0, H) for Q, [H, H+Hkv) for K, [H+Hkv, H+2Hkv) for V.
-__global__ void rope_kv_kernel(const float* __restrict__ part, int splits, size_t split_stride, int dqkv,
-                               int H, int Hkv, int dh, const float* __restrict__ rope,
-                               const int32_t* __restrict__ row_pos, const int32_t* __restrict__ row_seq,
-                               const int32_t* __restrict__ page_table, int pages_per_seq,
-                               bf16* __restrict__ pages_layer, size_t page_elems, bf16* __restrict__ q) {
-  const int r = blockIdx.x, slot = blockIdx.y, half = dh / 2;
-  const int pos = row_pos[r];
-  const float* src = part + size_t(r) * dqkv + size_t(slot) * dh;
-  for (int j = threadIdx.x; j < half; j += blockDim.x) {
-    float x1 = 0.f, x2 = 0.f;
-    for (int s = 0; s < splits; ++s) { x1 += src[s * split_stride + j]; x2 += src[s * split_stride + j + half]; }
-    float y1 = x1, y2 = x2;
-    if (slot < H + Hkv) {
-      const float c = rope[(size_t(r) * half + j) * 2], sn = rope[(size_t(r) * half + j) * 2 + 1];
-      y1 = x1 * c - x2 * sn;
-      y2 = x2 * c + x1 * sn;
-    }
-    if (slot < H) {
-      bf16* dst = q + size_t(r) * H * dh + size_t(slot) * dh;
-      dst[j] = __float2bfloat16(pos >= 0 ? y1 : 0.f);
-      dst[j + half] = __float2bfloat16(pos >= 0 ? y2 : 0.f);
-    } else if (pos >= 0) {
-      const int is_v = slot >= H + Hkv;
-      const int h = slot - H - (is_v ? Hkv : 0);
-      const int page = page_table[size_t(row_seq[r]) * pages_per_seq + pos / 16];
-      bf16* dst = pages_layer + size_t(page) * page_elems + (size_t(is_v) * Hkv + h) * 16 * dh + size_t(pos % 16) * dh;
-      dst[j] = __float2bfloat16(y1);
-      dst[j + half] = __float2bfloat16(y2);
-    }
-  }
+  if (threadIdx.x == 0) sumsq[r] = ss;
 }
 
 // Causal attention of the step's rows over the paged cache: grid (sequence, head).
@@ -320,7 +254,10 @@ LASER_API laser_status laser_model_create(const laser_model_cfg* cfg, const lase
   LASER_REQUIRE(cfg->n_layers >= 0 && cfg->d_model >= 16 && cfg->n_heads >= 1 && cfg->n_kv_heads >= 1 &&
                 cfg->d_ffn >= 16 && cfg->vocab >= 8, "bad model shape");
   LASER_REQUIRE(cfg->n_heads % cfg->n_kv_heads == 0, "n_heads must be a multiple of n_kv_heads");
-  LASER_REQUIRE(cfg->head_dim % 16 == 0 && cfg->head_dim >= 16 && cfg->head_dim <= 256, "head_dim = %d", cfg->head_dim);
+  LASER_REQUIRE(cfg->head_dim >= 16 && cfg->head_dim <= 128 && 128 % cfg->head_dim == 0,
+                "head_dim = %d (must be 16, 32, 64 or 128)", cfg->head_dim);
+  LASER_REQUIRE(cfg->d_model % 8 == 0 && cfg->d_ffn % 8 == 0 && cfg->vocab % 8 == 0,
+                "d_model, d_ffn and vocab must be multiples of 8");
   LASER_REQUIRE(cfg->page_size == 16, "page_size must be 16");
   LASER_REQUIRE(cfg->max_draft >= 0 && cfg->max_draft <= 63 && cfg->max_batch >= 1, "max_draft / max_batch");
   LASER_REQUIRE(w->tok_emb && w->lm_head && w->final_norm, "null weight");
@@ -360,11 +297,7 @@ LASER_API laser_status laser_model_create(const laser_model_cfg* cfg, const lase
   LASER_TRY(model_alloc(m, &m->q, Rp * m->dq));
   LASER_TRY(model_alloc(m, &m->attn, Rp * m->dq));
   LASER_TRY(model_alloc(m, &m->act, Rp * f));
-  size_t part = 0;
-  const int shapes[4][2] = {{m->dqkv, d}, {d, m->dq}, {2 * f, d}, {d, f}};
-  for (auto& s : shapes) part = std::max(part, size_t(gemm_plan(m->R_pad, s[0], s[1]).splits) * Rp * s[0]);
-  m->part_floats = part;
-  LASER_TRY(model_alloc(m, &m->part, part));
+  LASER_TRY(model_alloc(m, &m->sumsq, size_t(ceil_div(d, 128)) * Rp));
   LASER_TRY(model_alloc(m, &m->rope, Rp * (cfg->head_dim / 2) * 2));
   LASER_TRY(model_alloc(m, &m->row_pos, Rp));
   LASER_TRY(model_alloc(m, &m->row_seq, Rp));
@@ -509,7 +442,7 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
                                           double(c.rope_theta), dh, m->row_pos, m->row_seq, m->row_ctx, m->row_n,
                                           m->rope, m->status);
   const __nv_bfloat16* first_gain = c.n_layers > 0 ? m->attn_norm[0] : m->final_norm;
-  embed_norm_kernel<<<Rp, 256, 0, stream>>>(tokens, R, d, c.vocab, m->tok_emb, first_gain, c.rms_eps, m->resid, m->xn);
+  embed_kernel<<<Rp, 256, 0, stream>>>(tokens, R, d, c.vocab, m->tok_emb, first_gain, m->resid, m->xn, m->sumsq);
   count_launch(2);
   const bool use_tma_attn = attention_tma_supported(m, kv);
   const size_t attn_smem = (size_t(dh) + size_t(capacity) + 8) * sizeof(float);
@@ -517,15 +450,24 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
     LASER_REQUIRE(attn_smem <= 200 * 1024, "KV capacity of %d tokens per sequence exceeds the attention kernel's limit", capacity);
     LASER_CUDA(cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(attn_smem)));
   }
+  const int d_tiles = ceil_div(d, 128);
+  GemmEpilogue base;
+  base.R_rows = m->R_pad;
+  base.sumsq_ld = m->R_pad;
+  base.inv_d = 1.f / float(d);
+  base.eps = c.rms_eps;
+  int norm_tiles = 1;  // tile planes holding the sums of squares of the current residual
   for (int l = 0; l < c.n_layers; ++l) {
     __nv_bfloat16* pages_l = kv->pages + size_t(l) * kv->layer_elems();
-    // QKV projection, rotary embedding, cache write
-    GemmPlan p1 = gemm_plan(Rp, m->dqkv, d);
-    size_t stride = size_t(Rp) * m->dqkv;
-    { ProfScope ps(m, 0, stream); LASER_TRY(gemm_launch(m, m->xn, m->wqkv[l], m->part, Rp, Rp, m->dqkv, d, p1.splits, stride, m->dqkv, stream)); }
-    rope_kv_kernel<<<dim3(Rp, H + 2 * Hkv), 64, 0, stream>>>(m->part, p1.splits, stride, m->dqkv, H, Hkv, dh, m->rope,
-                                                             m->row_pos, m->row_seq, kv->page_table, kv->pages_per_seq,
-                                                             pages_l, kv->page_elems(), m->q);
+    {  // QKV projection of the normalised residual; rotary embedding; Q store; cache write
+      GemmEpilogue e = base;
+      e.sumsq_in = m->sumsq; e.sumsq_in_tiles = norm_tiles;
+      e.q = m->q; e.pages_layer = pages_l; e.page_elems = kv->page_elems(); e.page_table = kv->page_table;
+      e.pages_per_seq = kv->pages_per_seq; e.row_pos = m->row_pos; e.row_seq = m->row_seq; e.rope = m->rope;
+      e.H = H; e.Hkv = Hkv; e.dh = dh;
+      ProfScope ps(m, 0, stream);
+      LASER_TRY(gemm_fused(m, m->xn, m->wqkv[l], Rp, m->dqkv, d, EPI_QKV, e, stream));
+    }
     {
       ProfScope ps(m, 1, stream);
       if (use_tma_attn) {
@@ -537,25 +479,35 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
         count_launch();
       }
     }
-    // output projection, residual, norm
-    GemmPlan p2 = gemm_plan(Rp, d, m->dq);
-    stride = size_t(Rp) * d;
-    { ProfScope ps(m, 0, stream); LASER_TRY(gemm_launch(m, m->attn, m->wo[l], m->part, Rp, Rp, d, m->dq, p2.splits, stride, d, stream)); }
-    residual_norm_kernel<<<Rp, 256, 0, stream>>>(m->part, p2.splits, stride, d, d, m->ffn_norm[l], c.rms_eps, m->resid, m->xn);
-    // SwiGLU feed-forward, residual, next norm
-    GemmPlan p3 = gemm_plan(Rp, 2 * f, d);
-    stride = size_t(Rp) * 2 * f;
-    { ProfScope ps(m, 0, stream); LASER_TRY(gemm_launch(m, m->xn, m->wgu[l], m->part, Rp, Rp, 2 * f, d, p3.splits, stride, 2 * f, stream)); }
-    swiglu_kernel<<<dim3(ceil_div(f, 256), Rp), 256, 0, stream>>>(m->part, p3.splits, stride, f, m->act);
-    GemmPlan p4 = gemm_plan(Rp, d, f);
-    stride = size_t(Rp) * d;
-    { ProfScope ps(m, 0, stream); LASER_TRY(gemm_launch(m, m->act, m->wdown[l], m->part, Rp, Rp, d, f, p4.splits, stride, d, stream)); }
-    const __nv_bfloat16* next_gain = l + 1 < c.n_layers ? m->attn_norm[l + 1] : m->final_norm;
-    residual_norm_kernel<<<Rp, 256, 0, stream>>>(m->part, p4.splits, stride, d, d, next_gain, c.rms_eps, m->resid, m->xn);
-    count_launch(4);
+    {  // output projection; residual add; operand and statistics of the FFN norm
+      GemmEpilogue e = base;
+      e.resid = m->resid; e.xb = m->xn; e.gain_next = m->ffn_norm[l]; e.sumsq_out = m->sumsq;
+      ProfScope ps(m, 0, stream);
+      LASER_TRY(gemm_fused(m, m->attn, m->wo[l], Rp, d, m->dq, EPI_RESID, e, stream));
+    }
+    {  // gate and up projections of the normalised residual; SwiGLU
+      GemmEpilogue e = base;
+      e.sumsq_in = m->sumsq; e.sumsq_in_tiles = d_tiles;
+      e.act = m->act; e.f = f;
+      ProfScope ps(m, 0, stream);
+      LASER_TRY(gemm_fused(m, m->xn, m->wgu[l], Rp, 2 * f, d, EPI_SWIGLU, e, stream));
+    }
+    {  // down projection; residual add; operand and statistics of the next norm
+      GemmEpilogue e = base;
+      e.resid = m->resid; e.xb = m->xn; e.sumsq_out = m->sumsq;
+      e.gain_next = l + 1 < c.n_layers ? m->attn_norm[l + 1] : m->final_norm;
+      ProfScope ps(m, 0, stream);
+      LASER_TRY(gemm_fused(m, m->act, m->wdown[l], Rp, d, f, EPI_RESID, e, stream));
+    }
+    norm_tiles = d_tiles;
   }
-  // LM head straight into the caller's logits (one plane, rows beyond R not stored)
-  { ProfScope ps(m, 0, stream); LASER_TRY(gemm_launch(m, m->xn, m->lm_head, logits, Rp, R, c.vocab, d, 1, 0, c.vocab, stream)); }
+  {  // final norm (as a row scale) and LM head straight into the caller's logits
+    GemmEpilogue e = base;
+    e.sumsq_in = m->sumsq; e.sumsq_in_tiles = norm_tiles;
+    e.out = logits; e.ldo = c.vocab; e.R_store = R;
+    ProfScope ps(m, 0, stream);
+    LASER_TRY(gemm_fused(m, m->xn, m->lm_head, Rp, c.vocab, d, EPI_PLAIN, e, stream));
+  }
   LASER_CUDA(cudaGetLastError());
   return LASER_OK;
 }

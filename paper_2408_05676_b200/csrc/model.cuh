@@ -19,8 +19,7 @@ struct laser_model {
   __nv_bfloat16* q = nullptr;      // [R_pad, dq] rotated queries
   __nv_bfloat16* attn = nullptr;   // [R_pad, dq] attention output
   __nv_bfloat16* act = nullptr;    // [R_pad, f] SwiGLU output
-  float* part = nullptr;           // split-K partial sums
-  size_t part_floats = 0;
+  float* sumsq = nullptr;          // [ceil(d/128)][R_pad] per-tile sums of squares of the residual
   float* rope = nullptr;           // [R_pad, head_dim/2, 2] cos, sin of each row's position
   int32_t* row_pos = nullptr;      // [R_pad] position of the row, -1 = inactive
   int32_t* row_seq = nullptr;      // [R_pad] cache slot of the row
@@ -36,15 +35,43 @@ struct laser_model {
 
 namespace laser {
 
-// out[s][r][n] = sum over the s-th K-range of A[r][k] * W[n][k]; A bf16 [R_pad, K] row-major,
-// W bf16 [N, K] row-major, out fp32 with row stride ldo and split stride split_stride
-// (floats).  Rows >= R_store are not written.  Returns the number of splits used through
-// *splits_out; the caller sums the partial results.
-struct GemmPlan { int splits; };
-GemmPlan gemm_plan(int R_pad, int N, int K);
-laser_status gemm_launch(laser_model* m, const __nv_bfloat16* A, const __nv_bfloat16* W, float* out,
-                         int R_pad, int R_store, int N, int K, int splits, size_t split_stride, int ldo,
-                         cudaStream_t stream);
+// What the GEMM does with a finished 128-feature x NT-row accumulator tile.
+enum { EPI_PLAIN = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_QKV = 3 };
+
+struct GemmEpilogue {
+  int R_rows = 0;                    // rows the activation / output buffers really have
+  // RMSNorm of the A operand, applied as a per-row scale of the result: the producer left
+  // x * gain in bf16 and one sum of squares per (128-feature tile, row); null = no scale
+  const float* sumsq_in = nullptr;
+  int sumsq_in_tiles = 0, sumsq_ld = 0;
+  float inv_d = 0.f, eps = 0.f;
+  // EPI_PLAIN: out[r][n] = scale * acc (fp32), rows < R_store
+  float* out = nullptr;
+  int ldo = 0, R_store = 0;
+  // EPI_RESID: resid[r][n] += acc; xb = bf16(resid * gain_next); sumsq_out[tile][r]
+  float* resid = nullptr;
+  __nv_bfloat16* xb = nullptr;
+  const __nv_bfloat16* gain_next = nullptr;
+  float* sumsq_out = nullptr;
+  // EPI_SWIGLU: W is [gate rows | up rows] (f each); act[r][j] = silu(gate_j) * up_j
+  __nv_bfloat16* act = nullptr;
+  int f = 0;
+  // EPI_QKV: rotary embedding, Q store, K/V page write
+  __nv_bfloat16* q = nullptr;
+  __nv_bfloat16* pages_layer = nullptr;
+  size_t page_elems = 0;
+  const int32_t* page_table = nullptr;
+  int pages_per_seq = 0;
+  const int32_t* row_pos = nullptr;
+  const int32_t* row_seq = nullptr;
+  const float* rope = nullptr;
+  int H = 0, Hkv = 0, dh = 0;
+};
+
+// acc[r][n] = sum_k A[r][k] * W[n][k] (A bf16 [R_pad, K], W bf16 [N, K], both row-major),
+// finished by the epilogue `epi`.  N and K must be multiples of 8.
+laser_status gemm_fused(laser_model* m, const __nv_bfloat16* A, const __nv_bfloat16* W, int R_pad, int N, int K, int epi,
+                        const GemmEpilogue& e, cudaStream_t stream);
 void gemm_state_free(laser_model* m);
 
 // TMA-fed paged attention (head_dim 64 or 128 and a cache small enough for 32-bit row
