@@ -8,16 +8,21 @@
 // 128-wide M side of tcgen05.mma and the token rows the N side (NT <= 192, no padding of the
 // rows to 128); the accumulator is a 128 x NT fp32 tile in tensor memory.
 //
-// One CTA per (token tile, weight tile, K range); the CTAs that share an output tile form a
-// thread-block cluster along K.  Warp 0 streams weight and activation tiles with TMA
-// (128-byte swizzle) through a ring of shared-memory stages, warp 1 issues the MMAs and frees
-// stages with tcgen05.commit, warps 2-5 move the finished accumulator from tensor memory to
-// shared memory.  The partial tiles of a cluster are then summed through distributed shared
-// memory in a fixed order (run-to-run identical results, no partial sums in global memory);
-// each CTA reduces and finishes its own slice of the token columns with the fused epilogue.
-// Two CTAs fit on an SM, so one CTA's epilogue overlaps another's main loop.
-// Every mbarrier wait is bounded: on expiry the CTA records LASER_ERR_TIMEOUT, drains its
-// copies, still joins the cluster barriers, frees its tensor memory and exits.
+// Persistent kernel, one CTA per SM, CTAs grouped in thread-block clusters of `splits` along K.
+// A cluster walks the output tiles assigned to it; each of its CTAs contracts its own K range
+// of the tile.  Roles inside a CTA:
+//   warp 0     TMA producer: weight and activation tiles (128-byte swizzle) into a ring of
+//              shared-memory stages, running ahead across tile boundaries;
+//   warp 1     MMA issuer: tcgen05.mma into one of two TMEM accumulators, tcgen05.commit frees
+//              stages and publishes finished accumulators;
+//   warps 2-5  epilogue: read the accumulator (tcgen05.ld), send every token column to the
+//              CTA of the cluster that owns it (distributed shared memory), then sum the
+//              `splits` partial columns they own in rank order (run-to-run identical, no
+//              partial sums in global memory) and apply the fused epilogue.
+// The epilogue of tile i overlaps the main loop of tile i+1 (double-buffered accumulator);
+// cross-CTA hand-over uses cluster-scope mbarriers.  Every wait is bounded: on expiry the CTA
+// records LASER_ERR_TIMEOUT, stops issuing work, still joins the final cluster barrier, frees
+// its tensor memory and exits.
 #include <map>
 #include <tuple>
 
@@ -33,7 +38,7 @@ constexpr int kBM = 128;          // weight rows per tile (MMA M)
 constexpr int kBK = 64;           // K elements per stage = one 128-byte swizzle span of bf16
 constexpr int kMaxStages = 6;
 constexpr int kMaxNT = 192;       // token rows per tile: accumulator staging must fit shared memory
-constexpr int kSmemBudget = 110 * 1024;
+constexpr int kSmemLimit = 222 * 1024;   // dynamic shared memory one CTA may ask for
 
 // Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows 128 B apart, groups
 // of 8 rows 1024 B apart.
@@ -57,12 +62,42 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ float4 ld_cluster_f4(uint32_t local_addr, uint32_t rank) {
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {
   uint32_t remote;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-  float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
-  return v;
+  return remote;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait on a barrier that peers of the cluster arrive on.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_cluster(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_cluster(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; return false; }
+  }
+}
+// AND of a flag over the 128 epilogue threads (named barrier 1), so that they leave a loop together.
+__device__ __forceinline__ bool epilogue_all(bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n.reg .pred p, q;\nsetp.ne.u32 q, %1, 0;\nbar.red.and.pred p, 1, 128, q;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(r) : "r"(uint32_t(ok)) : "memory");
+  return r != 0;
 }
 __device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
   __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
@@ -118,7 +153,8 @@ __device__ __forceinline__ void epi_swiglu(const GemmEpilogue& e, int r, int f0,
 }
 
 // rotary embedding of Q and K (pair i, i + dh/2), bf16 rounding, Q store, K/V page write
-__device__ __forceinline__ void epi_qkv(const GemmEpilogue& e, int r, int n0, int lane, float4 v, float rstd, int N) {
+__device__ __forceinline__ void epi_qkv(const GemmEpilogue& e, int r, int n0, int lane, float4 v, float rstd, int N,
+                                        int pos, int page) {
   v.x *= rstd; v.y *= rstd; v.z *= rstd; v.w *= rstd;
   const int dh = e.dh, half = dh >> 1, dq = e.H * dh, dkv = e.Hkv * dh;
   const int shift = dh >> 3;  // lanes between a feature and its rotation partner
@@ -127,7 +163,6 @@ __device__ __forceinline__ void epi_qkv(const GemmEpilogue& e, int r, int n0, in
   pv.z = __shfl_xor_sync(0xffffffffu, v.z, shift); pv.w = __shfl_xor_sync(0xffffffffu, v.w, shift);
   const int n = n0 + 4 * lane;
   if (n >= N) return;
-  const int pos = e.row_pos[r];
   const int idx = n % dh;          // four consecutive features stay inside one half of one head
   float4 y = v;
   if (n < dq + dkv) {
@@ -146,156 +181,201 @@ __device__ __forceinline__ void epi_qkv(const GemmEpilogue& e, int r, int n0, in
   } else if (pos >= 0) {
     const int is_v = n >= dq + dkv;
     const int h = (n - dq - is_v * dkv) / dh;
-    const int page = e.page_table[size_t(e.row_seq[r]) * e.pages_per_seq + (pos >> 4)];
     bf16* dst = e.pages_layer + size_t(page) * e.page_elems + (size_t(is_v) * e.Hkv + h) * 16 * dh + size_t(pos & 15) * dh + idx;
     *reinterpret_cast<uint2*>(dst) = pack4_bf16(y.x, y.y, y.z, y.w);
   }
 }
 
+
 template <int EPI>
-__global__ void __launch_bounds__(kTcThreads)
+__global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, const GemmEpilogue e,
-               int N, int NT, int total_kb, int kb_per_split, int splits, int stages, int tmem_cols,
+               int N, int NT, int n_ttiles, int n_wtiles, int total_kb, int kb_per_split, int splits, int stages,
                int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_bar;
+  __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages];
+  __shared__ uint64_t acc_full[2], acc_empty[2];   // TMEM accumulator hand-over MMA <-> epilogue
+  __shared__ uint64_t red_full, red_free;          // reduction buffer hand-over between cluster peers
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   __shared__ float s_rstd[kMaxNT];
+  __shared__ int s_pos[kMaxNT], s_page[kMaxNT];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
-  float* stage_acc = reinterpret_cast<float*>(smem_raw + (tiles - raw));  // [NT][128] after the main loop
   const uint32_t w_bytes = kBM * 128, a_bytes = uint32_t(NT) * 128, stage_bytes = w_bytes + a_bytes;
+  const int slice = (NT + splits - 1) / splits;            // token columns owned by one CTA of the cluster
+  const uint32_t red_addr = tiles + uint32_t(stages) * stage_bytes;   // [splits][slice][128] fp32
+  const float* red = reinterpret_cast<const float*>(smem_raw + (red_addr - raw));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int krank = blockIdx.x % splits, ttile = blockIdx.x / splits, wtile = blockIdx.y;
-  const int r0 = ttile * NT, n0 = wtile * kBM;
+  const int krank = blockIdx.x % splits, cluster_id = blockIdx.x / splits, n_clusters = gridDim.x / splits;
+  const int n_tiles = n_ttiles * n_wtiles;
   const int kb0 = krank * kb_per_split;
   const int nkb = max(0, min(kb_per_split, total_kb - kb0));
-  // rows of the weight matrix behind the two 64-row halves of the tile
-  const int wrow0 = EPI == EPI_SWIGLU ? wtile * 64 : n0;
-  const int wrow1 = EPI == EPI_SWIGLU ? e.f + wtile * 64 : n0 + 64;
+  constexpr int kAccCols = 256;                             // TMEM columns per accumulator buffer
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
-    mbar_init(smem_u32(&acc_bar), 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&acc_full[b]), 1); mbar_init(smem_u32(&acc_empty[b]), 1); }
+    mbar_init(smem_u32(&red_full), uint32_t(splits));
+    mbar_init(smem_u32(&red_free), uint32_t(splits));
     mbar_fence_init();
     tma_prefetch_map(&tmW);
     tma_prefetch_map(&tmA);
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(2 * kAccCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  if (splits > 1) cluster_sync_all();   // peers' barriers exist before anyone arrives on them
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_acc = tmem_slot;
+  const uint32_t tmem_base = tmem_slot;
 
   if (warp == 0) {
-    if (lane == 0) {  // TMA producer
-      int issued = 0;
+    if (lane == 0) {  // ---- TMA producer ----
+      int it = 0;
       bool ok = true;
-      for (int kb = 0; kb < nkb && ok; ++kb) {
-        const int s = kb % stages;
-        if (kb >= stages) ok = mbar_wait(smem_u32(&empty_bar[s]), ((kb / stages) - 1) & 1, &abort_flag);
-        if (!ok) break;
-        const uint32_t bar = smem_u32(&full_bar[s]);
-        const uint32_t dst = tiles + uint32_t(s) * stage_bytes;
-        mbar_expect_tx(bar, stage_bytes);
-        const int k = (kb0 + kb) * kBK;
-        tma_load_2d(dst, &tmW, k, wrow0, bar);
-        tma_load_2d(dst + w_bytes / 2, &tmW, k, wrow1, bar);
-        tma_load_2d(dst + w_bytes, &tmA, k, r0, bar);
-        issued = kb + 1;
+      for (int t = cluster_id; t < n_tiles && ok; t += n_clusters) {
+        const int ttile = t % n_ttiles, wtile = t / n_ttiles;
+        const int wrow0 = EPI == EPI_SWIGLU ? wtile * 64 : wtile * kBM;
+        const int wrow1 = EPI == EPI_SWIGLU ? e.f + wtile * 64 : wtile * kBM + 64;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % stages;
+          if (it >= stages) ok = mbar_wait(smem_u32(&empty_bar[s]), ((it / stages) - 1) & 1, &abort_flag);
+          if (!ok) break;
+          const uint32_t bar = smem_u32(&full_bar[s]);
+          const uint32_t dst = tiles + uint32_t(s) * stage_bytes;
+          mbar_expect_tx(bar, stage_bytes);
+          const int k = (kb0 + kb) * kBK;
+          tma_load_2d(dst, &tmW, k, wrow0, bar);
+          tma_load_2d(dst + w_bytes / 2, &tmW, k, wrow1, bar);
+          tma_load_2d(dst + w_bytes, &tmA, k, ttile * NT, bar);
+        }
       }
       if (!ok)  // drain copies still in flight before the CTA may exit
-        for (int kb = max(0, issued - stages); kb < issued; ++kb) mbar_drain(smem_u32(&full_bar[kb % stages]), (kb / stages) & 1);
+        for (int j = max(0, it - stages); j < it; ++j) mbar_drain(smem_u32(&full_bar[j % stages]), (j / stages) & 1);
     }
   } else if (warp == 1) {
-    if (lane == 0) {  // MMA issuer
+    if (lane == 0) {  // ---- MMA issuer ----
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(NT >> 3) << 17) | (uint32_t(kBM >> 4) << 24);
+      int it = 0, i = 0;
       bool ok = true;
-      for (int kb = 0; kb < nkb && ok; ++kb) {
-        const int s = kb % stages;
-        ok = mbar_wait(smem_u32(&full_bar[s]), (kb / stages) & 1, &abort_flag);
+      for (int t = cluster_id; t < n_tiles && ok; t += n_clusters, ++i) {
+        const int buf = i & 1;
+        if (i >= 2) ok = mbar_wait(smem_u32(&acc_empty[buf]), ((i >> 1) - 1) & 1, &abort_flag);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t w_addr = tiles + uint32_t(s) * stage_bytes;
-        const uint64_t wdesc = umma_desc(w_addr), adesc = umma_desc(w_addr + w_bytes);
+        const uint32_t tmem_acc = tmem_base + uint32_t(buf * kAccCols);
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % stages;
+          ok = mbar_wait(smem_u32(&full_bar[s]), (it / stages) & 1, &abort_flag);
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t w_addr = tiles + uint32_t(s) * stage_bytes;
+          const uint64_t wdesc = umma_desc(w_addr), adesc = umma_desc(w_addr + w_bytes);
 #pragma unroll
-        for (int k = 0; k < kBK / 16; ++k)  // 16 bf16 = 32 bytes further along K inside the swizzle span
-          umma_bf16(tmem_acc, wdesc + uint64_t(k * 2), adesc + uint64_t(k * 2), idesc, (kb | k) != 0);
-        umma_commit(smem_u32(&empty_bar[s]));
+          for (int k = 0; k < kBK / 16; ++k)  // 16 bf16 = 32 bytes further along K inside the swizzle span
+            umma_bf16(tmem_acc, wdesc + uint64_t(k * 2), adesc + uint64_t(k * 2), idesc, (kb | k) != 0);
+          umma_commit(smem_u32(&empty_bar[s]));
+        }
+        if (ok) umma_commit(smem_u32(&acc_full[buf]));  // arrives when the tile's MMAs have finished
       }
-      umma_commit(smem_u32(&acc_bar));  // arrives when every MMA issued so far has finished
     }
   } else {
-    // RMSNorm scale of each token row of this tile, from the producer's per-tile sums of squares
-    for (int j = threadIdx.x - 64; j < NT; j += 128) {
-      float rstd = 1.f;
-      if (e.sumsq_in && r0 + j < e.R_rows) {
-        float ss = 0.f;
-        for (int t = 0; t < e.sumsq_in_tiles; ++t) ss += e.sumsq_in[size_t(t) * e.sumsq_ld + r0 + j];
-        rstd = rsqrtf(ss * e.inv_d + e.eps);
-      }
-      s_rstd[j] = rstd;
-    }
-    // accumulator: tensor memory -> shared memory, token-major [NT][128]
+    // ---- epilogue warps ----
+    const int et = threadIdx.x - 64, ew = warp - 2;
     const int quarter = warp & 3;  // a warp may only touch its own 32 TMEM lanes
-    const bool ok = mbar_wait(smem_u32(&acc_bar), 0, &abort_flag);
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    for (int c = 0; c < NT; c += 16) {
-      uint32_t v[16];
-      if (ok && nkb > 0) {
-        const uint32_t taddr = tmem_acc + (uint32_t(quarter * 32) << 16) + uint32_t(c);
+    int i = 0, cur_ttile = -1;
+    bool ok = true;
+    for (int t = cluster_id; t < n_tiles && ok; t += n_clusters, ++i) {
+      const int ttile = t % n_ttiles, wtile = t / n_ttiles, buf = i & 1;
+      const int r0 = ttile * NT, n0 = wtile * kBM;
+      if (ttile != cur_ttile) {  // per-row scale and cache coordinates of this token tile
+        cur_ttile = ttile;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        for (int j = et; j < NT; j += 128) {
+          const int r = r0 + j;
+          float rstd = 1.f;
+          int pos = -1, page = 0;
+          if (r < e.R_rows) {
+            if (e.sumsq_in) {
+              float ss = 0.f;
+              for (int tt = 0; tt < e.sumsq_in_tiles; ++tt) ss += e.sumsq_in[size_t(tt) * e.sumsq_ld + r];
+              rstd = rsqrtf(ss * e.inv_d + e.eps);
+            }
+            if (EPI == EPI_QKV) {
+              pos = e.row_pos[r];
+              if (pos >= 0) page = e.page_table[size_t(e.row_seq[r]) * e.pages_per_seq + (pos >> 4)];
+            }
+          }
+          s_rstd[j] = rstd; s_pos[j] = pos; s_page[j] = page;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+      }
+      ok = mbar_wait(smem_u32(&acc_full[buf]), (i >> 1) & 1, &abort_flag);
+      // the owners must have finished summing the previous tile before their buffers are overwritten
+      if (ok && splits > 1 && i >= 1) ok = mbar_wait_cluster(smem_u32(&red_free), (i - 1) & 1, &abort_flag);
+      ok = epilogue_all(ok);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      // send every token column of this partial tile to its owner: [rank][column][128 features]
+      const uint32_t tmem_acc = tmem_base + uint32_t(buf * kAccCols) + (uint32_t(quarter * 32) << 16);
+      for (int c = 0; c < NT; c += 16) {
+        uint32_t v[16];
         asm volatile(
             "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
             : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
               "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-            : "r"(taddr) : "memory");
+            : "r"(tmem_acc + uint32_t(c)) : "memory");
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      } else {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] = 0u;
+        for (int x = 0; x < 16; ++x) {
+          const int j = c + x, owner = j / slice, jj = j - owner * slice;
+          const uint32_t local = red_addr + uint32_t(((krank * slice + jj) * kBM + quarter * 32 + lane) * 4);
+          st_cluster_f32(splits > 1 ? map_to_rank(local, uint32_t(owner)) : local, __uint_as_float(v[x]));
+        }
       }
-#pragma unroll
-      for (int i = 0; i < 16; ++i) stage_acc[(c + i) * kBM + quarter * 32 + lane] = __uint_as_float(v[i]);
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (et == 0) {
+        mbar_arrive(smem_u32(&acc_empty[buf]));   // the accumulator may be overwritten
+        if (splits > 1) {
+          asm volatile("fence.acq_rel.cluster;" ::: "memory");
+          for (int rk = 0; rk < splits; ++rk) mbar_arrive_cluster(map_to_rank(smem_u32(&red_full), uint32_t(rk)));
+        }
+      }
+      if (splits > 1) {
+        ok = epilogue_all(mbar_wait_cluster(smem_u32(&red_full), i & 1, &abort_flag));
+        if (!ok) break;
+      }
+      // sum the partial columns this CTA owns (ranks in order) and finish them
+      const int own = min(slice, NT - krank * slice);
+      for (int jj = ew; jj < own; jj += 4) {
+        float4 v = *reinterpret_cast<const float4*>(red + (jj * kBM + 4 * lane));
+        for (int rk = 1; rk < splits; ++rk) {
+          const float4 w = *reinterpret_cast<const float4*>(red + ((rk * slice + jj) * kBM + 4 * lane));
+          v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+        }
+        const int j = krank * slice + jj, r = r0 + j;
+        if (r >= e.R_rows) continue;   // the last token tile may overhang the buffers
+        const float rstd = s_rstd[j];
+        if (EPI == EPI_PLAIN) epi_plain(e, r, n0, lane, v, rstd, N);
+        else if (EPI == EPI_RESID) epi_resid(e, r, n0, lane, v, N, wtile);
+        else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, wtile * 64, lane, v, rstd);
+        else epi_qkv(e, r, n0, lane, v, rstd, N, s_pos[j], s_page[j]);
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");   // buffer fully read
+      if (splits > 1 && et == 0)
+        for (int rk = 0; rk < splits; ++rk) mbar_arrive_cluster(map_to_rank(smem_u32(&red_free), uint32_t(rk)));
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (splits > 1) cluster_sync_all();  // every partial tile of the cluster is staged
-
-  // each CTA sums and finishes its slice of the token columns; ranks are added in order 0..splits-1
-  {
-    const int slice = (NT + splits - 1) / splits;
-    const int j_lo = krank * slice, j_hi = min(NT, j_lo + slice);
-    const uint32_t stage_addr = tiles;
-    for (int j = j_lo + warp; j < j_hi; j += kTcThreads / 32) {
-      float4 v;
-      if (splits > 1) {
-        v = ld_cluster_f4(stage_addr + uint32_t(j * kBM + 4 * lane) * 4, 0);
-        for (int rk = 1; rk < splits; ++rk) {
-          const float4 w = ld_cluster_f4(stage_addr + uint32_t(j * kBM + 4 * lane) * 4, uint32_t(rk));
-          v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
-        }
-      } else {
-        v = *reinterpret_cast<const float4*>(stage_acc + j * kBM + 4 * lane);
-      }
-      const int r = r0 + j;
-      if (r >= e.R_rows) continue;   // the last token tile may overhang the buffers
-      const float rstd = s_rstd[j];
-      if (EPI == EPI_PLAIN) epi_plain(e, r, n0, lane, v, rstd, N);
-      else if (EPI == EPI_RESID) epi_resid(e, r, n0, lane, v, N, wtile);
-      else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, wtile * 64, lane, v, rstd);
-      else epi_qkv(e, r, n0, lane, v, rstd, N);
-    }
-  }
-  if (splits > 1) cluster_sync_all();  // peers may still be reading this CTA's staged tile
-  __syncthreads();
+  if (splits > 1) cluster_sync_all();  // nobody leaves while a peer may still write to it
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * kAccCols) : "memory");
   }
   if (threadIdx.x == 0 && abort_flag) atomicCAS(status, 0, LASER_ERR_TIMEOUT);
 }
@@ -304,7 +384,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 struct GemmState {
   // (pointer, rows, cols, box rows) -> tensor map
   std::map<std::tuple<const void*, int, int, int>, CUtensorMap> maps;
-  bool attrs_set = false;
+  bool ready = false;
+  int max_clusters[5] = {0, 0, 0, 0, 0};   // co-resident clusters of size 1, 2, 4 (index = size)
 };
 
 GemmState* get_state(laser_model* m) {
@@ -324,58 +405,91 @@ laser_status tensor_map(GemmState* st, const void* ptr, int rows, int cols, int 
   return LASER_OK;
 }
 
-struct TcShape { int n_tiles, NT, stages, tmem_cols; size_t smem; };
+struct TcShape { int n_ttiles, NT, stages; size_t smem; };
 
-TcShape tc_shape(int R_pad) {
+TcShape tc_shape(int R_pad, int splits) {
   TcShape s;
-  s.n_tiles = ceil_div(R_pad, kMaxNT);
-  s.NT = ceil_div(ceil_div(R_pad, s.n_tiles), 16) * 16;
+  s.n_ttiles = ceil_div(R_pad, kMaxNT);
+  s.NT = ceil_div(ceil_div(R_pad, s.n_ttiles), 16) * 16;
   const int stage_bytes = kBM * 128 + s.NT * 128;
-  s.stages = std::max(2, std::min(kMaxStages, kSmemBudget / stage_bytes));
-  s.tmem_cols = 32;
-  while (s.tmem_cols < s.NT) s.tmem_cols <<= 1;
-  s.smem = std::max(size_t(s.stages) * stage_bytes, size_t(s.NT) * kBM * 4) + 1024;
+  const int red_bytes = splits * ceil_div(s.NT, splits) * kBM * 4;
+  s.stages = std::max(2, std::min(kMaxStages, (kSmemLimit - 1024 - red_bytes) / stage_bytes));
+  s.smem = size_t(s.stages) * stage_bytes + red_bytes + 1024;
   return s;
 }
 
 template <int EPI>
-laser_status launch_epi(const CUtensorMap& tw, const CUtensorMap& ta, const GemmEpilogue& e, int N, const TcShape& sh,
-                        int w_tiles, int total_kb, int kbps, int splits, int32_t* status, cudaStream_t stream) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(unsigned(sh.n_tiles * splits), unsigned(w_tiles), 1);
-  cfg.blockDim = dim3(kTcThreads, 1, 1);
-  cfg.dynamicSmemBytes = sh.smem;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+void fill_launch(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int grid, int splits, size_t smem, cudaStream_t stream) {
+  *cfg = cudaLaunchConfig_t{};
+  cfg->gridDim = dim3(unsigned(grid), 1, 1);
+  cfg->blockDim = dim3(kTcThreads, 1, 1);
+  cfg->dynamicSmemBytes = smem;
+  cfg->stream = stream;
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = unsigned(splits);
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  LASER_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI>, tw, ta, e, N, sh.NT, total_kb, kbps, splits, sh.stages,
-                                sh.tmem_cols, status));
+  cfg->attrs = attr;
+  cfg->numAttrs = 1;
+}
+
+template <int EPI>
+laser_status launch_epi(const CUtensorMap& tw, const CUtensorMap& ta, const GemmEpilogue& e, int N, const TcShape& sh,
+                        int n_wtiles, int total_kb, int kbps, int splits, int clusters, int32_t* status,
+                        cudaStream_t stream) {
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  fill_launch<EPI>(&cfg, attr, clusters * splits, splits, sh.smem, stream);
+  LASER_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI>, tw, ta, e, N, sh.NT, sh.n_ttiles, n_wtiles, total_kb, kbps,
+                                splits, sh.stages, status));
   return LASER_OK;
 }
 
-}  // namespace
+// One-off per model: opt in to large shared memory and ask how many clusters of each size fit.
+laser_status prepare(GemmState* st) {
+  if (st->ready) return LASER_OK;
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
+  int sms = 0, dev = 0;
+  LASER_CUDA(cudaGetDevice(&dev));
+  LASER_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  for (int s : {1, 2, 4}) {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    fill_launch<EPI_RESID>(&cfg, attr, (sms / s) * s, s, size_t(kSmemLimit) - 8192, nullptr);
+    int n = 0;
+    cudaError_t err = cudaOccupancyMaxActiveClusters(&n, gemm_tc_kernel<EPI_RESID>, &cfg);
+    if (err != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+    st->max_clusters[s] = std::max(0, std::min(n, sms / s));
+  }
+  if (st->max_clusters[1] <= 0) { set_error("the GEMM kernel does not fit this device"); return LASER_ERR_UNSUPPORTED; }
+  st->ready = true;
+  return LASER_OK;
+}
 
-int gemm_splits(int R_pad, int N, int K, int epi) {
-  // Modelled time: CTAs are spread over 148 SMs (two resident per SM); each costs its K blocks
-  // plus a fixed prologue/epilogue share; the cluster reduction grows with the split count.
-  const TcShape sh = tc_shape(R_pad);
-  const int w_tiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
-  const int tiles = w_tiles * sh.n_tiles, total_kb = ceil_div(K, kBK);
-  int best = 1;
+// Split count (cluster size) with the least modelled time: clusters work in lock step on one
+// tile each, a tile costs the K blocks of one rank plus a fixed share.
+int pick_splits(const GemmState* st, int R_pad, int N, int K, int epi, int* clusters_out) {
+  const int n_wtiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
+  const int total_kb = ceil_div(K, kBK);
+  int best = 1, best_clusters = 1;
   double best_cost = 1e30;
-  for (int s = 1; s <= std::min(total_kb, 8); ++s) {
+  for (int s : {1, 2, 4}) {
+    if (st->max_clusters[s] <= 0) continue;
     const int kbps = ceil_div(total_kb, s);
     if (kbps * (s - 1) >= total_kb) continue;  // a rank would have no K blocks
-    const double cost = double(ceil_div(tiles * s, 148)) * (kbps + 4.0) + 0.5 * s;
-    if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
+    const int tiles = n_wtiles * tc_shape(R_pad, s).n_ttiles;
+    const int clusters = std::min(st->max_clusters[s], tiles);
+    const double cost = double(ceil_div(tiles, clusters)) * (kbps + 1.5) + 2.0 + 0.5 * s;
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = s; best_clusters = clusters; }
   }
+  *clusters_out = best_clusters;
   return best;
 }
+
+}  // namespace
 
 laser_status gemm_fused(laser_model* m, const __nv_bfloat16* A, const __nv_bfloat16* W, int R_pad, int N, int K, int epi,
                         const GemmEpilogue& e, cudaStream_t stream) {
@@ -384,25 +498,20 @@ laser_status gemm_fused(laser_model* m, const __nv_bfloat16* A, const __nv_bfloa
     return LASER_ERR_UNSUPPORTED;
   }
   GemmState* st = get_state(m);
-  if (!st->attrs_set) {
-    LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048));
-    LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048));
-    LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048));
-    LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048));
-    st->attrs_set = true;
-  }
-  const TcShape sh = tc_shape(R_pad);
+  LASER_TRY(prepare(st));
+  int clusters = 1;
+  const int splits = pick_splits(st, R_pad, N, K, epi, &clusters);
+  const TcShape sh = tc_shape(R_pad, splits);
   const CUtensorMap *tw = nullptr, *ta = nullptr;
   LASER_TRY(tensor_map(st, W, N, K, 64, &tw));
   LASER_TRY(tensor_map(st, A, m->R_pad, K, sh.NT, &ta));
-  const int splits = gemm_splits(R_pad, N, K, epi);
   const int total_kb = ceil_div(K, kBK), kbps = ceil_div(total_kb, splits);
-  const int w_tiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
+  const int n_wtiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
   switch (epi) {
-    case EPI_PLAIN: LASER_TRY(launch_epi<EPI_PLAIN>(*tw, *ta, e, N, sh, w_tiles, total_kb, kbps, splits, m->status, stream)); break;
-    case EPI_RESID: LASER_TRY(launch_epi<EPI_RESID>(*tw, *ta, e, N, sh, w_tiles, total_kb, kbps, splits, m->status, stream)); break;
-    case EPI_SWIGLU: LASER_TRY(launch_epi<EPI_SWIGLU>(*tw, *ta, e, N, sh, w_tiles, total_kb, kbps, splits, m->status, stream)); break;
-    default: LASER_TRY(launch_epi<EPI_QKV>(*tw, *ta, e, N, sh, w_tiles, total_kb, kbps, splits, m->status, stream)); break;
+    case EPI_PLAIN: LASER_TRY(launch_epi<EPI_PLAIN>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, clusters, m->status, stream)); break;
+    case EPI_RESID: LASER_TRY(launch_epi<EPI_RESID>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, clusters, m->status, stream)); break;
+    case EPI_SWIGLU: LASER_TRY(launch_epi<EPI_SWIGLU>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, clusters, m->status, stream)); break;
+    default: LASER_TRY(launch_epi<EPI_QKV>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, clusters, m->status, stream)); break;
   }
   count_launch();
   return LASER_OK;
