@@ -39,6 +39,7 @@ constexpr int kBK = 64;           // K elements per stage = one 128-byte swizzle
 constexpr int kMaxStages = 6;
 constexpr int kMaxNT = 192;       // token rows per tile: accumulator staging must fit shared memory
 constexpr int kSmemLimit = 222 * 1024;   // dynamic shared memory one CTA may ask for
+constexpr int kBatch = 3, kPre = 3;      // epilogue: columns per group, groups whose operands are prefetched
 
 // Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows 128 B apart, groups
 // of 8 rows 1024 B apart.
@@ -68,7 +69,7 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t ra
   return remote;
 }
 __device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v) {
-  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v));
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
@@ -90,6 +91,20 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
     if (*abort_flag) return false;
     if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; return false; }
   }
+}
+// 16 consecutive fp32 columns of this thread's TMEM lane (no wait: pair with tmem_ld_wait)
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float4 ld_shared_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
 }
 // AND of a flag over the 128 epilogue threads (named barrier 1), so that they leave a loop together.
 __device__ __forceinline__ bool epilogue_all(bool ok) {
@@ -122,14 +137,13 @@ __device__ __forceinline__ void epi_plain(const GemmEpilogue& e, int r, int n0, 
 }
 
 // resid += acc; xb = bf16(resid * gain of the next norm); per-tile sum of squares for that norm
-__device__ __forceinline__ void epi_resid(const GemmEpilogue& e, int r, int n0, int lane, float4 v, int N, int tile) {
+__device__ __forceinline__ void epi_resid(const GemmEpilogue& e, int r, int n0, int lane, float4 v, int N, int tile,
+                                          float4 x, uint2 g2) {
   const int n = n0 + 4 * lane;
   float ss = 0.f;
   if (n < N) {  // N is a multiple of 8 (checked on the host), so the four features are all valid
-    float4 x = *reinterpret_cast<float4*>(e.resid + size_t(r) * N + n);
     x.x += v.x; x.y += v.y; x.z += v.z; x.w += v.w;
     *reinterpret_cast<float4*>(e.resid + size_t(r) * N + n) = x;
-    const uint2 g2 = *reinterpret_cast<const uint2*>(e.gain_next + n);
     const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&g2.x), g23 = *reinterpret_cast<const __nv_bfloat162*>(&g2.y);
     *reinterpret_cast<uint2*>(e.xb + size_t(r) * N + n) =
         pack4_bf16(x.x * __low2float(g01), x.y * __high2float(g01), x.z * __low2float(g23), x.w * __high2float(g23));
@@ -146,7 +160,7 @@ __device__ __forceinline__ void epi_swiglu(const GemmEpilogue& e, int r, int f0,
   u.z = __shfl_xor_sync(0xffffffffu, v.z, 16); u.w = __shfl_xor_sync(0xffffffffu, v.w, 16);
   const int fidx = f0 + 4 * lane;
   if (lane < 16 && fidx < e.f) {  // f is a multiple of 8 (checked on the host)
-    auto act = [rstd](float g, float up) { g *= rstd; up *= rstd; return g / (1.f + __expf(-g)) * up; };
+    auto act = [rstd](float g, float up) { g *= rstd; up *= rstd; return __fdividef(g, 1.f + __expf(-g)) * up; };
     *reinterpret_cast<uint2*>(e.act + size_t(r) * e.f + fidx) =
         pack4_bf16(act(v.x, u.x), act(v.y, u.y), act(v.z, u.z), act(v.w, u.w));
   }
@@ -154,7 +168,7 @@ __device__ __forceinline__ void epi_swiglu(const GemmEpilogue& e, int r, int f0,
 
 // rotary embedding of Q and K (pair i, i + dh/2), bf16 rounding, Q store, K/V page write
 __device__ __forceinline__ void epi_qkv(const GemmEpilogue& e, int r, int n0, int lane, float4 v, float rstd, int N,
-                                        int pos, int page) {
+                                        int pos, int page, float4 cs01, float4 cs23) {
   v.x *= rstd; v.y *= rstd; v.z *= rstd; v.w *= rstd;
   const int dh = e.dh, half = dh >> 1, dq = e.H * dh, dkv = e.Hkv * dh;
   const int shift = dh >> 3;  // lanes between a feature and its rotation partner
@@ -166,9 +180,6 @@ __device__ __forceinline__ void epi_qkv(const GemmEpilogue& e, int r, int n0, in
   const int idx = n % dh;          // four consecutive features stay inside one half of one head
   float4 y = v;
   if (n < dq + dkv) {
-    const int j = idx % half;
-    const float4 cs01 = *reinterpret_cast<const float4*>(e.rope + (size_t(r) * half + j) * 2);      // c0 s0 c1 s1
-    const float4 cs23 = *reinterpret_cast<const float4*>(e.rope + (size_t(r) * half + j + 2) * 2);  // c2 s2 c3 s3
     const float sg = idx < half ? -1.f : 1.f;
     y.x = v.x * cs01.x + sg * pv.x * cs01.y;
     y.y = v.y * cs01.z + sg * pv.y * cs01.w;
@@ -292,6 +303,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     for (int t = cluster_id; t < n_tiles && ok; t += n_clusters, ++i) {
       const int ttile = t % n_ttiles, wtile = t / n_ttiles, buf = i & 1;
       const int r0 = ttile * NT, n0 = wtile * kBM;
+      // Global operands of the fused epilogue (residual, rotary table, gains) do not depend on
+      // this kernel: ask for the first groups now, long before the accumulator is ready.
+      const int own = min(slice, NT - krank * slice);
+      const int nfeat = n0 + 4 * lane;
+      auto fetch_operands = [&](int jj, float4& g0, float4& g1) {
+        g0 = make_float4(0.f, 0.f, 0.f, 0.f); g1 = g0;
+        const int r = r0 + krank * slice + jj;
+        if (jj < own && r < e.R_rows && nfeat < N) {
+          if (EPI == EPI_RESID) g0 = *reinterpret_cast<const float4*>(e.resid + size_t(r) * N + nfeat);
+          if (EPI == EPI_QKV && nfeat < (e.H + e.Hkv) * e.dh) {
+            const float* cs = e.rope + (size_t(r) * (e.dh >> 1) + (nfeat % e.dh) % (e.dh >> 1)) * 2;
+            g0 = *reinterpret_cast<const float4*>(cs);       // c0 s0 c1 s1
+            g1 = *reinterpret_cast<const float4*>(cs + 4);   // c2 s2 c3 s3
+          }
+        }
+      };
+      uint2 gain4 = make_uint2(0u, 0u);   // gains of this lane's four features (next norm)
+      if (EPI == EPI_RESID && nfeat < N) gain4 = *reinterpret_cast<const uint2*>(e.gain_next + nfeat);
+      float4 pg0[kPre][kBatch], pg1[kPre][kBatch];
+#pragma unroll
+      for (int k = 0; k < kPre; ++k)
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) fetch_operands((ew + 4 * k) * kBatch + b, pg0[k][b], pg1[k][b]);
       if (ttile != cur_ttile) {  // per-row scale and cache coordinates of this token tile
         cur_ttile = ttile;
         asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -322,19 +356,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       // send every token column of this partial tile to its owner: [rank][column][128 features]
       const uint32_t tmem_acc = tmem_base + uint32_t(buf * kAccCols) + (uint32_t(quarter * 32) << 16);
-      for (int c = 0; c < NT; c += 16) {
-        uint32_t v[16];
-        asm volatile(
-            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-              "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-            : "r"(tmem_acc + uint32_t(c)) : "memory");
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      // columns are read 48 at a time (three loads in flight, one wait) and go to the owner of
+      // their slice; an owner's base address is mapped once, columns are 512 B apart behind it
+      for (int owner = 0; owner < splits; ++owner) {
+        const int c_lo = owner * slice, c_hi = min(NT, c_lo + slice);
+        const uint32_t local = red_addr + uint32_t(((krank * slice) * kBM + quarter * 32 + lane) * 4);
+        const uint32_t base = splits > 1 ? map_to_rank(local, uint32_t(owner)) : local;
+        for (int c = c_lo; c < c_hi; c += 48) {   // reads past c_hi stay inside the 256-column buffer
+          uint32_t v0[16], v1[16], v2[16];
+          tmem_ld16(tmem_acc + uint32_t(c), v0);
+          if (c + 16 < c_hi) tmem_ld16(tmem_acc + uint32_t(c + 16), v1);
+          if (c + 32 < c_hi) tmem_ld16(tmem_acc + uint32_t(c + 32), v2);
+          tmem_ld_wait();
+          const uint32_t dst = base + uint32_t(c - c_lo) * (kBM * 4);
 #pragma unroll
-        for (int x = 0; x < 16; ++x) {
-          const int j = c + x, owner = j / slice, jj = j - owner * slice;
-          const uint32_t local = red_addr + uint32_t(((krank * slice + jj) * kBM + quarter * 32 + lane) * 4);
-          st_cluster_f32(splits > 1 ? map_to_rank(local, uint32_t(owner)) : local, __uint_as_float(v[x]));
+          for (int x = 0; x < 16; ++x) {
+            if (c + x < c_hi) st_cluster_f32(dst + x * (kBM * 4), __uint_as_float(v0[x]));
+            if (c + 16 + x < c_hi) st_cluster_f32(dst + (16 + x) * (kBM * 4), __uint_as_float(v1[x]));
+            if (c + 32 + x < c_hi) st_cluster_f32(dst + (32 + x) * (kBM * 4), __uint_as_float(v2[x]));
+          }
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -351,20 +391,42 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         if (!ok) break;
       }
       // sum the partial columns this CTA owns (ranks in order) and finish them
-      const int own = min(slice, NT - krank * slice);
-      for (int jj = ew; jj < own; jj += 4) {
-        float4 v = *reinterpret_cast<const float4*>(red + (jj * kBM + 4 * lane));
-        for (int rk = 1; rk < splits; ++rk) {
-          const float4 w = *reinterpret_cast<const float4*>(red + ((rk * slice + jj) * kBM + 4 * lane));
-          v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+      // One group = kBatch columns: all partial columns of the group are read from shared
+      // memory first (independent loads), then summed in rank order and finished.  Warp w takes
+      // groups w, w+4, w+8, ...; the first kPre groups use the operands requested at the top
+      // of the tile loop, later groups ask now.
+      auto finish_group = [&](int jb, const float4 (&g0)[kBatch], const float4 (&g1)[kBatch]) {
+        float4 part[kBatch][4];
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b)
+#pragma unroll
+          for (int rk = 0; rk < 4; ++rk)
+            if (rk < splits && jb + b < own) part[b][rk] = ld_shared_f4(red_addr + uint32_t(((rk * slice + jb + b) * kBM + 4 * lane) * 4));
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) {
+          const int jj = jb + b;
+          if (jj >= own) break;
+          float4 v = part[b][0];
+#pragma unroll
+          for (int rk = 1; rk < 4; ++rk)
+            if (rk < splits) { v.x += part[b][rk].x; v.y += part[b][rk].y; v.z += part[b][rk].z; v.w += part[b][rk].w; }
+          const int j = krank * slice + jj, r = r0 + j;
+          if (r >= e.R_rows) continue;   // the last token tile may overhang the buffers
+          const float rstd = s_rstd[j];
+          if (EPI == EPI_PLAIN) epi_plain(e, r, n0, lane, v, rstd, N);
+          else if (EPI == EPI_RESID) epi_resid(e, r, n0, lane, v, N, wtile, g0[b], gain4);
+          else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, wtile * 64, lane, v, rstd);
+          else epi_qkv(e, r, n0, lane, v, rstd, N, s_pos[j], s_page[j], g0[b], g1[b]);
         }
-        const int j = krank * slice + jj, r = r0 + j;
-        if (r >= e.R_rows) continue;   // the last token tile may overhang the buffers
-        const float rstd = s_rstd[j];
-        if (EPI == EPI_PLAIN) epi_plain(e, r, n0, lane, v, rstd, N);
-        else if (EPI == EPI_RESID) epi_resid(e, r, n0, lane, v, N, wtile);
-        else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, wtile * 64, lane, v, rstd);
-        else epi_qkv(e, r, n0, lane, v, rstd, N, s_pos[j], s_page[j]);
+      };
+#pragma unroll
+      for (int k = 0; k < kPre; ++k)
+        if ((ew + 4 * k) * kBatch < own) finish_group((ew + 4 * k) * kBatch, pg0[k], pg1[k]);
+      for (int jb = (ew + 4 * kPre) * kBatch; jb < own; jb += 4 * kBatch) {
+        float4 g0[kBatch], g1[kBatch];
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) fetch_operands(jb + b, g0[b], g1[b]);
+        finish_group(jb, g0, g1);
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");   // buffer fully read
       if (splits > 1 && et == 0)
@@ -469,6 +531,11 @@ laser_status prepare(GemmState* st) {
   return LASER_OK;
 }
 
+}  // namespace
+// Tuning aid: a non-zero value overrides the modelled choice of the split count.
+int g_force_splits = 0;
+namespace {
+
 // Split count (cluster size) with the least modelled time: clusters work in lock step on one
 // tile each, a tile costs the K blocks of one rank plus a fixed share.
 int pick_splits(const GemmState* st, int R_pad, int N, int K, int epi, int* clusters_out) {
@@ -477,7 +544,7 @@ int pick_splits(const GemmState* st, int R_pad, int N, int K, int epi, int* clus
   int best = 1, best_clusters = 1;
   double best_cost = 1e30;
   for (int s : {1, 2, 4}) {
-    if (st->max_clusters[s] <= 0) continue;
+    if (st->max_clusters[s] <= 0 || (g_force_splits && s != g_force_splits)) continue;
     const int kbps = ceil_div(total_kb, s);
     if (kbps * (s - 1) >= total_kb) continue;  // a rank would have no K blocks
     const int tiles = n_wtiles * tc_shape(R_pad, s).n_ttiles;
