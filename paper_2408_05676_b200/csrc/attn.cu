@@ -44,7 +44,7 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
                   const int32_t* __restrict__ seq_ids, const int32_t* __restrict__ row_ctx,
                   const int32_t* __restrict__ row_n, int Rs, int H, int Hkv,
                   const int32_t* __restrict__ page_table, int pages_per_seq, int layer_row0,
-                  bf16* __restrict__ out, int32_t* __restrict__ status) {
+                  bf16* __restrict__ out, int32_t* __restrict__ status, const void* next_w, size_t next_bytes) {
   constexpr int HALVES = DH / 64;                 // 64-element (128-byte) column blocks per row
   constexpr int SUB = 16 * 128;                   // bytes of one 16-token x 64-element sub-tile
   constexpr int STAGE = 2 * HALVES * SUB;         // K then V
@@ -54,6 +54,10 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
   __shared__ float s_m[kConsumers][16], s_l[kConsumers][16];
   __shared__ int abort_flag;
 
+  // programmatic dependent launch: let the next kernel start its prologue, then wait for the
+  // kernel that produced Q and the new K/V rows
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int b = blockIdx.x, h = blockIdx.y, mt = blockIdx.z;
   const int hk = h / (H / Hkv);
   const int nr = row_n[b], ctx = row_ctx[b];
@@ -114,6 +118,9 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
       }
       if (!ok)
         for (int p = max(0, issued - kStages); p < issued; ++p) mbar_drain(smem_u32(&full_bar[p % kStages]), (p / kStages) & 1);
+      // all pages requested: warm the L2 with the weights of the projection that follows
+      if (ok) prefetch_l2(next_w, next_bytes, blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z),
+                          gridDim.x * gridDim.y * gridDim.z);
     }
     return;
   }
@@ -242,22 +249,31 @@ bool attention_tma_supported(const laser_model* m, const laser_kv* kv) {
 }
 
 laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const int32_t* seq_ids, int B,
-                                  cudaStream_t stream) {
+                                  const void* next_w, size_t next_bytes, cudaStream_t stream) {
   const int dh = m->cfg.head_dim, H = m->cfg.n_heads, Hkv = m->cfg.n_kv_heads, Rs = m->rows_per_seq;
   const int64_t rows_per_layer = int64_t(kv->n_pages) * 2 * Hkv * 16;
   const int layer_row0 = int(rows_per_layer * layer);
   const size_t smem = 1024 + size_t(kStages) * (2 * (dh / 64) * 16 * 128) + size_t(16) * (dh + 8) * 2;
-  dim3 grid(B, H, ceil_div(Rs, 16));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(B), unsigned(H), unsigned(ceil_div(Rs, 16)));
+  cfg.blockDim = dim3(kAttnThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const __nv_bfloat16* q = m->q;
+  const int32_t *rc = m->row_ctx, *rn = m->row_n, *pt = kv->page_table;
   if (dh == 128) {
     LASER_CUDA(cudaFuncSetAttribute(attn_paged_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-    attn_paged_kernel<128><<<grid, kAttnThreads, smem, stream>>>(kv->pages_map, m->q, seq_ids, m->row_ctx, m->row_n, Rs, H,
-                                                                 Hkv, kv->page_table, kv->pages_per_seq, layer_row0,
-                                                                 m->attn, m->status);
+    LASER_CUDA(cudaLaunchKernelEx(&cfg, attn_paged_kernel<128>, kv->pages_map, q, seq_ids, rc, rn, Rs, H, Hkv, pt,
+                                  kv->pages_per_seq, layer_row0, m->attn, m->status, next_w, next_bytes));
   } else {
     LASER_CUDA(cudaFuncSetAttribute(attn_paged_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-    attn_paged_kernel<64><<<grid, kAttnThreads, smem, stream>>>(kv->pages_map, m->q, seq_ids, m->row_ctx, m->row_n, Rs, H,
-                                                                Hkv, kv->page_table, kv->pages_per_seq, layer_row0,
-                                                                m->attn, m->status);
+    LASER_CUDA(cudaLaunchKernelEx(&cfg, attn_paged_kernel<64>, kv->pages_map, q, seq_ids, rc, rn, Rs, H, Hkv, pt,
+                                  kv->pages_per_seq, layer_row0, m->attn, m->status, next_w, next_bytes));
   }
   count_launch();
   LASER_CUDA(cudaGetLastError());

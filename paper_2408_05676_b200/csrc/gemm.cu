@@ -224,6 +224,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const int nkb = max(0, min(kb_per_split, total_kb - kb0));
   constexpr int kAccCols = 256;                             // TMEM columns per accumulator buffer
 
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its prologue
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
@@ -246,27 +247,46 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 
   if (warp == 0) {
     if (lane == 0) {  // ---- TMA producer ----
-      int it = 0;
+      // Flat iteration space: `it` walks the K blocks of this CTA's tiles in order.
+      const int my_tiles = cluster_id < n_tiles ? (n_tiles - cluster_id + n_clusters - 1) / n_clusters : 0;
+      const int total_it = my_tiles * nkb;
+      auto load_w = [&](int it) {
+        const int ti = it / nkb, kb = it - ti * nkb, wtile = (cluster_id + ti * n_clusters) / n_ttiles;
+        const int s = it % stages, k = (kb0 + kb) * kBK;
+        const uint32_t dst = tiles + uint32_t(s) * stage_bytes, bar = smem_u32(&full_bar[s]);
+        tma_load_2d(dst, &tmW, k, EPI == EPI_SWIGLU ? wtile * 64 : wtile * kBM, bar);
+        tma_load_2d(dst + w_bytes / 2, &tmW, k, EPI == EPI_SWIGLU ? e.f + wtile * 64 : wtile * kBM + 64, bar);
+      };
+      auto load_a = [&](int it) {
+        const int ti = it / nkb, kb = it - ti * nkb, ttile = (cluster_id + ti * n_clusters) % n_ttiles;
+        const int s = it % stages;
+        tma_load_2d(tiles + uint32_t(s) * stage_bytes + w_bytes, &tmA, (kb0 + kb) * kBK, ttile * NT,
+                    smem_u32(&full_bar[s]));
+      };
+      // The weights do not depend on the kernel before this one: fill the ring with weight
+      // tiles first, and only then wait for the previous kernel's results (the activations).
+      const int pre = min(stages, total_it);
+      for (int it = 0; it < pre; ++it) { mbar_expect_tx(smem_u32(&full_bar[it % stages]), stage_bytes); load_w(it); }
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      for (int it = 0; it < pre; ++it) load_a(it);
       bool ok = true;
-      for (int t = cluster_id; t < n_tiles && ok; t += n_clusters) {
-        const int ttile = t % n_ttiles, wtile = t / n_ttiles;
-        const int wrow0 = EPI == EPI_SWIGLU ? wtile * 64 : wtile * kBM;
-        const int wrow1 = EPI == EPI_SWIGLU ? e.f + wtile * 64 : wtile * kBM + 64;
-        for (int kb = 0; kb < nkb; ++kb, ++it) {
-          const int s = it % stages;
-          if (it >= stages) ok = mbar_wait(smem_u32(&empty_bar[s]), ((it / stages) - 1) & 1, &abort_flag);
-          if (!ok) break;
-          const uint32_t bar = smem_u32(&full_bar[s]);
-          const uint32_t dst = tiles + uint32_t(s) * stage_bytes;
-          mbar_expect_tx(bar, stage_bytes);
-          const int k = (kb0 + kb) * kBK;
-          tma_load_2d(dst, &tmW, k, wrow0, bar);
-          tma_load_2d(dst + w_bytes / 2, &tmW, k, wrow1, bar);
-          tma_load_2d(dst + w_bytes, &tmA, k, ttile * NT, bar);
-        }
+      int it = pre;
+      for (; it < total_it; ++it) {
+        const int s = it % stages;
+        ok = mbar_wait(smem_u32(&empty_bar[s]), ((it / stages) - 1) & 1, &abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(smem_u32(&full_bar[s]), stage_bytes);
+        load_w(it);
+        load_a(it);
       }
       if (!ok)  // drain copies still in flight before the CTA may exit
         for (int j = max(0, it - stages); j < it; ++j) mbar_drain(smem_u32(&full_bar[j % stages]), (j / stages) & 1);
+      // Warm the L2 with the head of the next kernel's weights: HBM would otherwise idle while
+      // the last epilogue, the exit and the next kernel's start-up run.
+      if (ok) {
+        prefetch_l2(e.next_w, e.next_bytes, blockIdx.x, gridDim.x);
+        prefetch_l2(e.next_w2, e.next_bytes2, blockIdx.x, gridDim.x);
+      }
     }
   } else if (warp == 1) {
     if (lane == 0) {  // ---- MMA issuer ----
@@ -296,6 +316,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
   } else {
     // ---- epilogue warps ----
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // everything below reads or overwrites earlier results
     const int et = threadIdx.x - 64, ew = warp - 2;
     const int quarter = warp & 3;  // a warp may only touch its own 32 TMEM lanes
     int i = 0, cur_ttile = -1;
@@ -439,7 +460,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   if (warp == 1) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * kAccCols) : "memory");
   }
-  if (threadIdx.x == 0 && abort_flag) atomicCAS(status, 0, LASER_ERR_TIMEOUT);
+  if (threadIdx.x == 0 && abort_flag) {
+    atomicCAS(status, 0, LASER_ERR_TIMEOUT);
+  }
 }
 
 // ---- host side --------------------------------------------------------------------------
@@ -491,8 +514,12 @@ void fill_launch(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int grid, i
   attr[0].val.clusterDim.x = unsigned(splits);
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // programmatic dependent launch: this kernel may begin while the previous one drains; it
+  // orders itself with griddepcontrol.wait
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg->attrs = attr;
-  cfg->numAttrs = 1;
+  cfg->numAttrs = 2;
 }
 
 template <int EPI>
@@ -500,7 +527,7 @@ laser_status launch_epi(const CUtensorMap& tw, const CUtensorMap& ta, const Gemm
                         int n_wtiles, int total_kb, int kbps, int splits, int clusters, int32_t* status,
                         cudaStream_t stream) {
   cudaLaunchConfig_t cfg;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   fill_launch<EPI>(&cfg, attr, clusters * splits, splits, sh.smem, stream);
   LASER_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI>, tw, ta, e, N, sh.NT, sh.n_ttiles, n_wtiles, total_kb, kbps,
                                 splits, sh.stages, status));
@@ -519,7 +546,7 @@ laser_status prepare(GemmState* st) {
   LASER_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   for (int s : {1, 2, 4}) {
     cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     fill_launch<EPI_RESID>(&cfg, attr, (sms / s) * s, s, size_t(kSmemLimit) - 8192, nullptr);
     int n = 0;
     cudaError_t err = cudaOccupancyMaxActiveClusters(&n, gemm_tc_kernel<EPI_RESID>, &cfg);

@@ -15,6 +15,8 @@ namespace {
 
 using bf16 = __nv_bfloat16;
 
+constexpr size_t kL2PrefetchBytes = size_t(48) << 20;
+
 // ---- row bookkeeping -------------------------------------------------------------------
 // One thread per row: position, cache slot, capacity check, rotary angles (fp64 -> fp32).
 __global__ void prep_rows_kernel(const int32_t* __restrict__ seq_ids, const int32_t* __restrict__ n_rows,
@@ -451,6 +453,8 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
     LASER_CUDA(cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(attn_smem)));
   }
   const int d_tiles = ceil_div(d, 128);
+  // bytes of a following weight matrix worth prefetching into L2 while a kernel drains
+  auto head_bytes = [](size_t bytes) { return std::min<size_t>(bytes, kL2PrefetchBytes) & ~size_t(16383); };
   GemmEpilogue base;
   base.R_rows = m->R_pad;
   base.sumsq_ld = m->R_pad;
@@ -471,7 +475,7 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
     {
       ProfScope ps(m, 1, stream);
       if (use_tma_attn) {
-        LASER_TRY(attention_tma_launch(m, kv, l, seq_ids, B, stream));
+        LASER_TRY(attention_tma_launch(m, kv, l, seq_ids, B, m->wo[l], head_bytes(size_t(d) * m->dq * 2), stream));
       } else {
         attention_kernel<<<dim3(B, H), 128, attn_smem, stream>>>(m->q, seq_ids, m->row_ctx, m->row_n, Rs, H, Hkv, dh,
                                                                 kv->page_table, kv->pages_per_seq, pages_l,
@@ -482,6 +486,8 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
     {  // output projection; residual add; operand and statistics of the FFN norm
       GemmEpilogue e = base;
       e.resid = m->resid; e.xb = m->xn; e.gain_next = m->ffn_norm[l]; e.sumsq_out = m->sumsq;
+      e.next_w = m->wgu[l]; e.next_bytes = head_bytes(size_t(f) * d * 2) / 2;          // gate rows
+      e.next_w2 = m->wgu[l] + size_t(f) * d; e.next_bytes2 = e.next_bytes;             // up rows
       ProfScope ps(m, 0, stream);
       LASER_TRY(gemm_fused(m, m->attn, m->wo[l], Rp, d, m->dq, EPI_RESID, e, stream));
     }
@@ -489,6 +495,7 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
       GemmEpilogue e = base;
       e.sumsq_in = m->sumsq; e.sumsq_in_tiles = d_tiles;
       e.act = m->act; e.f = f;
+      e.next_w = m->wdown[l]; e.next_bytes = head_bytes(size_t(d) * f * 2);
       ProfScope ps(m, 0, stream);
       LASER_TRY(gemm_fused(m, m->xn, m->wgu[l], Rp, 2 * f, d, EPI_SWIGLU, e, stream));
     }
@@ -496,6 +503,8 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
       GemmEpilogue e = base;
       e.resid = m->resid; e.xb = m->xn; e.sumsq_out = m->sumsq;
       e.gain_next = l + 1 < c.n_layers ? m->attn_norm[l + 1] : m->final_norm;
+      e.next_w = l + 1 < c.n_layers ? m->wqkv[l + 1] : m->lm_head;
+      e.next_bytes = head_bytes(l + 1 < c.n_layers ? size_t(m->dqkv) * d * 2 : size_t(c.vocab) * d * 2);
       ProfScope ps(m, 0, stream);
       LASER_TRY(gemm_fused(m, m->act, m->wdown[l], Rp, d, f, EPI_RESID, e, stream));
     }

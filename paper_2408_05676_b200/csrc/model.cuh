@@ -40,6 +40,12 @@ enum { EPI_PLAIN = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_QKV = 3 };
 
 struct GemmEpilogue {
   int R_rows = 0;                    // rows the activation / output buffers really have
+  // weights of the kernel that follows (head of the matrix, multiple of 16 KB): prefetched
+  // into L2 once this kernel has issued its own loads; null = nothing
+  const void* next_w = nullptr;
+  size_t next_bytes = 0;
+  const void* next_w2 = nullptr;     // second region (the up half of a gate/up matrix)
+  size_t next_bytes2 = 0;
   // RMSNorm of the A operand, applied as a per-row scale of the result: the producer left
   // x * gain in bf16 and one sum of squares per (128-feature tile, row); null = no scale
   const float* sumsq_in = nullptr;
@@ -78,6 +84,6 @@ void gemm_state_free(laser_model* m);
 // coordinates); the verify forward falls back to a plain kernel otherwise.
 bool attention_tma_supported(const laser_model* m, const laser_kv* kv);
 laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const int32_t* seq_ids, int B,
-                                  cudaStream_t stream);
+                                  const void* next_w, size_t next_bytes, cudaStream_t stream);
 
 }  // namespace laser

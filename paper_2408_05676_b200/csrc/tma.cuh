@@ -56,6 +56,15 @@ __device__ __forceinline__ void tma_prefetch_map(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
 
+// L2 prefetch of [ptr, ptr + bytes) in 16 KB pieces, piece c taken by worker c % n_workers.
+// `ptr` must be 16-byte aligned; a tail shorter than one piece is left out.
+__device__ __forceinline__ void prefetch_l2(const void* ptr, size_t bytes, unsigned worker, unsigned n_workers) {
+  if (ptr == nullptr) return;
+  const size_t chunk = 16384, n_chunks = bytes / chunk;
+  for (size_t c = worker; c < n_chunks; c += n_workers)
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(static_cast<const char*>(ptr) + c * chunk), "r"(uint32_t(chunk)) : "memory");
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
