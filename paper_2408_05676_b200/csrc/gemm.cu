@@ -8,21 +8,21 @@
 // 128-wide M side of tcgen05.mma and the token rows the N side (NT <= 192, no padding of the
 // rows to 128); the accumulator is a 128 x NT fp32 tile in tensor memory.
 //
-// Persistent kernel, one CTA per SM, CTAs grouped in thread-block clusters of `splits` along K.
-// A cluster walks the output tiles assigned to it; each of its CTAs contracts its own K range
-// of the tile.  Roles inside a CTA:
+// One CTA per (token tile, weight tile, K range); the CTAs that share an output tile form a
+// thread-block cluster along K.  Two CTAs fit on an SM and kernels are chained with
+// programmatic dependent launch, so while one CTA runs its epilogue, exits, or a CTA of the
+// next kernel starts up in its place, the other CTA of the SM keeps streaming weights.
 //   warp 0     TMA producer: weight and activation tiles (128-byte swizzle) into a ring of
-//              shared-memory stages, running ahead across tile boundaries;
-//   warp 1     MMA issuer: tcgen05.mma into one of two TMEM accumulators, tcgen05.commit frees
-//              stages and publishes finished accumulators;
-//   warps 2-5  epilogue: read the accumulator (tcgen05.ld), send every token column to the
-//              CTA of the cluster that owns it (distributed shared memory), then sum the
-//              `splits` partial columns they own in rank order (run-to-run identical, no
-//              partial sums in global memory) and apply the fused epilogue.
-// The epilogue of tile i overlaps the main loop of tile i+1 (double-buffered accumulator);
-// cross-CTA hand-over uses cluster-scope mbarriers.  Every wait is bounded: on expiry the CTA
-// records LASER_ERR_TIMEOUT, stops issuing work, still joins the final cluster barrier, frees
-// its tensor memory and exits.
+//              shared-memory stages; weight tiles are requested before the dependency wait,
+//              since they do not depend on the previous kernel;
+//   warp 1     MMA issuer: tcgen05.mma into a TMEM accumulator, tcgen05.commit frees stages;
+//   warps 2-5  epilogue: move the finished accumulator to shared memory (the free stages),
+//              then, after a cluster barrier, sum the partial tiles of the cluster through
+//              distributed shared memory in rank order (run-to-run identical, no partial sums
+//              in global memory) for the token columns this CTA owns and apply the fused
+//              epilogue, whose global operands were requested at kernel start.
+// Every mbarrier wait is bounded: on expiry the CTA records LASER_ERR_TIMEOUT, drains its
+// copies, still joins the cluster barriers, frees its tensor memory and exits.
 #include <map>
 #include <tuple>
 
@@ -38,7 +38,7 @@ constexpr int kBM = 128;          // weight rows per tile (MMA M)
 constexpr int kBK = 64;           // K elements per stage = one 128-byte swizzle span of bf16
 constexpr int kMaxStages = 6;
 constexpr int kMaxNT = 192;       // token rows per tile: accumulator staging must fit shared memory
-constexpr int kSmemLimit = 222 * 1024;   // dynamic shared memory one CTA may ask for
+constexpr int kSmemBudget = 110 * 1024;  // shared memory of one CTA: two CTAs per SM
 constexpr int kBatch = 3, kPre = 3;      // epilogue: columns per group, groups whose operands are prefetched
 
 // Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows 128 B apart, groups
@@ -101,10 +101,13 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
       : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ float4 ld_shared_f4(uint32_t addr) {
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t cluster_addr) {
   float4 v;
-  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr));
   return v;
+}
+__device__ __forceinline__ void st_shared_f32(uint32_t addr, float v) {
+  asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v));
 }
 // AND of a flag over the 128 epilogue threads (named barrier 1), so that they leave a loop together.
 __device__ __forceinline__ bool epilogue_all(bool ok) {
@@ -199,270 +202,229 @@ __device__ __forceinline__ void epi_qkv(const GemmEpilogue& e, int r, int n0, in
 
 
 template <int EPI>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, const GemmEpilogue e,
-               int N, int NT, int n_ttiles, int n_wtiles, int total_kb, int kb_per_split, int splits, int stages,
+               int N, int NT, int total_kb, int kb_per_split, int splits, int stages, int tmem_cols,
                int32_t* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages];
-  __shared__ uint64_t acc_full[2], acc_empty[2];   // TMEM accumulator hand-over MMA <-> epilogue
-  __shared__ uint64_t red_full, red_free;          // reduction buffer hand-over between cluster peers
+  __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_bar;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   __shared__ float s_rstd[kMaxNT];
   __shared__ int s_pos[kMaxNT], s_page[kMaxNT];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its prologue
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
   const uint32_t w_bytes = kBM * 128, a_bytes = uint32_t(NT) * 128, stage_bytes = w_bytes + a_bytes;
-  const int slice = (NT + splits - 1) / splits;            // token columns owned by one CTA of the cluster
-  const uint32_t red_addr = tiles + uint32_t(stages) * stage_bytes;   // [splits][slice][128] fp32
-  const float* red = reinterpret_cast<const float*>(smem_raw + (red_addr - raw));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int krank = blockIdx.x % splits, cluster_id = blockIdx.x / splits, n_clusters = gridDim.x / splits;
-  const int n_tiles = n_ttiles * n_wtiles;
+  const int krank = blockIdx.x % splits, ttile = blockIdx.x / splits, wtile = blockIdx.y;
+  const int r0 = ttile * NT, n0 = wtile * kBM;
   const int kb0 = krank * kb_per_split;
   const int nkb = max(0, min(kb_per_split, total_kb - kb0));
-  constexpr int kAccCols = 256;                             // TMEM columns per accumulator buffer
+  const int slice = (NT + splits - 1) / splits;            // token columns finished by one CTA of the cluster
+  const int own = max(0, min(slice, NT - krank * slice));
 
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its prologue
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&acc_full[b]), 1); mbar_init(smem_u32(&acc_empty[b]), 1); }
-    mbar_init(smem_u32(&red_full), uint32_t(splits));
-    mbar_init(smem_u32(&red_free), uint32_t(splits));
+    mbar_init(smem_u32(&acc_bar), 1);
     mbar_fence_init();
     tma_prefetch_map(&tmW);
     tma_prefetch_map(&tmA);
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(2 * kAccCols) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(tmem_cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (splits > 1) cluster_sync_all();   // peers' barriers exist before anyone arrives on them
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_base = tmem_slot;
+  const uint32_t tmem_acc = tmem_slot;
+
+  // epilogue operands live in registers of warps 2-5 from kernel start to the epilogue
+  const int ew = warp - 2, nfeat = n0 + 4 * lane;
+  uint2 gain4 = make_uint2(0u, 0u);
+  float4 pg0[kPre][kBatch], pg1[kPre][kBatch];
+  auto fetch_operands = [&](int jj, float4& g0, float4& g1) {
+    g0 = make_float4(0.f, 0.f, 0.f, 0.f); g1 = g0;
+    const int r = r0 + krank * slice + jj;
+    if (jj < own && r < e.R_rows && nfeat < N) {
+      if (EPI == EPI_RESID) g0 = *reinterpret_cast<const float4*>(e.resid + size_t(r) * N + nfeat);
+      if (EPI == EPI_QKV && nfeat < (e.H + e.Hkv) * e.dh) {
+        const float* cs = e.rope + (size_t(r) * (e.dh >> 1) + (nfeat % e.dh) % (e.dh >> 1)) * 2;
+        g0 = *reinterpret_cast<const float4*>(cs);       // c0 s0 c1 s1
+        g1 = *reinterpret_cast<const float4*>(cs + 4);   // c2 s2 c3 s3
+      }
+    }
+  };
 
   if (warp == 0) {
     if (lane == 0) {  // ---- TMA producer ----
-      // Flat iteration space: `it` walks the K blocks of this CTA's tiles in order.
-      const int my_tiles = cluster_id < n_tiles ? (n_tiles - cluster_id + n_clusters - 1) / n_clusters : 0;
-      const int total_it = my_tiles * nkb;
-      auto load_w = [&](int it) {
-        const int ti = it / nkb, kb = it - ti * nkb, wtile = (cluster_id + ti * n_clusters) / n_ttiles;
-        const int s = it % stages, k = (kb0 + kb) * kBK;
+      auto load_w = [&](int kb) {
+        const int s = kb % stages, k = (kb0 + kb) * kBK;
         const uint32_t dst = tiles + uint32_t(s) * stage_bytes, bar = smem_u32(&full_bar[s]);
-        tma_load_2d(dst, &tmW, k, EPI == EPI_SWIGLU ? wtile * 64 : wtile * kBM, bar);
-        tma_load_2d(dst + w_bytes / 2, &tmW, k, EPI == EPI_SWIGLU ? e.f + wtile * 64 : wtile * kBM + 64, bar);
+        tma_load_2d(dst, &tmW, k, EPI == EPI_SWIGLU ? wtile * 64 : n0, bar);
+        tma_load_2d(dst + w_bytes / 2, &tmW, k, EPI == EPI_SWIGLU ? e.f + wtile * 64 : n0 + 64, bar);
       };
-      auto load_a = [&](int it) {
-        const int ti = it / nkb, kb = it - ti * nkb, ttile = (cluster_id + ti * n_clusters) % n_ttiles;
-        const int s = it % stages;
-        tma_load_2d(tiles + uint32_t(s) * stage_bytes + w_bytes, &tmA, (kb0 + kb) * kBK, ttile * NT,
-                    smem_u32(&full_bar[s]));
+      auto load_a = [&](int kb) {
+        const int s = kb % stages;
+        tma_load_2d(tiles + uint32_t(s) * stage_bytes + w_bytes, &tmA, (kb0 + kb) * kBK, r0, smem_u32(&full_bar[s]));
       };
       // The weights do not depend on the kernel before this one: fill the ring with weight
       // tiles first, and only then wait for the previous kernel's results (the activations).
-      const int pre = min(stages, total_it);
-      for (int it = 0; it < pre; ++it) { mbar_expect_tx(smem_u32(&full_bar[it % stages]), stage_bytes); load_w(it); }
+      const int pre = min(stages, nkb);
+      for (int kb = 0; kb < pre; ++kb) { mbar_expect_tx(smem_u32(&full_bar[kb % stages]), stage_bytes); load_w(kb); }
       asm volatile("griddepcontrol.wait;" ::: "memory");
-      for (int it = 0; it < pre; ++it) load_a(it);
+      for (int kb = 0; kb < pre; ++kb) load_a(kb);
       bool ok = true;
-      int it = pre;
-      for (; it < total_it; ++it) {
-        const int s = it % stages;
-        ok = mbar_wait(smem_u32(&empty_bar[s]), ((it / stages) - 1) & 1, &abort_flag);
+      int kb = pre;
+      for (; kb < nkb; ++kb) {
+        const int s = kb % stages;
+        ok = mbar_wait(smem_u32(&empty_bar[s]), ((kb / stages) - 1) & 1, &abort_flag);
         if (!ok) break;
         mbar_expect_tx(smem_u32(&full_bar[s]), stage_bytes);
-        load_w(it);
-        load_a(it);
+        load_w(kb);
+        load_a(kb);
       }
       if (!ok)  // drain copies still in flight before the CTA may exit
-        for (int j = max(0, it - stages); j < it; ++j) mbar_drain(smem_u32(&full_bar[j % stages]), (j / stages) & 1);
-      // Warm the L2 with the head of the next kernel's weights: HBM would otherwise idle while
-      // the last epilogue, the exit and the next kernel's start-up run.
-      if (ok) {
-        prefetch_l2(e.next_w, e.next_bytes, blockIdx.x, gridDim.x);
-        prefetch_l2(e.next_w2, e.next_bytes2, blockIdx.x, gridDim.x);
-      }
+        for (int j = max(0, kb - stages); j < kb; ++j) mbar_drain(smem_u32(&full_bar[j % stages]), (j / stages) & 1);
     }
   } else if (warp == 1) {
     if (lane == 0) {  // ---- MMA issuer ----
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(NT >> 3) << 17) | (uint32_t(kBM >> 4) << 24);
-      int it = 0, i = 0;
       bool ok = true;
-      for (int t = cluster_id; t < n_tiles && ok; t += n_clusters, ++i) {
-        const int buf = i & 1;
-        if (i >= 2) ok = mbar_wait(smem_u32(&acc_empty[buf]), ((i >> 1) - 1) & 1, &abort_flag);
+      for (int kb = 0; kb < nkb && ok; ++kb) {
+        const int s = kb % stages;
+        ok = mbar_wait(smem_u32(&full_bar[s]), (kb / stages) & 1, &abort_flag);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t tmem_acc = tmem_base + uint32_t(buf * kAccCols);
-        for (int kb = 0; kb < nkb; ++kb, ++it) {
-          const int s = it % stages;
-          ok = mbar_wait(smem_u32(&full_bar[s]), (it / stages) & 1, &abort_flag);
-          if (!ok) break;
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t w_addr = tiles + uint32_t(s) * stage_bytes;
-          const uint64_t wdesc = umma_desc(w_addr), adesc = umma_desc(w_addr + w_bytes);
+        const uint32_t w_addr = tiles + uint32_t(s) * stage_bytes;
+        const uint64_t wdesc = umma_desc(w_addr), adesc = umma_desc(w_addr + w_bytes);
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k)  // 16 bf16 = 32 bytes further along K inside the swizzle span
-            umma_bf16(tmem_acc, wdesc + uint64_t(k * 2), adesc + uint64_t(k * 2), idesc, (kb | k) != 0);
-          umma_commit(smem_u32(&empty_bar[s]));
-        }
-        if (ok) umma_commit(smem_u32(&acc_full[buf]));  // arrives when the tile's MMAs have finished
+        for (int k = 0; k < kBK / 16; ++k)  // 16 bf16 = 32 bytes further along K inside the swizzle span
+          umma_bf16(tmem_acc, wdesc + uint64_t(k * 2), adesc + uint64_t(k * 2), idesc, (kb | k) != 0);
+        umma_commit(smem_u32(&empty_bar[s]));
       }
+      umma_commit(smem_u32(&acc_bar));  // arrives when every MMA issued so far has finished
     }
   } else {
-    // ---- epilogue warps ----
-    asm volatile("griddepcontrol.wait;" ::: "memory");   // everything below reads or overwrites earlier results
-    const int et = threadIdx.x - 64, ew = warp - 2;
+    // ---- epilogue warps, part 1: everything that can be done before the accumulator is ready ----
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // what follows reads earlier kernels' results
+    for (int j = threadIdx.x - 64; j < NT; j += 128) {   // per-row scale and cache coordinates
+      const int r = r0 + j;
+      float rstd = 1.f;
+      int pos = -1, page = 0;
+      if (r < e.R_rows) {
+        if (e.sumsq_in) {
+          float ss = 0.f;
+          for (int tt = 0; tt < e.sumsq_in_tiles; ++tt) ss += e.sumsq_in[size_t(tt) * e.sumsq_ld + r];
+          rstd = rsqrtf(ss * e.inv_d + e.eps);
+        }
+        if (EPI == EPI_QKV) {
+          pos = e.row_pos[r];
+          if (pos >= 0) page = e.page_table[size_t(e.row_seq[r]) * e.pages_per_seq + (pos >> 4)];
+        }
+      }
+      s_rstd[j] = rstd; s_pos[j] = pos; s_page[j] = page;
+    }
+    if (EPI == EPI_RESID && nfeat < N) gain4 = *reinterpret_cast<const uint2*>(e.gain_next + nfeat);
+#pragma unroll
+    for (int k = 0; k < kPre; ++k)
+#pragma unroll
+      for (int b = 0; b < kBatch; ++b) fetch_operands((ew + 4 * k) * kBatch + b, pg0[k][b], pg1[k][b]);
+    // part 2: accumulator from tensor memory to shared memory, token-major [NT][128]
     const int quarter = warp & 3;  // a warp may only touch its own 32 TMEM lanes
-    int i = 0, cur_ttile = -1;
-    bool ok = true;
-    for (int t = cluster_id; t < n_tiles && ok; t += n_clusters, ++i) {
-      const int ttile = t % n_ttiles, wtile = t / n_ttiles, buf = i & 1;
-      const int r0 = ttile * NT, n0 = wtile * kBM;
-      // Global operands of the fused epilogue (residual, rotary table, gains) do not depend on
-      // this kernel: ask for the first groups now, long before the accumulator is ready.
-      const int own = min(slice, NT - krank * slice);
-      const int nfeat = n0 + 4 * lane;
-      auto fetch_operands = [&](int jj, float4& g0, float4& g1) {
-        g0 = make_float4(0.f, 0.f, 0.f, 0.f); g1 = g0;
-        const int r = r0 + krank * slice + jj;
-        if (jj < own && r < e.R_rows && nfeat < N) {
-          if (EPI == EPI_RESID) g0 = *reinterpret_cast<const float4*>(e.resid + size_t(r) * N + nfeat);
-          if (EPI == EPI_QKV && nfeat < (e.H + e.Hkv) * e.dh) {
-            const float* cs = e.rope + (size_t(r) * (e.dh >> 1) + (nfeat % e.dh) % (e.dh >> 1)) * 2;
-            g0 = *reinterpret_cast<const float4*>(cs);       // c0 s0 c1 s1
-            g1 = *reinterpret_cast<const float4*>(cs + 4);   // c2 s2 c3 s3
-          }
-        }
-      };
-      uint2 gain4 = make_uint2(0u, 0u);   // gains of this lane's four features (next norm)
-      if (EPI == EPI_RESID && nfeat < N) gain4 = *reinterpret_cast<const uint2*>(e.gain_next + nfeat);
-      float4 pg0[kPre][kBatch], pg1[kPre][kBatch];
+    const bool ok = mbar_wait(smem_u32(&acc_bar), 0, &abort_flag);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t src = tmem_acc + (uint32_t(quarter * 32) << 16);
+    const uint32_t dst0 = tiles + uint32_t((quarter * 32 + lane) * 4);
+    for (int c = 0; c < NT; c += 48) {   // three loads in flight, one wait; reads past NT stay inside the allocation
+      uint32_t v0[16], v1[16], v2[16];
+      if (ok && nkb > 0) {
+        tmem_ld16(src + uint32_t(c), v0);
+        if (c + 16 < NT) tmem_ld16(src + uint32_t(c + 16), v1);
+        if (c + 32 < NT) tmem_ld16(src + uint32_t(c + 32), v2);
+        tmem_ld_wait();
+      } else {
 #pragma unroll
-      for (int k = 0; k < kPre; ++k)
-#pragma unroll
-        for (int b = 0; b < kBatch; ++b) fetch_operands((ew + 4 * k) * kBatch + b, pg0[k][b], pg1[k][b]);
-      if (ttile != cur_ttile) {  // per-row scale and cache coordinates of this token tile
-        cur_ttile = ttile;
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        for (int j = et; j < NT; j += 128) {
-          const int r = r0 + j;
-          float rstd = 1.f;
-          int pos = -1, page = 0;
-          if (r < e.R_rows) {
-            if (e.sumsq_in) {
-              float ss = 0.f;
-              for (int tt = 0; tt < e.sumsq_in_tiles; ++tt) ss += e.sumsq_in[size_t(tt) * e.sumsq_ld + r];
-              rstd = rsqrtf(ss * e.inv_d + e.eps);
-            }
-            if (EPI == EPI_QKV) {
-              pos = e.row_pos[r];
-              if (pos >= 0) page = e.page_table[size_t(e.row_seq[r]) * e.pages_per_seq + (pos >> 4)];
-            }
-          }
-          s_rstd[j] = rstd; s_pos[j] = pos; s_page[j] = page;
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        for (int x = 0; x < 16; ++x) v0[x] = v1[x] = v2[x] = 0u;
       }
-      ok = mbar_wait(smem_u32(&acc_full[buf]), (i >> 1) & 1, &abort_flag);
-      // the owners must have finished summing the previous tile before their buffers are overwritten
-      if (ok && splits > 1 && i >= 1) ok = mbar_wait_cluster(smem_u32(&red_free), (i - 1) & 1, &abort_flag);
-      ok = epilogue_all(ok);
-      if (!ok) break;
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      // send every token column of this partial tile to its owner: [rank][column][128 features]
-      const uint32_t tmem_acc = tmem_base + uint32_t(buf * kAccCols) + (uint32_t(quarter * 32) << 16);
-      // columns are read 48 at a time (three loads in flight, one wait) and go to the owner of
-      // their slice; an owner's base address is mapped once, columns are 512 B apart behind it
-      for (int owner = 0; owner < splits; ++owner) {
-        const int c_lo = owner * slice, c_hi = min(NT, c_lo + slice);
-        const uint32_t local = red_addr + uint32_t(((krank * slice) * kBM + quarter * 32 + lane) * 4);
-        const uint32_t base = splits > 1 ? map_to_rank(local, uint32_t(owner)) : local;
-        for (int c = c_lo; c < c_hi; c += 48) {   // reads past c_hi stay inside the 256-column buffer
-          uint32_t v0[16], v1[16], v2[16];
-          tmem_ld16(tmem_acc + uint32_t(c), v0);
-          if (c + 16 < c_hi) tmem_ld16(tmem_acc + uint32_t(c + 16), v1);
-          if (c + 32 < c_hi) tmem_ld16(tmem_acc + uint32_t(c + 32), v2);
-          tmem_ld_wait();
-          const uint32_t dst = base + uint32_t(c - c_lo) * (kBM * 4);
+      const uint32_t dst = dst0 + uint32_t(c) * (kBM * 4);
 #pragma unroll
-          for (int x = 0; x < 16; ++x) {
-            if (c + x < c_hi) st_cluster_f32(dst + x * (kBM * 4), __uint_as_float(v0[x]));
-            if (c + 16 + x < c_hi) st_cluster_f32(dst + (16 + x) * (kBM * 4), __uint_as_float(v1[x]));
-            if (c + 32 + x < c_hi) st_cluster_f32(dst + (32 + x) * (kBM * 4), __uint_as_float(v2[x]));
-          }
-        }
+      for (int x = 0; x < 16; ++x) {
+        if (c + x < NT) st_shared_f32(dst + x * (kBM * 4), __uint_as_float(v0[x]));
+        if (c + 16 + x < NT) st_shared_f32(dst + (16 + x) * (kBM * 4), __uint_as_float(v1[x]));
+        if (c + 32 + x < NT) st_shared_f32(dst + (32 + x) * (kBM * 4), __uint_as_float(v2[x]));
       }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (et == 0) {
-        mbar_arrive(smem_u32(&acc_empty[buf]));   // the accumulator may be overwritten
-        if (splits > 1) {
-          asm volatile("fence.acq_rel.cluster;" ::: "memory");
-          for (int rk = 0; rk < splits; ++rk) mbar_arrive_cluster(map_to_rank(smem_u32(&red_full), uint32_t(rk)));
-        }
-      }
-      if (splits > 1) {
-        ok = epilogue_all(mbar_wait_cluster(smem_u32(&red_full), i & 1, &abort_flag));
-        if (!ok) break;
-      }
-      // sum the partial columns this CTA owns (ranks in order) and finish them
-      // One group = kBatch columns: all partial columns of the group are read from shared
-      // memory first (independent loads), then summed in rank order and finished.  Warp w takes
-      // groups w, w+4, w+8, ...; the first kPre groups use the operands requested at the top
-      // of the tile loop, later groups ask now.
-      auto finish_group = [&](int jb, const float4 (&g0)[kBatch], const float4 (&g1)[kBatch]) {
-        float4 part[kBatch][4];
-#pragma unroll
-        for (int b = 0; b < kBatch; ++b)
-#pragma unroll
-          for (int rk = 0; rk < 4; ++rk)
-            if (rk < splits && jb + b < own) part[b][rk] = ld_shared_f4(red_addr + uint32_t(((rk * slice + jb + b) * kBM + 4 * lane) * 4));
-#pragma unroll
-        for (int b = 0; b < kBatch; ++b) {
-          const int jj = jb + b;
-          if (jj >= own) break;
-          float4 v = part[b][0];
-#pragma unroll
-          for (int rk = 1; rk < 4; ++rk)
-            if (rk < splits) { v.x += part[b][rk].x; v.y += part[b][rk].y; v.z += part[b][rk].z; v.w += part[b][rk].w; }
-          const int j = krank * slice + jj, r = r0 + j;
-          if (r >= e.R_rows) continue;   // the last token tile may overhang the buffers
-          const float rstd = s_rstd[j];
-          if (EPI == EPI_PLAIN) epi_plain(e, r, n0, lane, v, rstd, N);
-          else if (EPI == EPI_RESID) epi_resid(e, r, n0, lane, v, N, wtile, g0[b], gain4);
-          else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, wtile * 64, lane, v, rstd);
-          else epi_qkv(e, r, n0, lane, v, rstd, N, s_pos[j], s_page[j], g0[b], g1[b]);
-        }
-      };
-#pragma unroll
-      for (int k = 0; k < kPre; ++k)
-        if ((ew + 4 * k) * kBatch < own) finish_group((ew + 4 * k) * kBatch, pg0[k], pg1[k]);
-      for (int jb = (ew + 4 * kPre) * kBatch; jb < own; jb += 4 * kBatch) {
-        float4 g0[kBatch], g1[kBatch];
-#pragma unroll
-        for (int b = 0; b < kBatch; ++b) fetch_operands(jb + b, g0[b], g1[b]);
-        finish_group(jb, g0, g1);
-      }
-      asm volatile("bar.sync 1, 128;" ::: "memory");   // buffer fully read
-      if (splits > 1 && et == 0)
-        for (int rk = 0; rk < splits; ++rk) mbar_arrive_cluster(map_to_rank(smem_u32(&red_free), uint32_t(rk)));
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (splits > 1) cluster_sync_all();  // nobody leaves while a peer may still write to it
+  if (splits > 1) cluster_sync_all();  // every partial tile of the cluster is staged
+
+  if (warp >= 2) {
+    // part 3: sum the partial columns this CTA owns (ranks in order 0..splits-1) and finish them.
+    // One group = kBatch columns: all partial columns of a group are requested first
+    // (independent loads), then summed and finished.  Warp w takes groups w, w+4, w+8, ...
+    uint32_t rank_base[8];
+#pragma unroll
+    for (int rk = 0; rk < 8; ++rk) rank_base[rk] = splits > 1 ? map_to_rank(tiles, uint32_t(min(rk, splits - 1))) : tiles;
+    auto finish_group = [&](int jb, const float4 (&g0)[kBatch], const float4 (&g1)[kBatch]) {
+      float4 acc[kBatch];
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {   // ranks 0-3, then 4-7: at most 12 loads in flight
+        float4 part[kBatch][4];
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b)
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (half * 4 + q < splits && jb + b < own)
+              part[b][q] = ld_cluster_f4(rank_base[half * 4 + q] + uint32_t(((krank * slice + jb + b) * kBM + 4 * lane) * 4));
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b)
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (half * 4 + q < splits && jb + b < own) {
+              if (half == 0 && q == 0) acc[b] = part[b][0];
+              else { acc[b].x += part[b][q].x; acc[b].y += part[b][q].y; acc[b].z += part[b][q].z; acc[b].w += part[b][q].w; }
+            }
+        if (splits <= 4) break;
+      }
+#pragma unroll
+      for (int b = 0; b < kBatch; ++b) {
+        const int jj = jb + b;
+        if (jj >= own) break;
+        const int j = krank * slice + jj, r = r0 + j;
+        if (r >= e.R_rows) continue;   // the last token tile may overhang the buffers
+        const float rstd = s_rstd[j];
+        if (EPI == EPI_PLAIN) epi_plain(e, r, n0, lane, acc[b], rstd, N);
+        else if (EPI == EPI_RESID) epi_resid(e, r, n0, lane, acc[b], N, wtile, g0[b], gain4);
+        else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, wtile * 64, lane, acc[b], rstd);
+        else epi_qkv(e, r, n0, lane, acc[b], rstd, N, s_pos[j], s_page[j], g0[b], g1[b]);
+      }
+    };
+#pragma unroll
+    for (int k = 0; k < kPre; ++k)
+      if ((ew + 4 * k) * kBatch < own) finish_group((ew + 4 * k) * kBatch, pg0[k], pg1[k]);
+    for (int jb = (ew + 4 * kPre) * kBatch; jb < own; jb += 4 * kBatch) {
+      float4 g0[kBatch], g1[kBatch];
+#pragma unroll
+      for (int b = 0; b < kBatch; ++b) fetch_operands(jb + b, g0[b], g1[b]);
+      finish_group(jb, g0, g1);
+    }
+  } else if (warp == 0 && lane == 0 && !abort_flag) {
+    // Warm the L2 with the head of the next kernel's weights while the epilogue runs.
+    const unsigned worker = blockIdx.x + gridDim.x * blockIdx.y, n_workers = gridDim.x * gridDim.y;
+    prefetch_l2(e.next_w, e.next_bytes, worker, n_workers);
+    prefetch_l2(e.next_w2, e.next_bytes2, worker, n_workers);
+  }
+  __syncwarp();
+  if (splits > 1) cluster_sync_all();  // peers may still be reading this CTA's staged tile
+  __syncthreads();
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * kAccCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(tmem_cols) : "memory");
   }
-  if (threadIdx.x == 0 && abort_flag) {
-    atomicCAS(status, 0, LASER_ERR_TIMEOUT);
-  }
+  if (threadIdx.x == 0 && abort_flag) atomicCAS(status, 0, LASER_ERR_TIMEOUT);
 }
 
 // ---- host side --------------------------------------------------------------------------
@@ -470,7 +432,6 @@ struct GemmState {
   // (pointer, rows, cols, box rows) -> tensor map
   std::map<std::tuple<const void*, int, int, int>, CUtensorMap> maps;
   bool ready = false;
-  int max_clusters[5] = {0, 0, 0, 0, 0};   // co-resident clusters of size 1, 2, 4 (index = size)
 };
 
 GemmState* get_state(laser_model* m) {
@@ -490,26 +451,29 @@ laser_status tensor_map(GemmState* st, const void* ptr, int rows, int cols, int 
   return LASER_OK;
 }
 
-struct TcShape { int n_ttiles, NT, stages; size_t smem; };
+struct TcShape { int n_ttiles, NT, stages, tmem_cols; size_t smem; };
 
-TcShape tc_shape(int R_pad, int splits) {
+TcShape tc_shape(int R_pad) {
   TcShape s;
   s.n_ttiles = ceil_div(R_pad, kMaxNT);
   s.NT = ceil_div(ceil_div(R_pad, s.n_ttiles), 16) * 16;
   const int stage_bytes = kBM * 128 + s.NT * 128;
-  const int red_bytes = splits * ceil_div(s.NT, splits) * kBM * 4;
-  s.stages = std::max(2, std::min(kMaxStages, (kSmemLimit - 1024 - red_bytes) / stage_bytes));
-  s.smem = size_t(s.stages) * stage_bytes + red_bytes + 1024;
+  s.stages = std::max(2, std::min(kMaxStages, kSmemBudget / stage_bytes));
+  s.tmem_cols = 32;
+  while (s.tmem_cols < s.NT) s.tmem_cols <<= 1;
+  s.smem = std::max(size_t(s.stages) * stage_bytes, size_t(s.NT) * kBM * 4) + 1024;
   return s;
 }
 
 template <int EPI>
-void fill_launch(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int grid, int splits, size_t smem, cudaStream_t stream) {
-  *cfg = cudaLaunchConfig_t{};
-  cfg->gridDim = dim3(unsigned(grid), 1, 1);
-  cfg->blockDim = dim3(kTcThreads, 1, 1);
-  cfg->dynamicSmemBytes = smem;
-  cfg->stream = stream;
+laser_status launch_epi(const CUtensorMap& tw, const CUtensorMap& ta, const GemmEpilogue& e, int N, const TcShape& sh,
+                        int n_wtiles, int total_kb, int kbps, int splits, int32_t* status, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(sh.n_ttiles * splits), unsigned(n_wtiles), 1);
+  cfg.blockDim = dim3(kTcThreads, 1, 1);
+  cfg.dynamicSmemBytes = sh.smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = unsigned(splits);
   attr[0].val.clusterDim.y = 1;
@@ -518,42 +482,20 @@ void fill_launch(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int grid, i
   // orders itself with griddepcontrol.wait
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
-  cfg->attrs = attr;
-  cfg->numAttrs = 2;
-}
-
-template <int EPI>
-laser_status launch_epi(const CUtensorMap& tw, const CUtensorMap& ta, const GemmEpilogue& e, int N, const TcShape& sh,
-                        int n_wtiles, int total_kb, int kbps, int splits, int clusters, int32_t* status,
-                        cudaStream_t stream) {
-  cudaLaunchConfig_t cfg;
-  cudaLaunchAttribute attr[2];
-  fill_launch<EPI>(&cfg, attr, clusters * splits, splits, sh.smem, stream);
-  LASER_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI>, tw, ta, e, N, sh.NT, sh.n_ttiles, n_wtiles, total_kb, kbps,
-                                splits, sh.stages, status));
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  LASER_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI>, tw, ta, e, N, sh.NT, total_kb, kbps, splits, sh.stages,
+                                sh.tmem_cols, status));
   return LASER_OK;
 }
 
-// One-off per model: opt in to large shared memory and ask how many clusters of each size fit.
 laser_status prepare(GemmState* st) {
   if (st->ready) return LASER_OK;
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
-  int sms = 0, dev = 0;
-  LASER_CUDA(cudaGetDevice(&dev));
-  LASER_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  for (int s : {1, 2, 4}) {
-    cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[2];
-    fill_launch<EPI_RESID>(&cfg, attr, (sms / s) * s, s, size_t(kSmemLimit) - 8192, nullptr);
-    int n = 0;
-    cudaError_t err = cudaOccupancyMaxActiveClusters(&n, gemm_tc_kernel<EPI_RESID>, &cfg);
-    if (err != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
-    st->max_clusters[s] = std::max(0, std::min(n, sms / s));
-  }
-  if (st->max_clusters[1] <= 0) { set_error("the GEMM kernel does not fit this device"); return LASER_ERR_UNSUPPORTED; }
+  const int bytes = kSmemBudget + 2048;
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
   st->ready = true;
   return LASER_OK;
 }
@@ -563,23 +505,21 @@ laser_status prepare(GemmState* st) {
 int g_force_splits = 0;
 namespace {
 
-// Split count (cluster size) with the least modelled time: clusters work in lock step on one
-// tile each, a tile costs the K blocks of one rank plus a fixed share.
-int pick_splits(const GemmState* st, int R_pad, int N, int K, int epi, int* clusters_out) {
+// Split count (cluster size along K) with the least modelled time: the CTAs spread over
+// 2 x 148 slots; a slot's CTAs run one after the other and two slots share an SM's ingest, so
+// a CTA costs its K blocks plus a fixed share that the other slot can only partly hide.
+int pick_splits(int R_pad, int N, int K, int epi) {
   const int n_wtiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
-  const int total_kb = ceil_div(K, kBK);
-  int best = 1, best_clusters = 1;
+  const int tiles = n_wtiles * tc_shape(R_pad).n_ttiles, total_kb = ceil_div(K, kBK);
+  int best = 1;
   double best_cost = 1e30;
-  for (int s : {1, 2, 4}) {
-    if (st->max_clusters[s] <= 0 || (g_force_splits && s != g_force_splits)) continue;
+  for (int s = 1; s <= std::min(total_kb, 8); ++s) {
+    if (g_force_splits && s != g_force_splits) continue;
     const int kbps = ceil_div(total_kb, s);
     if (kbps * (s - 1) >= total_kb) continue;  // a rank would have no K blocks
-    const int tiles = n_wtiles * tc_shape(R_pad, s).n_ttiles;
-    const int clusters = std::min(st->max_clusters[s], tiles);
-    const double cost = double(ceil_div(tiles, clusters)) * (kbps + 1.5) + 2.0 + 0.5 * s;
-    if (cost < best_cost - 1e-9) { best_cost = cost; best = s; best_clusters = clusters; }
+    const double cost = double(ceil_div(tiles * s, 148)) * (kbps + 4.0) + 0.5 * s;
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
   }
-  *clusters_out = best_clusters;
   return best;
 }
 
@@ -593,19 +533,18 @@ laser_status gemm_fused(laser_model* m, const __nv_bfloat16* A, const __nv_bfloa
   }
   GemmState* st = get_state(m);
   LASER_TRY(prepare(st));
-  int clusters = 1;
-  const int splits = pick_splits(st, R_pad, N, K, epi, &clusters);
-  const TcShape sh = tc_shape(R_pad, splits);
+  const int splits = pick_splits(R_pad, N, K, epi);
+  const TcShape sh = tc_shape(R_pad);
   const CUtensorMap *tw = nullptr, *ta = nullptr;
   LASER_TRY(tensor_map(st, W, N, K, 64, &tw));
   LASER_TRY(tensor_map(st, A, m->R_pad, K, sh.NT, &ta));
   const int total_kb = ceil_div(K, kBK), kbps = ceil_div(total_kb, splits);
   const int n_wtiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
   switch (epi) {
-    case EPI_PLAIN: LASER_TRY(launch_epi<EPI_PLAIN>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, clusters, m->status, stream)); break;
-    case EPI_RESID: LASER_TRY(launch_epi<EPI_RESID>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, clusters, m->status, stream)); break;
-    case EPI_SWIGLU: LASER_TRY(launch_epi<EPI_SWIGLU>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, clusters, m->status, stream)); break;
-    default: LASER_TRY(launch_epi<EPI_QKV>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, clusters, m->status, stream)); break;
+    case EPI_PLAIN: LASER_TRY(launch_epi<EPI_PLAIN>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, m->status, stream)); break;
+    case EPI_RESID: LASER_TRY(launch_epi<EPI_RESID>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, m->status, stream)); break;
+    case EPI_SWIGLU: LASER_TRY(launch_epi<EPI_SWIGLU>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, m->status, stream)); break;
+    default: LASER_TRY(launch_epi<EPI_QKV>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, m->status, stream)); break;
   }
   count_launch();
   return LASER_OK;
