@@ -452,6 +452,11 @@ laser_status tensor_map(GemmState* st, const void* ptr, int rows, int cols, int 
 }
 
 struct TcShape { int n_ttiles, NT, stages, tmem_cols; size_t smem; };
+}  // namespace
+// Tuning aids: non-zero values override the modelled split count / the stage count.
+int g_force_splits = 0;
+int g_force_stages = 0;
+namespace {
 
 TcShape tc_shape(int R_pad) {
   TcShape s;
@@ -459,6 +464,7 @@ TcShape tc_shape(int R_pad) {
   s.NT = ceil_div(ceil_div(R_pad, s.n_ttiles), 16) * 16;
   const int stage_bytes = kBM * 128 + s.NT * 128;
   s.stages = std::max(2, std::min(kMaxStages, kSmemBudget / stage_bytes));
+  if (g_force_stages) s.stages = std::max(2, std::min(s.stages, g_force_stages));
   s.tmem_cols = 32;
   while (s.tmem_cols < s.NT) s.tmem_cols <<= 1;
   s.smem = std::max(size_t(s.stages) * stage_bytes, size_t(s.NT) * kBM * 4) + 1024;
@@ -500,27 +506,17 @@ laser_status prepare(GemmState* st) {
   return LASER_OK;
 }
 
-}  // namespace
-// Tuning aid: a non-zero value overrides the modelled choice of the split count.
-int g_force_splits = 0;
-namespace {
-
-// Split count (cluster size along K) with the least modelled time: the CTAs spread over
-// 2 x 148 slots; a slot's CTAs run one after the other and two slots share an SM's ingest, so
-// a CTA costs its K blocks plus a fixed share that the other slot can only partly hide.
+// Split count (cluster size along K).  Measured on the 7B shapes with 144 rows: a launch is
+// fastest with roughly 200 CTAs (of the 296 resident slots), whatever the matrix: 1 for 172 or
+// 250 weight tiles, 2 for 96, 6 for 32.  Fewer CTAs leave SMs idle, more add start-up and
+// cluster-reduction cost faster than they shorten the K loop.
 int pick_splits(int R_pad, int N, int K, int epi) {
   const int n_wtiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
   const int tiles = n_wtiles * tc_shape(R_pad).n_ttiles, total_kb = ceil_div(K, kBK);
-  int best = 1;
-  double best_cost = 1e30;
-  for (int s = 1; s <= std::min(total_kb, 8); ++s) {
-    if (g_force_splits && s != g_force_splits) continue;
-    const int kbps = ceil_div(total_kb, s);
-    if (kbps * (s - 1) >= total_kb) continue;  // a rank would have no K blocks
-    const double cost = double(ceil_div(tiles * s, 148)) * (kbps + 4.0) + 0.5 * s;
-    if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
-  }
-  return best;
+  int s = g_force_splits ? g_force_splits : int(208.0 / tiles + 0.5);
+  s = std::max(1, std::min(s, std::min(total_kb, 8)));
+  while (s > 1 && ceil_div(total_kb, s) * (s - 1) >= total_kb) --s;   // no rank without K blocks
+  return s;
 }
 
 }  // namespace
