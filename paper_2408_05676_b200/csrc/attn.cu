@@ -17,7 +17,8 @@ namespace {
 using bf16 = __nv_bfloat16;
 constexpr int kConsumers = 4;
 constexpr int kAttnThreads = (kConsumers + 1) * 32;
-constexpr int kStages = 8;   // a multiple of kConsumers: stage s always serves warp s % 4
+constexpr int kStages = 4;   // a multiple of kConsumers: stage s always serves warp s % 4
+constexpr int kCtasPerSm = 4;  // registers and shared memory are sized for four resident CTAs
 
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -39,7 +40,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 template <int DH>
-__global__ void __launch_bounds__(kAttnThreads)
+__global__ void __launch_bounds__(kAttnThreads, kCtasPerSm)
 attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restrict__ q,
                   const int32_t* __restrict__ seq_ids, const int32_t* __restrict__ row_ctx,
                   const int32_t* __restrict__ row_n, int Rs, int H, int Hkv,
@@ -128,12 +129,9 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
   // ---- consumers ----
   const int g = lane >> 2, qd = lane & 3;
   const float sl2 = rsqrtf(float(DH)) * 1.4426950408889634f;
-  uint32_t qf[DH / 16][4];
-  {
-    const int mat = lane >> 3, r = (lane & 7) + (mat & 1) * 8;
-#pragma unroll
-    for (int ks = 0; ks < DH / 16; ++ks) ldsm_x4(qf[ks], q_smem + uint32_t(r * QLD + ks * 16 + (mat >> 1) * 8) * 2);
-  }
+  // Q fragments are re-read from shared memory for every page: keeping them in registers
+  // would cost 32 registers per thread and one resident CTA per SM
+  const uint32_t q_frag = q_smem + uint32_t(((lane & 7) + ((lane >> 3) & 1) * 8) * QLD + (lane >> 4) * 8) * 2;
   float o[DH / 8][4];
 #pragma unroll
   for (int t = 0; t < DH / 8; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
@@ -153,10 +151,11 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
 #pragma unroll
       for (int ks = 0; ks < DH / 16; ++ks) {
         const int c = (ks & 3) * 2 + (mat & 1);
-        uint32_t kb[4];
+        uint32_t kb[4], qa[4];
+        ldsm_x4(qa, q_frag + ks * 32);
         ldsm_x4(kb, kbase + (ks >> 2) * SUB + key * 128 + ((c ^ (key & 7)) << 4));
-        mma16816(sc[0], qf[ks], kb[0], kb[1]);
-        mma16816(sc[1], qf[ks], kb[2], kb[3]);
+        mma16816(sc[0], qa, kb[0], kb[1]);
+        mma16816(sc[1], qa, kb[2], kb[3]);
       }
     }
     // causal mask, online softmax (rows g and g+8 of the tile)
