@@ -122,7 +122,7 @@ class Pool:
         return dict(n_tokens=a.value, n_keys=b.value, device_bytes=c.value)
 
     def free(self):
-        if self.handle:
+        if self.handle and lib is not None:      # lib is None while the interpreter shuts down
             lib.laser_pool_free(self.handle)
             self.handle = None
 
@@ -174,7 +174,7 @@ class Model:
         self.handle, self.cfg, self._keep = handle, cfg, keep
 
     def free(self):
-        if self.handle:
+        if self.handle and lib is not None:
             lib.laser_model_free(self.handle)
             self.handle = None
 
@@ -213,7 +213,7 @@ class KV:
         self.handle, self.model, self.max_seqs, self.n_pages = handle, model, max_seqs, n_pages
 
     def free(self):
-        if self.handle:
+        if self.handle and lib is not None:
             lib.laser_kv_free(self.handle)
             self.handle = None
 
