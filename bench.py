@@ -30,6 +30,8 @@ from paper_2408_05676_b200 import synth  # noqa: E402
 WORKLOAD = "verify-step-7b: batch 16, ctx 512 (16-token pages), 1+8 rows/seq, drafts 60% agreement"
 B, K, CTX, N_MAX = 16, 8, 512, 4
 POOL_TOKENS, POOL_GROUPS = 5_000_000, 1000
+# (105.4 + 76.5 + 218.1 + 138.7) MB per layer x 32 + 267.2 MB LM head, from the ncu capture
+GEMM_DRAM_TRAFFIC_PER_STEP = int((105.4 + 76.5 + 218.1 + 138.7) * 32e6 + 267.2e6)
 SAMPLE_LAYERS = 4          # layers the CPU baseline really runs (time is extrapolated to all)
 
 
@@ -158,15 +160,11 @@ def build_workload(L, dev, cfg):
 
 def run_ours(args):
     from paper_2408_05676_b200 import binding as L
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from paper_2408_05676_b200 import replicas
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = "cuda:%d" % local
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    dist, rank, world = replicas.init("nccl", torch.device(dev))
     cfg = synth.model_cfg("7b", n_layers=args.layers)
     wl = build_workload(L, dev, cfg)
     model, kv, seq_ids, lens = wl["model"], wl["kv"], wl["seq_ids"], wl["lens"]
@@ -207,10 +205,7 @@ def run_ours(args):
                  relaxed_cal=L.make_params(K=K, n_min=1, n_max=N_MAX, max_occ=64, mode=L.MODE_RELAXED, topk=2, p=p_cal))
 
     def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
+        replicas.barrier(dist, torch.device(dev))
 
     def timed(prm, steps, warmup, sample_clocks=False):
         for _ in range(warmup):
@@ -228,11 +223,7 @@ def run_ours(args):
         barrier()
         if sampler:
             sampler.__exit__()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t[0])
+        ms, _ = replicas.reduce_step(dist, e0.elapsed_time(e1), 0, torch.device(dev))
         n_out = int(outs[2].sum())
         n_acc = int(outs[0].sum())
         return dict(ms=ms / steps, tokens=n_out, accepted=n_acc, launches=(L.launch_count() - l0) // steps,
@@ -283,11 +274,7 @@ def run_ours(args):
         e2e_step()
     e1.record()
     barrier()
-    e2e_ms = e0.elapsed_time(e1) / args.steps
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t[0])
+    e2e_ms, _ = replicas.reduce_step(dist, e0.elapsed_time(e1) / args.steps, 0, torch.device(dev))
     e2e_value = world * int(h_out[2].sum()) / (e2e_ms * 1e-3)
 
     if rank != 0:
@@ -313,7 +300,8 @@ def run_ours(args):
         "gpu_launches": int(main["launches"] * args.steps),
         "roofline": {"kernel": "gemm_tc_kernel (all dense contractions of one verify step)", "bound": "hbm",
                      "achieved": gemm_gbs, "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
-                     "frac": gemm_gbs / peaks["hbm_gbs"], "traffic": None,
+                     "frac": gemm_gbs / peaks["hbm_gbs"], "traffic": GEMM_DRAM_TRAFFIC_PER_STEP if args.layers == 32 else None,
+                     "traffic_note": "ncu dram read+write summed over the 129 launches of a step (per-launch figures in profiles/gemm_tc_kernel_7b_rows144.md, scaled from a 2-layer capture); includes up to 48 MB of next-kernel L2 prefetch per launch, counted twice under ncu's serialised replay",
                      "algorithmic_bytes_per_step": ab["weights"], "ms_per_step": gemm_ms, "launches_per_step": gemm_n // args.steps},
         "verify_step": {"ms": verify_ms, "algorithmic_bytes": ab["total"],
                         "achieved_gbs": ab["total"] / (verify_ms * 1e-3) / 1e9,

@@ -30,10 +30,15 @@ def setup(L):
     cfg = synth.model_cfg("tiny")
     Wc = synth.make_weights(cfg, seed=0)
     m = L.model_create(cfg, weights_to(Wc, "cuda"), max_batch=16)
-    kv = L.kv_create(m, 16, 16 * 40)
-    # pool: the library's own greedy outputs on 12 other prompts, 3 per group
-    pool_prompts = [synth.make_prompt(64, cfg["vocab"], 1000 + i) for i in range(12)]
-    docs = L.generate(m, kv, None, pool_prompts, [0] * 12, L.make_params(K=8, max_new=200))["out"]
+    kv = L.kv_create(m, 16, 16 * 40)      # 640 tokens per sequence
+    # pool: the library's own greedy outputs (400 tokens each, 20k in all) on 50 other prompts,
+    # prompts 0-12 / 13-24 / 25-37 / 38-49 -> groups 0-3
+    pool_prompts = [synth.make_prompt(64, cfg["vocab"], 1000 + i) for i in range(50)]
+    docs = []
+    for i in range(0, 50, 16):
+        part = pool_prompts[i:i + 16]
+        docs += L.generate(m, kv, None, part, [0] * len(part), L.make_params(K=8, max_new=400))["out"]
+    bounds = [0, 13, 25, 38, 50]
     prompts = [synth.make_prompt(64, cfg["vocab"], 2000 + b) for b in range(4)]
     # "old knowledge resembles new knowledge": each group also holds a corrupted copy of what
     # its test prompt will generate, so drafts are found and are sometimes wrong
@@ -42,7 +47,8 @@ def setup(L):
     for o in own:
         for i in range(3, len(o), 11):
             o[i] = int(rng.integers(0, cfg["vocab"]))
-    pool, offs = synth.pool_from_documents([docs[3 * g:3 * g + 3] + [own[g]] for g in range(4)])
+    pool, offs = synth.pool_from_documents([docs[bounds[g]:bounds[g + 1]] + [own[g]] for g in range(4)])
+    assert 20000 <= len(pool) <= 20400
     return cfg, Wc, m, kv, pool, offs, prompts
 
 
