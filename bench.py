@@ -233,25 +233,30 @@ def run_ours(args):
     main = res["strict"]
     value = world * main["tokens"] / (main["ms"] * 1e-3)
 
-    # kernel-class profile: verify-step, dense-contraction and attention device time per step
-    L.profile_enable(model, True)
-    L.profile_read(model, 0), L.profile_read(model, 1)
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * args.steps)]
-    for i in range(args.steps):
-        L.kv_set_len_dev(kv, lens)
-        L.draft(pool, d_tails, d_tl, d_gid, strict, draft, dlen, mn)
-        L.make_rows(d_last, draft, dlen, K, tokens, n_rows)
-        ev[2 * i].record()
-        L.verify_step(model, kv, seq_ids, tokens, n_rows, logits)
-        ev[2 * i + 1].record()
-        L.accept_commit(kv, seq_ids, logits, tokens, n_rows, strict, out=outs)
-    torch.cuda.synchronize()
-    gemm_ms, gemm_n = L.profile_read(model, 0)
-    attn_ms, attn_n = L.profile_read(model, 1)
-    L.profile_enable(model, False)
-    verify_ms = sum(ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(args.steps)) / args.steps
-    gemm_ms /= args.steps
-    attn_ms /= args.steps
+    def verify_pass(profile):
+        """Same steps again with events around laser_verify_step; with `profile` every dense
+        contraction and attention launch is bracketed by events too (which keeps consecutive
+        kernels from overlapping, so those class times sum to more than the plain verify time)."""
+        L.profile_enable(model, profile)
+        L.profile_read(model, 0), L.profile_read(model, 1)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * args.steps)]
+        for i in range(args.steps):
+            L.kv_set_len_dev(kv, lens)
+            L.draft(pool, d_tails, d_tl, d_gid, strict, draft, dlen, mn)
+            L.make_rows(d_last, draft, dlen, K, tokens, n_rows)
+            ev[2 * i].record()
+            L.verify_step(model, kv, seq_ids, tokens, n_rows, logits)
+            ev[2 * i + 1].record()
+            L.accept_commit(kv, seq_ids, logits, tokens, n_rows, strict, out=outs)
+        torch.cuda.synchronize()
+        g_ms, g_n = L.profile_read(model, 0)
+        a_ms, _ = L.profile_read(model, 1)
+        L.profile_enable(model, False)
+        v_ms = sum(ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(args.steps)) / args.steps
+        return v_ms, g_ms / args.steps, a_ms / args.steps, g_n
+
+    verify_ms, _, _, _ = verify_pass(False)
+    verify_prof_ms, gemm_ms, attn_ms, gemm_n = verify_pass(True)
 
     # end to end: step inputs from pinned host memory, results back to the host, every step
     h_in = [t.cpu().pin_memory() for t in (d_tails, d_tl, d_gid, d_last)]
@@ -307,7 +312,9 @@ def run_ours(args):
                         "achieved_gbs": ab["total"] / (verify_ms * 1e-3) / 1e9,
                         "frac_of_measured_hbm": ab["total"] / (verify_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                         "frac_of_nominal_8tbs": ab["total"] / (verify_ms * 1e-3) / 1e9 / 8000.0,
-                        "gemm_ms": gemm_ms, "attention_ms": attn_ms, "other_ms": verify_ms - gemm_ms - attn_ms},
+                        "profiled": {"note": "per-launch events on: kernels no longer overlap", "ms": verify_prof_ms,
+                                     "gemm_ms": gemm_ms, "attention_ms": attn_ms,
+                                     "other_ms": verify_prof_ms - gemm_ms - attn_ms}},
         "acceptance": {name: {"tokens_per_s": world * r["tokens"] / (r["ms"] * 1e-3), "ms_per_step": r["ms"],
                               "accepted_drafts_per_step": r["accepted"] / B, "emitted_per_step": r["tokens"] / B}
                        for name, r in res.items()},
