@@ -440,11 +440,13 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
   const int d = c.d_model, f = c.d_ffn, dh = c.head_dim, H = c.n_heads, Hkv = c.n_kv_heads;
   const int capacity = int(std::min<int64_t>(kv->capacity_tokens(), INT32_MAX));
 
-  prep_rows_kernel<<<Rp, 64, 0, stream>>>(seq_ids, n_rows, B, Rs, Rp, kv->seq_len, kv->max_seqs, capacity, dh / 2,
+  // Every row of the workspace is (re)marked: a GEMM's last token tile may reach past this call's
+  // rows, and whatever it finds there must be inactive (no cache write) and finite.
+  prep_rows_kernel<<<m->R_pad, 64, 0, stream>>>(seq_ids, n_rows, B, Rs, Rp, kv->seq_len, kv->max_seqs, capacity, dh / 2,
                                           double(c.rope_theta), dh, m->row_pos, m->row_seq, m->row_ctx, m->row_n,
                                           m->rope, m->status);
   const __nv_bfloat16* first_gain = c.n_layers > 0 ? m->attn_norm[0] : m->final_norm;
-  embed_kernel<<<Rp, 256, 0, stream>>>(tokens, R, d, c.vocab, m->tok_emb, first_gain, m->resid, m->xn, m->sumsq);
+  embed_kernel<<<m->R_pad, 256, 0, stream>>>(tokens, R, d, c.vocab, m->tok_emb, first_gain, m->resid, m->xn, m->sumsq);
   count_launch(2);
   const bool use_tma_attn = attention_tma_supported(m, kv);
   const size_t attn_smem = (size_t(dh) + size_t(capacity) + 8) * sizeof(float);

@@ -73,6 +73,8 @@ def _check_new_kv(L, kv, okv, cfg, seq, n_new):
     ("tiny", dict(), 4, [150, 0, 170, 5]),
     ("tiny", dict(n_layers=3, d_model=512, n_heads=4, n_kv_heads=4, head_dim=128, d_ffn=1376, vocab=8192), 3, [130, 16, 1]),
     ("tiny", dict(n_layers=2, d_model=256, n_heads=8, n_kv_heads=2, head_dim=32, d_ffn=256, vocab=1000, max_draft=3), 5, [9, 33, 2, 0, 17]),
+    # 30 sequences x 9 rows = 270 rows: two token tiles in every GEMM, the second one overhanging
+    ("tiny", dict(), 30, [int(x) for x in np.random.default_rng(3).integers(0, 150, 30)]),
 ])
 def test_logits_and_cache_match_oracle(L, name, over, B, ctx):
     cfg = synth.model_cfg(name, **over)
