@@ -60,6 +60,26 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// ---- two-CTA forms: the CTAs of ranks 2i and 2i+1 of a cluster run one 256-row MMA together ----
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives on the barrier at the same shared-memory offset in every CTA named by the rank mask
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint32_t rank_mask) {
+  asm volatile(
+      "{\n.reg .b16 m;\ncvt.u16.u32 m, %1;\n"
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n}"
+      ::"r"(bar), "r"(rank_mask) : "memory");
+}
+// tile load whose completion bytes are counted on a barrier of the pair's first CTA
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t leader_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(leader_bar) : "memory");
+}
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
@@ -123,85 +143,116 @@ __device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) 
 }
 
 // ---- fused epilogues: one warp finishes one token row r of a 128-feature tile; lane l holds
-//      features n0 + 4l .. 4l+3 in v ----------------------------------------------------------
-__device__ __forceinline__ void epi_plain(const GemmEpilogue& e, int r, int n0, int lane, float4 v, float rstd, int N) {
-  if (r >= e.R_store) return;
-  const int n = n0 + 4 * lane;
-  float* o = e.out + size_t(r) * e.ldo + n;
+//      features n0 + 4l .. 4l+3 in v.  What depends on the feature alone is worked out once per
+//      thread (LaneCtx); rows are finished without branches (`live` predicates the stores), so
+//      that the rows of a group interleave. ------------------------------------------------------
+struct LaneCtx {
+  int n;            // first of the lane's four features
+  bool in_range;    // n < N (N is a multiple of 8: then all four features are valid)
+  bool vec_out;     // EPI_PLAIN: the four results may be stored as one float4
+  // EPI_QKV
+  int kind;         // 0 = Q, 1 = K, 2 = V
+  int idx;          // offset of the feature inside its head
+  int shift;        // lanes between a feature and its rotation partner
+  float sg;         // sign of the partner's term
+  size_t kv_off;    // offset of (K or V, head, idx) inside a page
+  int rope_off;     // offset of the lane's first (cos, sin) pair inside a row of the table
+};
+
+template <int EPI>
+__device__ __forceinline__ LaneCtx make_lane_ctx(const GemmEpilogue& e, int n0, int lane, int N) {
+  LaneCtx c;
+  c.n = n0 + 4 * lane;
+  c.in_range = c.n < N;
+  c.vec_out = c.n + 3 < N && (e.ldo & 3) == 0;
+  c.kind = 0; c.idx = 0; c.shift = 0; c.sg = 0.f; c.kv_off = 0; c.rope_off = 0;
+  if (EPI == EPI_QKV) {
+    const int dh = e.dh, half = dh >> 1, dq = e.H * dh, dkv = e.Hkv * dh;
+    c.shift = dh >> 3;
+    c.kind = c.n < dq ? 0 : (c.n < dq + dkv ? 1 : 2);
+    c.idx = c.n % dh;          // four consecutive features stay inside one half of one head
+    c.sg = c.idx < half ? -1.f : 1.f;
+    c.rope_off = (c.idx % half) * 2;
+    if (c.kind) {
+      const int h = (c.n - dq - (c.kind - 1) * dkv) / dh;
+      c.kv_off = (size_t(c.kind - 1) * e.Hkv + h) * 16 * dh + c.idx;
+    }
+  }
+  return c;
+}
+
+__device__ __forceinline__ void epi_plain(const GemmEpilogue& e, const LaneCtx& c, int r, bool live, float4 v, float rstd, int N) {
+  if (!live || r >= e.R_store) return;
+  float* o = e.out + size_t(r) * e.ldo + c.n;
   v.x *= rstd; v.y *= rstd; v.z *= rstd; v.w *= rstd;
-  if (n + 3 < N && (e.ldo & 3) == 0) {
+  if (c.vec_out) {
     *reinterpret_cast<float4*>(o) = v;
   } else {
-    if (n < N) o[0] = v.x;
-    if (n + 1 < N) o[1] = v.y;
-    if (n + 2 < N) o[2] = v.z;
-    if (n + 3 < N) o[3] = v.w;
+    if (c.n < N) o[0] = v.x;
+    if (c.n + 1 < N) o[1] = v.y;
+    if (c.n + 2 < N) o[2] = v.z;
+    if (c.n + 3 < N) o[3] = v.w;
   }
 }
 
 // resid += acc; xb = bf16(resid * gain of the next norm); per-tile sum of squares for that norm
-__device__ __forceinline__ void epi_resid(const GemmEpilogue& e, int r, int n0, int lane, float4 v, int N, int tile,
-                                          float4 x, uint2 g2) {
-  const int n = n0 + 4 * lane;
+__device__ __forceinline__ void epi_resid(const GemmEpilogue& e, const LaneCtx& c, int r, bool live, int lane, float4 v, int N,
+                                          int tile, float4 x, uint2 g2) {
   float ss = 0.f;
-  if (n < N) {  // N is a multiple of 8 (checked on the host), so the four features are all valid
-    x.x += v.x; x.y += v.y; x.z += v.z; x.w += v.w;
-    *reinterpret_cast<float4*>(e.resid + size_t(r) * N + n) = x;
+  x.x += v.x; x.y += v.y; x.z += v.z; x.w += v.w;
+  if (live && c.in_range) {
+    *reinterpret_cast<float4*>(e.resid + size_t(r) * N + c.n) = x;
     const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&g2.x), g23 = *reinterpret_cast<const __nv_bfloat162*>(&g2.y);
-    *reinterpret_cast<uint2*>(e.xb + size_t(r) * N + n) =
+    *reinterpret_cast<uint2*>(e.xb + size_t(r) * N + c.n) =
         pack4_bf16(x.x * __low2float(g01), x.y * __high2float(g01), x.z * __low2float(g23), x.w * __high2float(g23));
     ss = x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
   }
   for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-  if (lane == 0) e.sumsq_out[size_t(tile) * e.sumsq_ld + r] = ss;
+  if (live && lane == 0) e.sumsq_out[size_t(tile) * e.sumsq_ld + r] = ss;
 }
 
-// tile rows 0..63 = gate features f0.., rows 64..127 = up features f0..; act = silu(g) * u
-__device__ __forceinline__ void epi_swiglu(const GemmEpilogue& e, int r, int f0, int lane, float4 v, float rstd) {
-  float4 u;
-  u.x = __shfl_xor_sync(0xffffffffu, v.x, 16); u.y = __shfl_xor_sync(0xffffffffu, v.y, 16);
-  u.z = __shfl_xor_sync(0xffffffffu, v.z, 16); u.w = __shfl_xor_sync(0xffffffffu, v.w, 16);
-  const int fidx = f0 + 4 * lane;
-  if (lane < 16 && fidx < e.f) {  // f is a multiple of 8 (checked on the host)
-    auto act = [rstd](float g, float up) { g *= rstd; up *= rstd; return __fdividef(g, 1.f + __expf(-g)) * up; };
-    *reinterpret_cast<uint2*>(e.act + size_t(r) * e.f + fidx) =
-        pack4_bf16(act(v.x, u.x), act(v.y, u.y), act(v.z, u.z), act(v.w, u.w));
+// Tile rows 0..63 = gate features f0.., rows 64..127 = up features f0..: lanes 0-15 hold four
+// gate values each, lanes 16-31 the four up values of the same features.  Each pair of lanes
+// (l, l+16) trades two values, so that every lane finishes two features: act = silu(g) * u.
+__device__ __forceinline__ void epi_swiglu(const GemmEpilogue& e, int r, bool live, int f0, int lane, float4 v, float rstd) {
+  const bool lo = lane < 16;
+  const float t0 = __shfl_xor_sync(0xffffffffu, lo ? v.z : v.x, 16);
+  const float t1 = __shfl_xor_sync(0xffffffffu, lo ? v.w : v.y, 16);
+  const float g0 = (lo ? v.x : t0) * rstd, g1 = (lo ? v.y : t1) * rstd;
+  const float u0 = (lo ? t0 : v.z) * rstd, u1 = (lo ? t1 : v.w) * rstd;
+  const int fidx = f0 + 4 * (lane & 15) + (lo ? 0 : 2);
+  if (live && fidx < e.f) {  // f is a multiple of 8 (checked on the host)
+    const __nv_bfloat162 a = __floats2bfloat162_rn(__fdividef(g0, 1.f + __expf(-g0)) * u0, __fdividef(g1, 1.f + __expf(-g1)) * u1);
+    *reinterpret_cast<__nv_bfloat162*>(e.act + size_t(r) * e.f + fidx) = a;
   }
 }
 
 // rotary embedding of Q and K (pair i, i + dh/2), bf16 rounding, Q store, K/V page write
-__device__ __forceinline__ void epi_qkv(const GemmEpilogue& e, int r, int n0, int lane, float4 v, float rstd, int N,
+__device__ __forceinline__ void epi_qkv(const GemmEpilogue& e, const LaneCtx& c, int r, bool live, float4 v, float rstd,
                                         int pos, int page, float4 cs01, float4 cs23) {
   v.x *= rstd; v.y *= rstd; v.z *= rstd; v.w *= rstd;
-  const int dh = e.dh, half = dh >> 1, dq = e.H * dh, dkv = e.Hkv * dh;
-  const int shift = dh >> 3;  // lanes between a feature and its rotation partner
   float4 pv;
-  pv.x = __shfl_xor_sync(0xffffffffu, v.x, shift); pv.y = __shfl_xor_sync(0xffffffffu, v.y, shift);
-  pv.z = __shfl_xor_sync(0xffffffffu, v.z, shift); pv.w = __shfl_xor_sync(0xffffffffu, v.w, shift);
-  const int n = n0 + 4 * lane;
-  if (n >= N) return;
-  const int idx = n % dh;          // four consecutive features stay inside one half of one head
+  pv.x = __shfl_xor_sync(0xffffffffu, v.x, c.shift); pv.y = __shfl_xor_sync(0xffffffffu, v.y, c.shift);
+  pv.z = __shfl_xor_sync(0xffffffffu, v.z, c.shift); pv.w = __shfl_xor_sync(0xffffffffu, v.w, c.shift);
   float4 y = v;
-  if (n < dq + dkv) {
-    const float sg = idx < half ? -1.f : 1.f;
-    y.x = v.x * cs01.x + sg * pv.x * cs01.y;
-    y.y = v.y * cs01.z + sg * pv.y * cs01.w;
-    y.z = v.z * cs23.x + sg * pv.z * cs23.y;
-    y.w = v.w * cs23.z + sg * pv.w * cs23.w;
+  if (c.kind < 2) {
+    y.x = v.x * cs01.x + c.sg * pv.x * cs01.y;
+    y.y = v.y * cs01.z + c.sg * pv.y * cs01.w;
+    y.z = v.z * cs23.x + c.sg * pv.z * cs23.y;
+    y.w = v.w * cs23.z + c.sg * pv.w * cs23.w;
   }
-  if (n < dq) {
+  if (!live || !c.in_range) return;
+  if (c.kind == 0) {
     if (pos < 0) y = make_float4(0.f, 0.f, 0.f, 0.f);
-    *reinterpret_cast<uint2*>(e.q + size_t(r) * dq + n) = pack4_bf16(y.x, y.y, y.z, y.w);
+    *reinterpret_cast<uint2*>(e.q + size_t(r) * (e.H * e.dh) + c.n) = pack4_bf16(y.x, y.y, y.z, y.w);
   } else if (pos >= 0) {
-    const int is_v = n >= dq + dkv;
-    const int h = (n - dq - is_v * dkv) / dh;
-    bf16* dst = e.pages_layer + size_t(page) * e.page_elems + (size_t(is_v) * e.Hkv + h) * 16 * dh + size_t(pos & 15) * dh + idx;
+    bf16* dst = e.pages_layer + size_t(page) * e.page_elems + c.kv_off + size_t(pos & 15) * e.dh;
     *reinterpret_cast<uint2*>(dst) = pack4_bf16(y.x, y.y, y.z, y.w);
   }
 }
 
 
-template <int EPI>
+template <int EPI, bool PAIR>
 __global__ void __launch_bounds__(kTcThreads, 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, const GemmEpilogue e,
                int N, int NT, int total_kb, int kb_per_split, int splits, int stages, int tmem_cols,
@@ -215,9 +266,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its prologue
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
-  const uint32_t w_bytes = kBM * 128, a_bytes = uint32_t(NT) * 128, stage_bytes = w_bytes + a_bytes;
+  // PAIR: the cluster holds 2 x splits CTAs, rank = 2 x (K range) + (half of a 256-row weight tile);
+  // each CTA stages its own 128 weight rows and half of the token rows.
+  const uint32_t w_bytes = kBM * 128, a_bytes = uint32_t(PAIR ? NT / 2 : NT) * 128, stage_bytes = w_bytes + a_bytes;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int krank = blockIdx.x % splits, ttile = blockIdx.x / splits, wtile = blockIdx.y;
+  const int csize = PAIR ? 2 * splits : splits, crank = blockIdx.x % csize, ttile = blockIdx.x / csize;
+  const int half = PAIR ? (crank & 1) : 0, krank = PAIR ? (crank >> 1) : crank;
+  const int wtile = PAIR ? 2 * blockIdx.y + half : blockIdx.y;
   const int r0 = ttile * NT, n0 = wtile * kBM;
   const int kb0 = krank * kb_per_split;
   const int nkb = max(0, min(kb_per_split, total_kb - kb0));
@@ -233,16 +288,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     tma_prefetch_map(&tmA);
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(tmem_cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (PAIR) {  // issued by the same warp of both CTAs of the pair
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(tmem_cols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(tmem_cols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  if (PAIR) cluster_sync_all();   // the partner's copies count on this CTA's barriers: they must exist first
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = tmem_slot;
 
   // epilogue operands live in registers of warps 2-5 from kernel start to the epilogue
   const int ew = warp - 2, nfeat = n0 + 4 * lane;
+  const LaneCtx lc = make_lane_ctx<EPI>(e, n0, lane, N);
   uint2 gain4 = make_uint2(0u, 0u);
   float4 pg0[kPre][kBatch], pg1[kPre][kBatch];
   auto fetch_operands = [&](int jj, float4& g0, float4& g1) {
@@ -250,8 +312,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const int r = r0 + krank * slice + jj;
     if (jj < own && r < e.R_rows && nfeat < N) {
       if (EPI == EPI_RESID) g0 = *reinterpret_cast<const float4*>(e.resid + size_t(r) * N + nfeat);
-      if (EPI == EPI_QKV && nfeat < (e.H + e.Hkv) * e.dh) {
-        const float* cs = e.rope + (size_t(r) * (e.dh >> 1) + (nfeat % e.dh) % (e.dh >> 1)) * 2;
+      if (EPI == EPI_QKV && lc.kind < 2) {
+        const float* cs = e.rope + size_t(r) * e.dh + lc.rope_off;
         g0 = *reinterpret_cast<const float4*>(cs);       // c0 s0 c1 s1
         g1 = *reinterpret_cast<const float4*>(cs + 4);   // c2 s2 c3 s3
       }
@@ -260,20 +322,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 
   if (warp == 0) {
     if (lane == 0) {  // ---- TMA producer ----
+      // PAIR: both CTAs' copies complete on the first CTA's barrier, which expects the bytes of both
+      const uint32_t full0 = PAIR ? map_to_rank(smem_u32(&full_bar[0]), uint32_t(crank & ~1)) : smem_u32(&full_bar[0]);
+      auto load = [&](uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+        if (PAIR) tma_load_2d_pair(dst, tm, x, y, bar); else tma_load_2d(dst, tm, x, y, bar);
+      };
+      auto expect = [&](int s) {
+        if (!PAIR) mbar_expect_tx(smem_u32(&full_bar[s]), stage_bytes);
+        else if (half == 0) mbar_expect_tx(smem_u32(&full_bar[s]), 2 * stage_bytes);
+      };
       auto load_w = [&](int kb) {
         const int s = kb % stages, k = (kb0 + kb) * kBK;
-        const uint32_t dst = tiles + uint32_t(s) * stage_bytes, bar = smem_u32(&full_bar[s]);
-        tma_load_2d(dst, &tmW, k, EPI == EPI_SWIGLU ? wtile * 64 : n0, bar);
-        tma_load_2d(dst + w_bytes / 2, &tmW, k, EPI == EPI_SWIGLU ? e.f + wtile * 64 : n0 + 64, bar);
+        const uint32_t dst = tiles + uint32_t(s) * stage_bytes, bar = full0 + uint32_t(s) * 8;
+        load(dst, &tmW, k, EPI == EPI_SWIGLU ? wtile * 64 : n0, bar);
+        load(dst + w_bytes / 2, &tmW, k, EPI == EPI_SWIGLU ? e.f + wtile * 64 : n0 + 64, bar);
       };
       auto load_a = [&](int kb) {
         const int s = kb % stages;
-        tma_load_2d(tiles + uint32_t(s) * stage_bytes + w_bytes, &tmA, (kb0 + kb) * kBK, r0, smem_u32(&full_bar[s]));
+        load(tiles + uint32_t(s) * stage_bytes + w_bytes, &tmA, (kb0 + kb) * kBK, r0 + half * (NT / 2), full0 + uint32_t(s) * 8);
       };
       // The weights do not depend on the kernel before this one: fill the ring with weight
       // tiles first, and only then wait for the previous kernel's results (the activations).
       const int pre = min(stages, nkb);
-      for (int kb = 0; kb < pre; ++kb) { mbar_expect_tx(smem_u32(&full_bar[kb % stages]), stage_bytes); load_w(kb); }
+      for (int kb = 0; kb < pre; ++kb) { expect(kb % stages); load_w(kb); }
       asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int kb = 0; kb < pre; ++kb) load_a(kb);
       bool ok = true;
@@ -282,16 +353,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const int s = kb % stages;
         ok = mbar_wait(smem_u32(&empty_bar[s]), ((kb / stages) - 1) & 1, &abort_flag);
         if (!ok) break;
-        mbar_expect_tx(smem_u32(&full_bar[s]), stage_bytes);
+        expect(s);
         load_w(kb);
         load_a(kb);
       }
-      if (!ok)  // drain copies still in flight before the CTA may exit
+      if (!ok && half == 0)  // drain copies still in flight (the partner's too) before the CTAs may exit
         for (int j = max(0, kb - stages); j < kb; ++j) mbar_drain(smem_u32(&full_bar[j % stages]), (j / stages) & 1);
     }
   } else if (warp == 1) {
-    if (lane == 0) {  // ---- MMA issuer ----
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(NT >> 3) << 17) | (uint32_t(kBM >> 4) << 24);
+    if (lane == 0 && half == 0) {  // ---- MMA issuer (PAIR: the first CTA issues for both) ----
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(NT >> 3) << 17) | (uint32_t((PAIR ? 2 * kBM : kBM) >> 4) << 24);
+      const uint32_t pair_mask = 3u << (crank & ~1);
       bool ok = true;
       for (int kb = 0; kb < nkb && ok; ++kb) {
         const int s = kb % stages;
@@ -302,10 +374,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const uint64_t wdesc = umma_desc(w_addr), adesc = umma_desc(w_addr + w_bytes);
 #pragma unroll
         for (int k = 0; k < kBK / 16; ++k)  // 16 bf16 = 32 bytes further along K inside the swizzle span
-          umma_bf16(tmem_acc, wdesc + uint64_t(k * 2), adesc + uint64_t(k * 2), idesc, (kb | k) != 0);
-        umma_commit(smem_u32(&empty_bar[s]));
+          if (PAIR) umma_bf16_pair(tmem_acc, wdesc + uint64_t(k * 2), adesc + uint64_t(k * 2), idesc, (kb | k) != 0);
+          else umma_bf16(tmem_acc, wdesc + uint64_t(k * 2), adesc + uint64_t(k * 2), idesc, (kb | k) != 0);
+        if (PAIR) umma_commit_pair(smem_u32(&empty_bar[s]), pair_mask); else umma_commit(smem_u32(&empty_bar[s]));
       }
-      umma_commit(smem_u32(&acc_bar));  // arrives when every MMA issued so far has finished
+      // arrives when every MMA issued so far has finished
+      if (PAIR) umma_commit_pair(smem_u32(&acc_bar), pair_mask); else umma_commit(smem_u32(&acc_bar));
     }
   } else {
     // ---- epilogue warps, part 1: everything that can be done before the accumulator is ready ----
@@ -368,7 +442,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     // (independent loads), then summed and finished.  Warp w takes groups w, w+4, w+8, ...
     uint32_t rank_base[8];
 #pragma unroll
-    for (int rk = 0; rk < 8; ++rk) rank_base[rk] = splits > 1 ? map_to_rank(tiles, uint32_t(min(rk, splits - 1))) : tiles;
+    for (int rk = 0; rk < 8; ++rk)
+      rank_base[rk] = splits > 1 ? map_to_rank(tiles, uint32_t(PAIR ? 2 * min(rk, splits - 1) + half : min(rk, splits - 1))) : tiles;
     auto finish_group = [&](int jb, const float4 (&g0)[kBatch], const float4 (&g1)[kBatch]) {
       float4 acc[kBatch];
 #pragma unroll
@@ -393,14 +468,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 #pragma unroll
       for (int b = 0; b < kBatch; ++b) {
         const int jj = jb + b;
-        if (jj >= own) break;
-        const int j = krank * slice + jj, r = r0 + j;
-        if (r >= e.R_rows) continue;   // the last token tile may overhang the buffers
+        const int j = jj < own ? krank * slice + jj : 0, r = r0 + j;
+        const bool live = jj < own && r < e.R_rows;   // the last token tile may overhang the buffers
+        if (jj >= own) acc[b] = make_float4(0.f, 0.f, 0.f, 0.f);
         const float rstd = s_rstd[j];
-        if (EPI == EPI_PLAIN) epi_plain(e, r, n0, lane, acc[b], rstd, N);
-        else if (EPI == EPI_RESID) epi_resid(e, r, n0, lane, acc[b], N, wtile, g0[b], gain4);
-        else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, wtile * 64, lane, acc[b], rstd);
-        else epi_qkv(e, r, n0, lane, acc[b], rstd, N, s_pos[j], s_page[j], g0[b], g1[b]);
+        if (EPI == EPI_PLAIN) epi_plain(e, lc, r, live, acc[b], rstd, N);
+        else if (EPI == EPI_RESID) epi_resid(e, lc, r, live, lane, acc[b], N, wtile, g0[b], gain4);
+        else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, live, wtile * 64, lane, acc[b], rstd);
+        else epi_qkv(e, lc, r, live, acc[b], rstd, s_pos[j], s_page[j], g0[b], g1[b]);
       }
     };
 #pragma unroll
@@ -419,10 +494,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     prefetch_l2(e.next_w2, e.next_bytes2, worker, n_workers);
   }
   __syncwarp();
-  if (splits > 1) cluster_sync_all();  // peers may still be reading this CTA's staged tile
+  if (splits > 1 || PAIR) cluster_sync_all();  // peers may still be reading this CTA's staged tile or tensor memory
   __syncthreads();
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(tmem_cols) : "memory");
+    if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(tmem_cols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(tmem_cols) : "memory");
   }
   if (threadIdx.x == 0 && abort_flag) atomicCAS(status, 0, LASER_ERR_TIMEOUT);
 }
@@ -453,16 +529,18 @@ laser_status tensor_map(GemmState* st, const void* ptr, int rows, int cols, int 
 
 struct TcShape { int n_ttiles, NT, stages, tmem_cols; size_t smem; };
 }  // namespace
-// Tuning aids: non-zero values override the modelled split count / the stage count.
+// Tuning aids: non-zero values override the modelled split count / the stage count;
+// g_force_pair: 0 = single-CTA MMA only, 1 = two-CTA MMA wherever the shape allows it.
 int g_force_splits = 0;
 int g_force_stages = 0;
+int g_force_pair = 1;
 namespace {
 
-TcShape tc_shape(int R_pad) {
+TcShape tc_shape(int R_pad, bool pair) {
   TcShape s;
   s.n_ttiles = ceil_div(R_pad, kMaxNT);
   s.NT = ceil_div(ceil_div(R_pad, s.n_ttiles), 16) * 16;
-  const int stage_bytes = kBM * 128 + s.NT * 128;
+  const int stage_bytes = kBM * 128 + (pair ? s.NT / 2 : s.NT) * 128;
   s.stages = std::max(2, std::min(kMaxStages, kSmemBudget / stage_bytes));
   if (g_force_stages) s.stages = std::max(2, std::min(s.stages, g_force_stages));
   s.tmem_cols = 32;
@@ -471,17 +549,18 @@ TcShape tc_shape(int R_pad) {
   return s;
 }
 
-template <int EPI>
+template <int EPI, bool PAIR>
 laser_status launch_epi(const CUtensorMap& tw, const CUtensorMap& ta, const GemmEpilogue& e, int N, const TcShape& sh,
                         int n_wtiles, int total_kb, int kbps, int splits, int32_t* status, cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(unsigned(sh.n_ttiles * splits), unsigned(n_wtiles), 1);
+  cfg.gridDim = PAIR ? dim3(unsigned(sh.n_ttiles * splits * 2), unsigned(n_wtiles / 2), 1)
+                     : dim3(unsigned(sh.n_ttiles * splits), unsigned(n_wtiles), 1);
   cfg.blockDim = dim3(kTcThreads, 1, 1);
   cfg.dynamicSmemBytes = sh.smem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = unsigned(splits);
+  attr[0].val.clusterDim.x = unsigned(PAIR ? 2 * splits : splits);
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   // programmatic dependent launch: this kernel may begin while the previous one drains; it
@@ -490,7 +569,7 @@ laser_status launch_epi(const CUtensorMap& tw, const CUtensorMap& ta, const Gemm
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  LASER_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI>, tw, ta, e, N, sh.NT, total_kb, kbps, splits, sh.stages,
+  LASER_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI, PAIR>, tw, ta, e, N, sh.NT, total_kb, kbps, splits, sh.stages,
                                 sh.tmem_cols, status));
   return LASER_OK;
 }
@@ -498,10 +577,14 @@ laser_status launch_epi(const CUtensorMap& tw, const CUtensorMap& ta, const Gemm
 laser_status prepare(GemmState* st) {
   if (st->ready) return LASER_OK;
   const int bytes = kSmemBudget + 2048;
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
   st->ready = true;
   return LASER_OK;
 }
@@ -510,11 +593,11 @@ laser_status prepare(GemmState* st) {
 // fastest with roughly 200 CTAs (of the 296 resident slots), whatever the matrix: 1 for 172 or
 // 250 weight tiles, 2 for 96, 6 for 32.  Fewer CTAs leave SMs idle, more add start-up and
 // cluster-reduction cost faster than they shorten the K loop.
-int pick_splits(int R_pad, int N, int K, int epi) {
+int pick_splits(int R_pad, int N, int K, int epi, bool pair) {
   const int n_wtiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
-  const int tiles = n_wtiles * tc_shape(R_pad).n_ttiles, total_kb = ceil_div(K, kBK);
+  const int tiles = n_wtiles * tc_shape(R_pad, pair).n_ttiles, total_kb = ceil_div(K, kBK);
   int s = g_force_splits ? g_force_splits : int(208.0 / tiles + 0.5);
-  s = std::max(1, std::min(s, std::min(total_kb, 8)));
+  s = std::max(1, std::min(s, std::min(total_kb, pair ? 4 : 8)));   // a cluster holds 8 CTAs at most
   while (s > 1 && ceil_div(total_kb, s) * (s - 1) >= total_kb) --s;   // no rank without K blocks
   return s;
 }
@@ -529,19 +612,26 @@ laser_status gemm_fused(laser_model* m, const __nv_bfloat16* A, const __nv_bfloa
   }
   GemmState* st = get_state(m);
   LASER_TRY(prepare(st));
-  const int splits = pick_splits(R_pad, N, K, epi);
-  const TcShape sh = tc_shape(R_pad);
+  const int n_wtiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
+  // Two weight tiles share one 256-row MMA of a CTA pair (each CTA then stages only half of the
+  // token rows) when the tiles come in pairs.
+  const bool pair = g_force_pair != 0 && n_wtiles % 2 == 0;
+  const int splits = pick_splits(R_pad, N, K, epi, pair);
+  const TcShape sh = tc_shape(R_pad, pair);
   const CUtensorMap *tw = nullptr, *ta = nullptr;
   LASER_TRY(tensor_map(st, W, N, K, 64, &tw));
-  LASER_TRY(tensor_map(st, A, m->R_pad, K, sh.NT, &ta));
+  LASER_TRY(tensor_map(st, A, m->R_pad, K, pair ? sh.NT / 2 : sh.NT, &ta));
   const int total_kb = ceil_div(K, kBK), kbps = ceil_div(total_kb, splits);
-  const int n_wtiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
+#define LASER_GEMM_LAUNCH(E)                                                                                            \
+  if (pair) LASER_TRY((launch_epi<E, true>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, m->status, stream)));  \
+  else LASER_TRY((launch_epi<E, false>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, m->status, stream)));
   switch (epi) {
-    case EPI_PLAIN: LASER_TRY(launch_epi<EPI_PLAIN>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, m->status, stream)); break;
-    case EPI_RESID: LASER_TRY(launch_epi<EPI_RESID>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, m->status, stream)); break;
-    case EPI_SWIGLU: LASER_TRY(launch_epi<EPI_SWIGLU>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, m->status, stream)); break;
-    default: LASER_TRY(launch_epi<EPI_QKV>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, m->status, stream)); break;
+    case EPI_PLAIN: LASER_GEMM_LAUNCH(EPI_PLAIN) break;
+    case EPI_RESID: LASER_GEMM_LAUNCH(EPI_RESID) break;
+    case EPI_SWIGLU: LASER_GEMM_LAUNCH(EPI_SWIGLU) break;
+    default: LASER_GEMM_LAUNCH(EPI_QKV) break;
   }
+#undef LASER_GEMM_LAUNCH
   count_launch();
   return LASER_OK;
 }
