@@ -436,7 +436,35 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   __syncthreads();
   if (splits > 1) cluster_sync_all();  // every partial tile of the cluster is staged
 
-  if (warp >= 2) {
+  if (warp == 0 && lane == 0 && !abort_flag) {
+    // Warm the L2 with the head of the next kernel's weights while the epilogue runs.
+    const unsigned worker = blockIdx.x + gridDim.x * blockIdx.y, n_workers = gridDim.x * gridDim.y;
+    prefetch_l2(e.next_w, e.next_bytes, worker, n_workers);
+    prefetch_l2(e.next_w2, e.next_bytes2, worker, n_workers);
+  }
+  __syncwarp();
+  if ((EPI == EPI_SWIGLU || EPI == EPI_PLAIN) && splits == 1) {
+    // part 3 without partial tiles to sum or operands to prefetch: all six warps finish rows,
+    // in wide groups whose loads are issued first.
+    constexpr int kWide = 12;
+    for (int jb = warp * kWide; jb < NT; jb += (kTcThreads / 32) * kWide) {
+      float4 acc[kWide];
+#pragma unroll
+      for (int b = 0; b < kWide; ++b) {
+        const int j = min(jb + b, NT - 1);
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
+                     : "=f"(acc[b].x), "=f"(acc[b].y), "=f"(acc[b].z), "=f"(acc[b].w) : "r"(tiles + uint32_t((j * kBM + 4 * lane) * 4)));
+      }
+#pragma unroll
+      for (int b = 0; b < kWide; ++b) {
+        const int j = min(jb + b, NT - 1), r = r0 + j;
+        const bool live = jb + b < NT && r < e.R_rows && !(abort_flag);
+        const float rstd = s_rstd[j];
+        if (EPI == EPI_PLAIN) epi_plain(e, lc, r, live, acc[b], rstd, N);
+        else epi_swiglu(e, r, live, wtile * 64, lane, acc[b], rstd);
+      }
+    }
+  } else if (warp >= 2) {
     // part 3: sum the partial columns this CTA owns (ranks in order 0..splits-1) and finish them.
     // One group = kBatch columns: all partial columns of a group are requested first
     // (independent loads), then summed and finished.  Warp w takes groups w, w+4, w+8, ...
@@ -487,11 +515,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       for (int b = 0; b < kBatch; ++b) fetch_operands(jb + b, g0[b], g1[b]);
       finish_group(jb, g0, g1);
     }
-  } else if (warp == 0 && lane == 0 && !abort_flag) {
-    // Warm the L2 with the head of the next kernel's weights while the epilogue runs.
-    const unsigned worker = blockIdx.x + gridDim.x * blockIdx.y, n_workers = gridDim.x * gridDim.y;
-    prefetch_l2(e.next_w, e.next_bytes, worker, n_workers);
-    prefetch_l2(e.next_w2, e.next_bytes2, worker, n_workers);
   }
   __syncwarp();
   if (splits > 1 || PAIR) cluster_sync_all();  // peers may still be reading this CTA's staged tile or tensor memory
