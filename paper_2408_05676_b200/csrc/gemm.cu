@@ -608,6 +608,10 @@ laser_status prepare(GemmState* st) {
   LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
   LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
   LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
   st->ready = true;
   return LASER_OK;
 }
@@ -620,7 +624,8 @@ int pick_splits(int R_pad, int N, int K, int epi, bool pair) {
   const int n_wtiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
   const int tiles = n_wtiles * tc_shape(R_pad, pair).n_ttiles, total_kb = ceil_div(K, kBK);
   int s = g_force_splits ? g_force_splits : int(208.0 / tiles + 0.5);
-  s = std::max(1, std::min(s, std::min(total_kb, pair ? 4 : 8)));   // a cluster holds 8 CTAs at most
+  // clusters of up to 12 CTAs schedule well (they need the non-portable size attribute), larger ones do not
+  s = std::max(1, std::min(s, std::min(total_kb, pair ? 6 : 8)));
   while (s > 1 && ceil_div(total_kb, s) * (s - 1) >= total_kb) --s;   // no rank without K blocks
   return s;
 }
