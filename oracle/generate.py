@@ -35,8 +35,10 @@ def generate(W: Dict, cfg: Dict, prompts: Sequence[np.ndarray], group_id: Sequen
              pool: Optional[np.ndarray], group_offsets: Optional[np.ndarray], *,
              K: int, n_min: int, n_max: int, max_new: int, mode: int = acc.STRICT,
              topk: int = 2, p: float = 0.1, min_draft: int = 1, max_occ: int = 0,
-             eos_id: int = -1, capacity: Optional[int] = None) -> Dict:
+             eos_id: int = -1, capacity: Optional[int] = None, temp_branches: bool = False) -> Dict:
     """Draft-Then-Verify generation.  pool=None (or K=0) gives plain greedy decoding.
+    temp_branches: the sequence's prompt and the tokens generated so far are searched as a
+    temporary branch beside the pool (Section 3.2).
 
     Returns dict(out=[token lists], steps, drafted, accepted, emitted) where the three
     counters are sums over all decoding steps of all sequences, and trace = per sequence
@@ -61,7 +63,8 @@ def generate(W: Dict, cfg: Dict, prompts: Sequence[np.ndarray], group_id: Sequen
                 g = int(group_id[b])
                 draft, _ = ret.draft_one(pool, int(group_offsets[g]), int(group_offsets[g + 1]),
                                          np.asarray(seqs[b][-n_max:]), K, n_min, n_max,
-                                         min_draft, max_occ)
+                                         min_draft, max_occ,
+                                         np.asarray(seqs[b]) if temp_branches else None)
             rows = np.asarray([seqs[b][-1]] + draft, dtype=np.int32)
             logits = fwd.forward(W, cfg, kv, [b], [rows])[0].to(torch.float32).numpy()
             a, em = acc.accept_one(logits, rows, len(rows), mode, topk, p)

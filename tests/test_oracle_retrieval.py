@@ -154,3 +154,70 @@ def test_min_draft_and_batch_layout():
     offs2 = np.asarray([0, 5, 15], dtype=np.int64)
     d, ln, mn = R.draft_batch(pool, offs2, tails[:1], tl[:1], np.asarray([0], np.int32), 4, 1, 3)
     assert d[0].tolist() == [4, -1, -1, -1] and mn[0] == 2
+
+
+# ---- temporary branches (Section 3.2): the sequence's own text is one more document ----
+TEMP_GOLD = os.path.join(os.path.dirname(__file__), "golden", "retrieval_temp_hand_examples.txt")
+
+
+def _temp_cases():
+    out = []
+    for line in open(TEMP_GOLD):
+        if line.startswith("#") or not line.strip():
+            continue
+        f = [x.strip() for x in line.split("|")]
+        out.append((_ints(f[0]), _ints(f[1]), _ints(f[2]), *map(int, f[3:8]), _ints(f[8]), int(f[9])))
+    return out
+
+
+@pytest.mark.parametrize("case", _temp_cases())
+def test_temp_hand_examples(case):
+    pool, history, tail, K, n_min, n_max, min_draft, max_occ, want, want_n = case
+    pool = np.asarray(pool, dtype=np.int32)
+    d, n = R.draft_one(pool, 0, len(pool), np.asarray(tail), K, n_min, n_max, min_draft, max_occ,
+                       history=np.asarray(history, dtype=np.int32))
+    assert d == want and n == want_n
+
+
+def test_temp_matches_literal_trie():
+    """Inserting the history's windows into the group's trie as one more document and walking
+    the trie gives the same draft as the oracle with `history` (no occurrence cap)."""
+    rng = np.random.default_rng(15)
+    for trial in range(120):
+        vocab = int(rng.integers(2, 6))
+        pool, offs = _random_pool(rng, 2, vocab, 100)
+        K, n_max = int(rng.integers(1, 7)), int(rng.integers(1, 5))
+        n_min = int(rng.integers(1, n_max + 1))
+        for _ in range(12):
+            g = int(rng.integers(0, 2))
+            hist = rng.integers(0, vocab, size=int(rng.integers(1, 40)))
+            root = build_trie(pool, offs[g], offs[g + 1], n_max + K)
+            for i in range(len(hist)):
+                root.insert(hist[i:i + n_max + K].tolist())
+            tail = hist[-int(rng.integers(1, 6)):].tolist()      # the tail is the end of the history
+            want = trie_draft(root, tail, K, n_min, n_max)
+            got = R.draft_one(pool, int(offs[g]), int(offs[g + 1]), np.asarray(tail), K, n_min, n_max, 1, 0,
+                              history=hist)
+            assert got == want, (trial, pool.tolist(), hist.tolist(), tail, K, n_min, n_max)
+
+
+def test_temp_history_first_under_cap_and_reduces_to_plain():
+    rng = np.random.default_rng(16)
+    for trial in range(60):
+        vocab = int(rng.integers(2, 5))
+        pool, offs = _random_pool(rng, 1, vocab, 150)
+        hist = rng.integers(0, vocab, size=30)
+        tail = hist[-3:]
+        # an empty history, or one too short to hold a continuation, changes nothing
+        a = R.draft_one(pool, 0, len(pool), tail, 5, 1, 3, 1, 0)
+        assert R.draft_one(pool, 0, len(pool), tail, 5, 1, 3, 1, 0, history=np.zeros(0, dtype=np.int32)) == a
+        assert R.draft_one(pool, 0, len(pool), tail, 5, 1, 3, 1, 0, history=tail[-1:]) == a
+        # with a cap of one occurrence and a history hit, only the history speaks
+        for n in (3, 2, 1):
+            hocc = R.occurrences(hist.astype(np.int64), 0, len(hist), tail[3 - n:])
+            hocc = hocc[hocc + 1 < len(hist)]
+            if hocc.size:
+                d, nn = R.draft_one(pool, 0, len(pool), tail, 4, n, n, 1, 1, history=hist)
+                p = int(hocc[0])
+                assert nn == n and d == hist[p + 1:p + 1 + 4].tolist()
+                break
