@@ -147,6 +147,23 @@ laser_status laser_draft(const laser_pool* pool, const int32_t* tails, const int
                          const int32_t* group_id, int32_t B, const laser_params* p,
                          int32_t* draft, int32_t* draft_len, int32_t* match_n, void* stream);
 
+/* ---- Draft retrieval with temporary branches (Section 3.2) ---------------------------------
+ * While a text is generated, its prompt and the tokens generated so far belong to the trie as
+ * a temporary branch and leave it when the generation ends.  Same retrieval as laser_draft,
+ * with the sequence's own text searched as one more document: its occurrences of the tail that
+ * still have a following token come first (ascending), the group's follow (ascending), and the
+ * list is cut to p->max_occ, which must lie in 1..64 here; the frequencies of both add up.
+ *   hist      dev int32[B, hist_stride]: row b holds the sequence's text, oldest first, ids >= 0
+ *             (normally it ends with the tail)
+ *   hist_len  dev int32[B], 0..hist_stride
+ * group_id[b] outside the pool's groups searches the history alone.  Nothing is stored in the
+ * pool: the branch lasts as long as the caller keeps passing the buffer.
+ * Errors: as laser_draft; INVALID_ARG also for max_occ outside 1..64. */
+laser_status laser_draft_temp(const laser_pool* pool, const int32_t* tails, const int32_t* tail_len,
+                              const int32_t* group_id, const int32_t* hist, const int32_t* hist_len,
+                              int64_t hist_stride, int32_t B, const laser_params* p,
+                              int32_t* draft, int32_t* draft_len, int32_t* match_n, void* stream);
+
 /* Builds the verify rows from the drafts: tokens[b,0] = last_token[b],
  * tokens[b,1..] = draft[b,:draft_len[b]], rest -1; n_rows[b] = 1 + draft_len[b], or 0
  * where last_token[b] < 0 (inactive slot).  All dev; tokens is [B, K+1]. */

@@ -123,7 +123,8 @@ def draft_batch(pool: np.ndarray, group_offsets: np.ndarray, tails: np.ndarray,
     width = tails.shape[1]
     for b in range(B):
         g = int(group_id[b])
-        lo, hi = int(group_offsets[g]), int(group_offsets[g + 1])
+        # a group id outside the pool searches nothing of the pool (the history alone, if given)
+        lo, hi = (int(group_offsets[g]), int(group_offsets[g + 1])) if 0 <= g < len(group_offsets) - 1 else (0, 0)
         tl = int(tail_len[b])
         d, n = draft_one(pool, lo, hi, tails[b, width - tl:], K, n_min, n_max, min_draft, max_occ,
                          None if histories is None else histories[b])

@@ -57,7 +57,7 @@ class Stats(C.Structure):
 
 
 EXPORTS = ["laser_version", "laser_last_error", "laser_launch_count", "laser_pool_build", "laser_pool_free",
-           "laser_pool_info", "laser_draft", "laser_make_rows", "laser_model_create", "laser_model_free",
+           "laser_pool_info", "laser_draft", "laser_draft_temp", "laser_make_rows", "laser_model_create", "laser_model_free",
            "laser_kv_create", "laser_kv_free", "laser_kv_set_page_table", "laser_kv_set_len",
            "laser_kv_get_len", "laser_kv_set_len_dev", "laser_kv_import", "laser_kv_export",
            "laser_verify_step", "laser_check", "laser_profile_enable", "laser_profile_read", "laser_accept_commit", "laser_accept_commit_noalloc",
@@ -154,6 +154,23 @@ def draft(pool: Pool, tails, tail_len, group_id, params: Params, draft_out=None,
     _chk(lib.laser_draft(pool.handle, _ptr(_dev(tails, torch.int32)), _ptr(_dev(tail_len, torch.int32)),
                          _ptr(_dev(group_id, torch.int32)), C.c_int32(B), C.byref(params),
                          _ptr(draft_out), _ptr(draft_len), _ptr(match_n), _stream(stream)))
+    return draft_out, draft_len, match_n
+
+
+def draft_temp(pool: Pool, tails, tail_len, group_id, hist, hist_len, params: Params, draft_out=None,
+               draft_len=None, match_n=None, stream=None):
+    """laser_draft_temp: hist int32[B, stride] holds each sequence's own text, hist_len int32[B]."""
+    B = tail_len.shape[0]
+    dev = tails.device
+    if draft_out is None:
+        draft_out = torch.empty(B, params.K, dtype=torch.int32, device=dev)
+        draft_len = torch.empty(B, dtype=torch.int32, device=dev)
+        match_n = torch.empty(B, dtype=torch.int32, device=dev)
+    hist = _dev(hist, torch.int32)
+    _chk(lib.laser_draft_temp(pool.handle, _ptr(_dev(tails, torch.int32)), _ptr(_dev(tail_len, torch.int32)),
+                              _ptr(_dev(group_id, torch.int32)), _ptr(hist), _ptr(_dev(hist_len, torch.int32)),
+                              C.c_int64(hist.shape[1] if hist.dim() == 2 else 0), C.c_int32(B), C.byref(params),
+                              _ptr(draft_out), _ptr(draft_len), _ptr(match_n), _stream(stream)))
     return draft_out, draft_len, match_n
 
 

@@ -267,6 +267,114 @@ draft_warp_kernel(PoolView pv, DraftArgs a) {
   if (lane == 0) { a.draft_len[q] = best_len; a.match_n[q] = best_len ? best_n : 0; }
 }
 
+// Temporary branches (Section 3.2): the same retrieval with the sequence's own text (prompt +
+// generated tokens) searched as one more document.  Its occurrences of the tail that still have
+// a following token come first in the occurrence list, the group's follow, and the list is cut
+// to max_occ (1..64).  An occurrence is tagged with bit 31 when it lies in the history.
+struct TempArgs {
+  const int32_t* hist; const int32_t* hist_len; int64_t hist_stride;
+};
+
+__global__ void __launch_bounds__(kDraftWarps * 32)
+draft_temp_kernel(PoolView pv, DraftArgs a, TempArgs t) {
+  __shared__ uint32_t s_occ[kDraftWarps][64];
+  __shared__ int32_t s_tok[kDraftWarps][64];
+  __shared__ int32_t s_cur[kDraftWarps][kMaxK];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int q = blockIdx.x * kDraftWarps + warp;
+  if (q >= a.B) return;
+  int32_t* out = a.draft + size_t(q) * a.K;
+  const int g = a.group_id[q];
+  const bool has_group = g >= 0 && g < pv.G;
+  const int64_t lo = has_group ? pv.goff[g] : 0, hi = has_group ? pv.goff[g + 1] : 0;
+  const int32_t* h = t.hist + size_t(q) * t.hist_stride;
+  const int hl = max(t.hist_len[q], 0);
+  const int cap = a.max_occ;
+  int best_len = 0, best_n = 0;
+  const int tl = min(max(a.tail_len[q], 0), a.n_max);
+  for (int n = tl; n >= a.n_min; --n) {
+    int32_t tn[kMaxN];  // the last n tail tokens, oldest first
+    bool bad = false;
+    uint64_t key = key_begin(g, n);
+    for (int j = 0; j < n; ++j) {
+      tn[j] = a.tails[size_t(q) * a.n_max + a.n_max - n + j];
+      bad |= tn[j] < 0;
+      key = key_push(key, tn[j]);
+    }
+    if (bad) continue;
+    int n_occ = 0;
+    for (int base = 0; base + 1 < hl && n_occ < cap; base += 32) {   // the history, ascending
+      const int idx = base + lane;
+      bool ok = idx >= n - 1 && idx + 1 < hl;
+      for (int j = 0; ok && j < n; ++j) ok = h[idx - n + 1 + j] == tn[j];
+      const unsigned ball = __ballot_sync(0xffffffffu, ok);
+      const int slot = n_occ + __popc(ball & ((1u << lane) - 1));
+      if (ok && slot < 64) s_occ[warp][slot] = uint32_t(idx) | 0x80000000u;
+      n_occ += __popc(ball);
+    }
+    n_occ = min(n_occ, cap);
+    uint32_t start = 0, count = 0;
+    if (has_group && n_occ < cap && probe(pv.table[n], pv.mask[n], key_end(key), lane, start, count)) {
+      const uint32_t* plist = pv.positions[n] + start;
+      for (uint32_t base = 0; base < count && n_occ < cap; base += 32) {   // the group, ascending
+        const uint32_t idx = base + lane;
+        const int64_t p = idx < count ? int64_t(plist[idx]) : -1;
+        const bool ok = idx < count && is_occurrence(pv.tok, lo, hi, p, tn, n);
+        const unsigned ball = __ballot_sync(0xffffffffu, ok);
+        const int slot = n_occ + __popc(ball & ((1u << lane) - 1));
+        if (ok && slot < 64) s_occ[warp][slot] = uint32_t(p);
+        n_occ += __popc(ball);
+      }
+      n_occ = min(n_occ, cap);
+    }
+    if (n_occ == 0) continue;
+    __syncwarp();
+    // greedy highest-frequency walk over both sources
+    const uint32_t e0 = lane < n_occ ? s_occ[warp][lane] : 0u, e1 = lane + 32 < n_occ ? s_occ[warp][lane + 32] : 0u;
+    bool al0 = lane < n_occ, al1 = lane + 32 < n_occ;
+    auto next_token = [&](uint32_t e, int j) -> int32_t {
+      if (e & 0x80000000u) {
+        const int idx = int(e & 0x7fffffffu) + j;
+        return idx < hl ? h[idx] : -1;
+      }
+      const int64_t p = int64_t(e) + j;
+      return p < hi ? pv.tok[p] : -1;
+    };
+    int len = 0;
+    for (int j = 1; j <= a.K; ++j) {
+      const int32_t t0 = al0 ? next_token(e0, j) : -1;
+      const int32_t t1 = al1 ? next_token(e1, j) : -1;
+      al0 = t0 >= 0; al1 = t1 >= 0;
+      if (!__any_sync(0xffffffffu, al0 || al1)) break;
+      s_tok[warp][lane] = t0;
+      s_tok[warp][lane + 32] = t1;
+      __syncwarp();
+      uint32_t c0 = 0, c1 = 0;
+      for (int e = 0; e < n_occ; ++e) {
+        const int32_t x = s_tok[warp][e];
+        c0 += (x == t0); c1 += (x == t1);
+      }
+      unsigned long long cand = 0;
+      if (al0) cand = (uint64_t(c0) << 32) | uint32_t(0x7fffffff - t0);
+      if (al1) cand = max(cand, (unsigned long long)((uint64_t(c1) << 32) | uint32_t(0x7fffffff - t1)));
+      for (int o = 16; o; o >>= 1) cand = max(cand, __shfl_xor_sync(0xffffffffu, cand, o));
+      const int32_t pick = 0x7fffffff - int32_t(uint32_t(cand));
+      if (lane == 0) s_cur[warp][j - 1] = pick;
+      al0 = al0 && t0 == pick; al1 = al1 && t1 == pick;
+      len = j;
+      __syncwarp();
+    }
+    if (len > best_len) {
+      for (int j = lane; j < len; j += 32) out[j] = s_cur[warp][j];
+      best_len = len; best_n = n;
+    }
+    __syncwarp();
+    if (best_len >= max(a.min_draft, 1)) break;
+  }
+  for (int j = best_len + lane; j < a.K; j += 32) out[j] = -1;
+  if (lane == 0) { a.draft_len[q] = best_len; a.match_n[q] = best_len ? best_n : 0; }
+}
+
 // Large-run path: one CTA per query, votes through a shared-memory histogram over the
 // vocabulary.  Occurrences are streamed from the run at every depth; one is alive at depth
 // j if its tokens match the tail and its continuation agrees with the draft so far.
@@ -542,6 +650,35 @@ LASER_API laser_status laser_draft(const laser_pool* pool, const int32_t* tails,
     draft_cta_kernel<<<std::min(B, 296), kBigThreads, smem, stream>>>(pv, a, pool->vocab_bound);
     count_launch();
   }
+  LASER_CUDA(cudaGetLastError());
+  return LASER_OK;
+}
+
+LASER_API laser_status laser_draft_temp(const laser_pool* pool, const int32_t* tails, const int32_t* tail_len,
+                                        const int32_t* group_id, const int32_t* hist, const int32_t* hist_len,
+                                        int64_t hist_stride, int32_t B, const laser_params* p,
+                                        int32_t* draft, int32_t* draft_len, int32_t* match_n, void* stream_) {
+  using namespace laser;
+  LASER_REQUIRE(pool && tails && tail_len && group_id && hist && hist_len && p && draft && draft_len && match_n, "null argument");
+  LASER_REQUIRE(B >= 0 && hist_stride >= 0, "B = %d, hist_stride = %lld", B, (long long)hist_stride);
+  LASER_REQUIRE(p->K >= 1 && p->K <= kMaxK, "K = %d outside [1, %d]", p->K, kMaxK);
+  LASER_REQUIRE(p->n_min >= pool->n_min && p->n_max <= pool->n_max && p->n_min <= p->n_max,
+                "suffix range [%d, %d] outside the pool's [%d, %d]", p->n_min, p->n_max, pool->n_min, pool->n_max);
+  LASER_REQUIRE(p->max_occ >= 1 && p->max_occ <= 64 && p->min_draft >= 0,
+                "max_occ = %d: the temporary-branch draft keeps 1..64 occurrences", p->max_occ);
+  if (B == 0) return LASER_OK;
+  cudaStream_t stream = as_stream(stream_);
+  PoolView pv{};
+  pv.tok = pool->tokens; pv.goff = pool->group_offsets; pv.G = pool->n_groups;
+  for (int n = pool->n_min; n <= pool->n_max; ++n) {
+    pv.table[n] = pool->level[n].table; pv.mask[n] = pool->level[n].mask;
+    pv.positions[n] = pool->level[n].positions;
+  }
+  DraftArgs a{tails, tail_len, group_id, B, p->K, p->n_min, p->n_max, p->min_draft, p->max_occ,
+              draft, draft_len, match_n, nullptr};
+  TempArgs t{hist, hist_len, hist_stride};
+  draft_temp_kernel<<<ceil_div(B, kDraftWarps), kDraftWarps * 32, 0, stream>>>(pv, a, t);
+  count_launch();
   LASER_CUDA(cudaGetLastError());
   return LASER_OK;
 }

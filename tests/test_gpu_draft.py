@@ -111,3 +111,92 @@ def test_rejects_bad_arguments(L):
     t = dev_i32(np.zeros((1, 4)))
     with pytest.raises(L.LaserError):
         L.draft(h, t, dev_i32([4]), dev_i32([0]), L.make_params(K=4, n_min=1, n_max=4))
+
+
+# ---- temporary branches: laser_draft_temp against the oracle with `history` ------------------
+def _compare_temp(L, pool, pool_np, offs, tails, tail_len, gid, hists, K, n_min, n_max, min_draft, max_occ):
+    B = len(tail_len)
+    stride = max(1, max(len(h) for h in hists))
+    hist = np.zeros((B, stride), np.int32)
+    hl = np.zeros(B, np.int32)
+    for b, h in enumerate(hists):
+        hist[b, :len(h)] = h
+        hl[b] = len(h)
+    prm = L.make_params(K=K, n_min=n_min, n_max=n_max, min_draft=min_draft, max_occ=max_occ)
+    d, dl, mn = L.draft_temp(pool, dev_i32(tails), dev_i32(tail_len), dev_i32(gid), dev_i32(hist), dev_i32(hl), prm)
+    torch.cuda.synchronize()
+    wd, wl, wn = R.draft_batch(pool_np, offs, tails, tail_len, gid, K, n_min, n_max, min_draft, max_occ,
+                               histories=hists)
+    assert (dl.cpu().numpy() == wl).all()
+    assert (mn.cpu().numpy() == wn).all()
+    assert (d.cpu().numpy() == wd).all()
+    return wl
+
+
+def test_temp_hand_examples(L):
+    gold = os.path.join(os.path.dirname(__file__), "golden", "retrieval_temp_hand_examples.txt")
+    ints = lambda s: [int(x) for x in s.split(",")] if s else []
+    for line in open(gold):
+        if line.startswith("#") or not line.strip():
+            continue
+        f = [x.strip() for x in line.split("|")]
+        pool_np, hist, tail = np.asarray(ints(f[0]), np.int32), np.asarray(ints(f[1]), np.int32), ints(f[2])
+        K, n_min, n_max, min_draft, max_occ = map(int, f[3:8])
+        max_occ = max_occ or 64              # the kernel keeps 1..64 occurrences; the examples have fewer
+        tails = np.full((1, n_max), -1, np.int32)
+        t = tail[-n_max:]
+        tails[0, n_max - len(t):] = t
+        offs = np.asarray([0, len(pool_np)], np.int64)
+        pool = L.pool_build(pool_np, offs, n_min, n_max)
+        wl = _compare_temp(L, pool, pool_np, offs, tails, np.asarray([len(t)], np.int32), np.zeros(1, np.int32),
+                           [hist], K, n_min, n_max, min_draft, max_occ)
+        assert wl[0] == len(ints(f[8]))
+        pool.free()
+
+
+@pytest.mark.parametrize("vocab,max_occ,seed", [(3, 64, 11), (4, 3, 12), (6, 1, 13), (40, 64, 14)])
+def test_temp_random(L, vocab, max_occ, seed):
+    """Histories of ragged lengths (empty, shorter than the tail, longer than a warp's sweep) that end
+    with the tail, tiny vocabularies so that history and pool both match, capped lists."""
+    rng = np.random.default_rng(seed)
+    G = 4
+    toks, offs = [], [0]
+    for g in range(G):
+        ln = int(rng.integers(1, 900))
+        t = rng.integers(0, vocab, size=ln)
+        t[rng.random(ln) < 0.05] = -1
+        toks.extend(t.tolist())
+        offs.append(len(toks))
+    pool_np, offs = np.asarray(toks, np.int32), np.asarray(offs, np.int64)
+    n_min, n_max, K = 1, 4, 8
+    pool = L.pool_build(pool_np, offs, n_min, n_max)
+    B = 150
+    hists, tails, tl = [], np.full((B, n_max), -1, np.int32), np.zeros(B, np.int32)
+    for b in range(B):
+        hl = int(rng.choice([0, 1, 2, 3, 7, 33, 64, 65, 200, 700]))
+        h = rng.integers(0, vocab, size=hl).astype(np.int32)
+        if hl >= 12 and rng.random() < 0.6:      # plant a repeat so the history itself matches
+            h[-4:] = h[hl // 2 - 4:hl // 2]
+        hists.append(h)
+        if rng.random() < 0.8 and hl > 0:
+            t = h[-n_max:]
+        else:                                     # a tail that is not the end of the history
+            t = rng.integers(0, vocab, size=int(rng.integers(0, n_max + 1))).astype(np.int32)
+        tails[b, n_max - len(t):] = t
+        tl[b] = len(t)
+    gid = rng.integers(0, G, size=B).astype(np.int32)
+    gid[::17] = -1                                # no group: the history alone
+    for min_draft in (1, 4):
+        wl = _compare_temp(L, pool, pool_np, offs, tails, tl, gid, hists, K, n_min, n_max, min_draft, max_occ)
+    assert (wl > 0).mean() > 0.3
+    pool.free()
+
+
+def test_temp_rejects_uncapped(L):
+    pool_np, offs = np.asarray([1, 2, 3], np.int32), np.asarray([0, 3], np.int64)
+    pool = L.pool_build(pool_np, offs, 1, 2)
+    z = dev_i32(np.zeros((1, 2), np.int32))
+    one = dev_i32(np.zeros(1, np.int32))
+    with pytest.raises(L.LaserError):
+        L.draft_temp(pool, z, one, one, z, one, L.make_params(K=4, n_min=1, n_max=2, max_occ=0))
+    pool.free()
