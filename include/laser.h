@@ -95,6 +95,8 @@ typedef struct {
   /* generation loop */
   int32_t max_new;    /* tokens to generate per sequence                                   */
   int32_t eos_id;     /* stop after emitting this token; -1 = none                         */
+  int32_t temp_branches; /* laser_generate: non-zero = also draft from the sequence's own prompt and
+                            generated tokens (temporary branch, Section 3.2; needs max_occ in 1..64) */
 } laser_params;
 
 typedef struct {

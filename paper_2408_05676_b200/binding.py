@@ -45,7 +45,7 @@ class Weights(C.Structure):
 
 class Params(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("K", "n_min", "n_max", "min_draft", "max_occ", "mode", "topk")] + \
-               [("p", C.c_float), ("max_new", C.c_int32), ("eos_id", C.c_int32)]
+               [("p", C.c_float), ("max_new", C.c_int32), ("eos_id", C.c_int32), ("temp_branches", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -99,8 +99,8 @@ def _stream(stream) -> C.c_void_p:
 
 
 def make_params(K=8, n_min=1, n_max=4, min_draft=1, max_occ=64, mode=MODE_STRICT, topk=2, p=0.1,
-                max_new=0, eos_id=-1) -> Params:
-    return Params(K, n_min, n_max, min_draft, max_occ, mode, topk, p, max_new, eos_id)
+                max_new=0, eos_id=-1, temp_branches=0) -> Params:
+    return Params(K, n_min, n_max, min_draft, max_occ, mode, topk, p, max_new, eos_id, temp_branches)
 
 
 def version() -> str:

@@ -118,6 +118,7 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
   LASER_REQUIRE(p->K == m->cfg.max_draft, "params K = %d differs from the model's max_draft = %d", p->K, m->cfg.max_draft);
   LASER_REQUIRE(p->max_new >= 1, "max_new = %d", p->max_new);
   LASER_REQUIRE(pool == nullptr || (p->K >= 1 && p->n_max >= 1 && p->n_max <= 8), "drafting needs K >= 1 and n_max in [1, 8]");
+  LASER_REQUIRE(!p->temp_branches || pool != nullptr, "temporary branches are drafted beside a pool");
   cudaStream_t stream = as_stream(stream_);
   const int K = p->K, Rs = K + 1, n_max = pool ? p->n_max : 1;
   int max_prompt = 0;
@@ -202,7 +203,12 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
     step_prep_kernel<<<ceil_div(B, 128), 128, 0, stream>>>(g, B, n_max, tails, tail_len, last);
     count_launch();
     if (pool) {
-      LASER_TRY(laser_draft(pool, tails, tail_len, gid, B, p, draft, draft_len, match_n, stream));
+      // temporary branch: the sequence's prompt and generated tokens (seq_tok) are searched as well
+      if (p->temp_branches)
+        LASER_TRY(laser_draft_temp(pool, tails, tail_len, gid, g.seq_tok, g.seq_len, g.max_total, B, p, draft, draft_len,
+                                   match_n, stream));
+      else
+        LASER_TRY(laser_draft(pool, tails, tail_len, gid, B, p, draft, draft_len, match_n, stream));
     } else {
       no_draft_kernel<<<ceil_div(B * std::max(K, 1), 128), 128, 0, stream>>>(B, K, draft, draft_len);
       count_launch();

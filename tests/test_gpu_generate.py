@@ -52,7 +52,7 @@ def setup(L):
     return cfg, Wc, m, kv, pool, offs, prompts
 
 
-def _teacher_forced(cfg, Wc, pool, offs, prompts, gid, out, prm, mode, k, p):
+def _teacher_forced(cfg, Wc, pool, offs, prompts, gid, out, prm, mode, k, p, temp=False):
     """Replays the library's committed tokens through the oracle.  Every step the oracle drafts
     and verifies from the library's own history; its emitted tokens must equal the library's
     next tokens unless the deciding logits are within NEAR_TIE."""
@@ -65,7 +65,7 @@ def _teacher_forced(cfg, Wc, pool, offs, prompts, gid, out, prm, mode, k, p):
         while at < len(out[b]):
             lo, hi = int(offs[gid[b]]), int(offs[gid[b] + 1])
             d, _ = R.draft_one(pool, lo, hi, np.asarray(seq[-prm.n_max:]), prm.K, prm.n_min, prm.n_max,
-                               prm.min_draft, prm.max_occ)
+                               prm.min_draft, prm.max_occ, np.asarray(seq) if temp else None)
             rows = np.asarray([seq[-1]] + d, np.int32)
             lg = O.forward(Wc, cfg, kvo, [0], [rows])[0].float().numpy()
             a, em = A.accept_one(lg, rows, len(rows), mode, k, p)
@@ -127,6 +127,33 @@ def test_relaxed_matches_oracle_under_teacher_forcing(L, setup):
                                          float(np.float32(p_low)))
     print("relaxed: steps", steps, "exact", exact, "near-tie", near)
     assert near <= max(2, steps // 10)
+
+
+def test_temporary_branches(L, setup):
+    """Drafting also from the sequence's own prompt + generated text: still lossless under strict
+    verification, every step agrees with the oracle's (history included), and prompts that hold
+    their own continuation are drafted from it although their group knows nothing of it."""
+    cfg, Wc, m, kv, pool, offs, prompts = setup
+    h = L.pool_build(pool, offs, 1, 3)
+    # sequence b's prompt: a fresh prefix, then what the model generates after it, then the prefix's
+    # end again -- the history then matches the tail from the first step on
+    base = [synth.make_prompt(24, cfg["vocab"], 3000 + b) for b in range(4)]
+    cont = L.generate(m, kv, None, base, [0] * 4, L.make_params(K=8, max_new=24))["out"]
+    tprompts = [np.concatenate([base[b], np.asarray(cont[b], np.int32), base[b][-6:]]) for b in range(4)]
+    gid = [3, 2, 1, 0]
+    greedy = L.generate(m, kv, None, tprompts, gid, L.make_params(K=8, max_new=48))
+    prm = L.make_params(K=8, n_min=1, n_max=3, max_occ=64, max_new=48, temp_branches=1)
+    plain = L.generate(m, kv, h, tprompts, gid, L.make_params(K=8, n_min=1, n_max=3, max_occ=64, max_new=48))
+    temp = L.generate(m, kv, h, tprompts, gid, prm)
+    assert temp["out"] == greedy["out"] and temp["emitted"] == 4 * 48          # lossless
+    assert temp["drafted"] > plain["drafted"]                                  # the history adds drafts
+    exact, near, steps = _teacher_forced(cfg, Wc, pool, offs, tprompts, gid, temp["out"], prm, A.STRICT, 1, 0.0,
+                                         temp=True)
+    print("temp: steps", steps, "exact", exact, "near-tie", near, "drafted", temp["drafted"], "plain", plain["drafted"],
+          "accepted", temp["accepted"])
+    assert near <= max(2, steps // 20)
+    with pytest.raises(L.LaserError):      # the temporary-branch draft keeps a capped occurrence list
+        L.generate(m, kv, h, tprompts, gid, L.make_params(K=8, n_min=1, n_max=3, max_occ=0, max_new=8, temp_branches=1))
 
 
 def test_eos_and_argument_checks(L, setup):
