@@ -6,9 +6,11 @@ The paper treats the target model M as a black box; the model here is the
 Llama-style decoder the workloads name: RMSNorm, rotary position embedding
 (rotate-half pairing of feature i with i + head_dim/2), causal attention scaled by
 1/sqrt(head_dim), SwiGLU feed-forward, no biases, separate embedding and LM head.
-The pseudo-sequence is a chain, so the mask M_t is causal and the position ids
-P_t are consecutive: row i of a sequence with ctx cached tokens sits at position
-ctx + i and attends to the cache [0, ctx) and to rows 0..i of the same step.
+For a chain pseudo-sequence the mask M_t is causal and the position ids P_t are
+consecutive: row i of a sequence with ctx cached tokens sits at position ctx + i and
+attends to the cache [0, ctx) and to rows 0..i of the same step.  For a token tree
+(Section 3.3, `parents` given) row i sits at position ctx + depth(i), attends to the
+cache and to its ancestors and itself, and its K and V still go to cache slot ctx + i.
 
 Arithmetic: everything in fp64 except what the data contract fixes - weights are
 bf16 values, and K and V are rounded to bf16 (round-to-nearest-even) when they
@@ -17,7 +19,7 @@ interface says fp32.
 """
 from __future__ import annotations
 
-from typing import Dict, List, Sequence
+from typing import Dict, List, Optional, Sequence
 
 import numpy as np
 import torch
@@ -62,21 +64,36 @@ def _r(x: torch.Tensor, mirror: bool) -> torch.Tensor:
 
 
 def forward(W: Dict, cfg: Dict, kv: KVCache, seq_ids: Sequence[int],
-            tokens: Sequence[np.ndarray], mirror_bf16: bool = False) -> List[torch.Tensor]:
+            tokens: Sequence[np.ndarray], mirror_bf16: bool = False,
+            parents: Optional[Sequence[Sequence[int]]] = None) -> List[torch.Tensor]:
     """One forward over the new rows of each listed sequence.
 
     tokens[j] holds the rows of sequence seq_ids[j]: the pending token followed by its
     drafts (or a prompt chunk).  K and V of every row are written to the cache at
     positions ctx .. ctx + rows - 1; kv.ctx itself is not changed (committing is the
     acceptance step's job).  Returns one fp64 logits tensor [rows, vocab] per sequence.
+    parents[j][i-1] (optional) = row of row i's parent in sequence j's token tree (row 0 is the
+    root); without it the rows are a chain.
     """
     H, Hkv, dh = cfg["n_heads"], cfg["n_kv_heads"], cfg["head_dim"]
     eps, theta = cfg["rms_eps"], cfg["rope_theta"]
     rows = [len(t) for t in tokens]
     starts = np.concatenate([[0], np.cumsum(rows)]).astype(int)
     flat = torch.as_tensor(np.concatenate([np.asarray(t, dtype=np.int64) for t in tokens]))
-    pos = torch.cat([torch.arange(r, dtype=torch.int64) + int(kv.ctx[s])
-                     for s, r in zip(seq_ids, rows)])
+    anc: List[List[List[int]]] = []      # per sequence, per row: the rows it sees (ancestors and itself)
+    dep: List[List[int]] = []
+    for j, r in enumerate(rows):
+        par = [i - 1 for i in range(1, r)] if parents is None else [int(x) for x in parents[j][:max(r - 1, 0)]]
+        d, a = [0] * r, [[0]] * r if r else []
+        for i in range(1, r):
+            if not 0 <= par[i - 1] < i:
+                raise ValueError("a parent must be an earlier row")
+            d[i] = d[par[i - 1]] + 1
+            a[i] = a[par[i - 1]] + [i]
+        dep.append(d)
+        anc.append(a)
+    pos = torch.cat([torch.as_tensor(dep[j], dtype=torch.int64) + int(kv.ctx[s])
+                     for j, s in enumerate(seq_ids)])
     for s, r in zip(seq_ids, rows):
         if kv.ctx[s] + r > kv.capacity:
             raise ValueError("KV capacity exceeded")
@@ -95,10 +112,10 @@ def forward(W: Dict, cfg: Dict, kv: KVCache, seq_ids: Sequence[int],
             a, b, c = starts[j], starts[j + 1], int(kv.ctx[s])
             kv.k[l, s, c:c + rows[j]] = k[a:b]
             kv.v[l, s, c:c + rows[j]] = v[a:b]
-            for i in range(rows[j]):                          # row i sees cache + rows 0..i
-                n = c + i + 1
-                kk = kv.k[l, s, :n].to(F64).repeat_interleave(rep, dim=1)   # [n, H, dh]
-                vv = kv.v[l, s, :n].to(F64).repeat_interleave(rep, dim=1)
+            for i in range(rows[j]):                          # row i sees the cache + its ancestors + itself
+                see = list(range(c)) + [c + r_ for r_ in anc[j][i]]
+                kk = kv.k[l, s, see].to(F64).repeat_interleave(rep, dim=1)   # [n, H, dh]
+                vv = kv.v[l, s, see].to(F64).repeat_interleave(rep, dim=1)
                 sc = torch.einsum("hd,nhd->hn", q[a + i], kk) / (dh ** 0.5)
                 pr = torch.softmax(sc, dim=-1)
                 att[a + i] = torch.einsum("hn,nhd->hd", pr, vv)

@@ -20,6 +20,7 @@ import torch
 from . import accept as acc
 from . import forward as fwd
 from . import retrieval as ret
+from . import tree as tr
 
 
 def prefill(W: Dict, cfg: Dict, kv: fwd.KVCache, seq: int, prompt: np.ndarray, chunk: int = 64) -> None:
@@ -35,10 +36,13 @@ def generate(W: Dict, cfg: Dict, prompts: Sequence[np.ndarray], group_id: Sequen
              pool: Optional[np.ndarray], group_offsets: Optional[np.ndarray], *,
              K: int, n_min: int, n_max: int, max_new: int, mode: int = acc.STRICT,
              topk: int = 2, p: float = 0.1, min_draft: int = 1, max_occ: int = 0,
-             eos_id: int = -1, capacity: Optional[int] = None, temp_branches: bool = False) -> Dict:
+             eos_id: int = -1, capacity: Optional[int] = None, temp_branches: bool = False,
+             tree: bool = False) -> Dict:
     """Draft-Then-Verify generation.  pool=None (or K=0) gives plain greedy decoding.
     temp_branches: the sequence's prompt and the tokens generated so far are searched as a
     temporary branch beside the pool (Section 3.2).
+    tree: draft a token tree of up to K nodes and verify it with tree attention (Section 3.3); the
+    accepted path's K and V move from their rows' cache slots to consecutive positions.
 
     Returns dict(out=[token lists], steps, drafted, accepted, emitted) where the three
     counters are sums over all decoding steps of all sequences, and trace = per sequence
@@ -59,15 +63,29 @@ def generate(W: Dict, cfg: Dict, prompts: Sequence[np.ndarray], group_id: Sequen
             if done[b]:
                 continue
             draft: List[int] = []
+            par: List[int] = []
             if pool is not None and K > 0:
                 g = int(group_id[b])
-                draft, _ = ret.draft_one(pool, int(group_offsets[g]), int(group_offsets[g + 1]),
-                                         np.asarray(seqs[b][-n_max:]), K, n_min, n_max,
-                                         min_draft, max_occ,
-                                         np.asarray(seqs[b]) if temp_branches else None)
+                hist = np.asarray(seqs[b]) if temp_branches else None
+                if tree:
+                    draft, par, _ = tr.draft_tree_one(pool, int(group_offsets[g]), int(group_offsets[g + 1]),
+                                                      np.asarray(seqs[b][-n_max:]), K, n_min, n_max,
+                                                      min_draft, max_occ, hist)
+                else:
+                    draft, _ = ret.draft_one(pool, int(group_offsets[g]), int(group_offsets[g + 1]),
+                                             np.asarray(seqs[b][-n_max:]), K, n_min, n_max,
+                                             min_draft, max_occ, hist)
             rows = np.asarray([seqs[b][-1]] + draft, dtype=np.int32)
-            logits = fwd.forward(W, cfg, kv, [b], [rows])[0].to(torch.float32).numpy()
-            a, em = acc.accept_one(logits, rows, len(rows), mode, topk, p)
+            if tree:
+                logits = fwd.forward(W, cfg, kv, [b], [rows], parents=[par])[0].to(torch.float32).numpy()
+                a, em, path = tr.accept_tree(logits, rows, par, len(rows), mode, topk, p)
+                c = int(kv.ctx[b])
+                for d, row in enumerate(path, 1):       # ascending: a target slot is never a later source
+                    kv.k[:, b, c + d] = kv.k[:, b, c + row]
+                    kv.v[:, b, c + d] = kv.v[:, b, c + row]
+            else:
+                logits = fwd.forward(W, cfg, kv, [b], [rows])[0].to(torch.float32).numpy()
+                a, em = acc.accept_one(logits, rows, len(rows), mode, topk, p)
             room = max_new - len(out[b])
             em = em[:room]
             if eos_id >= 0 and eos_id in em:
