@@ -216,6 +216,20 @@ laser_status laser_kv_export(const laser_kv* kv, int32_t seq, int32_t layer, int
 laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int32_t* seq_ids,
                                const int32_t* tokens, const int32_t* n_rows, int32_t B,
                                float* logits, void* stream);
+
+/* ---- Verify forward of a token tree (Section 3.3, tree attention) ------------------------------
+ * As laser_verify_step, for a pseudo-sequence that lists a token tree in depth-first order.
+ *   parents  dev int32[B, K+1]: parents[b,i] = row of row i's parent, 0 <= parents[b,i] < i for
+ *            i >= 1; entry [b,0] is not read (row 0, the pending token, is the root)
+ * Row i takes the position ctx + depth(i) (P_t), attends to the cache and to its ancestors and
+ * itself (M_t), and its K and V are written to cache slot ctx + i: after acceptance the
+ * accepted path is moved to consecutive slots (laser_accept_tree, laser_kv_compact_path).
+ * A chain given as parents[b,i] = i - 1 gives laser_verify_step's result.
+ * Errors: as laser_verify_step; INVALID_ARG when K + 1 > 64 or (reported by laser_check) when
+ * a parent is not an earlier row. */
+laser_status laser_verify_step_tree(laser_model* m, laser_kv* kv, const int32_t* seq_ids,
+                                    const int32_t* tokens, const int32_t* parents,
+                                    const int32_t* n_rows, int32_t B, float* logits, void* stream);
 /* Synchronises `stream` and returns the first device-side error recorded since the last
  * check (CAPACITY, TIMEOUT), clearing it. */
 laser_status laser_check(laser_model* m, void* stream);

@@ -60,7 +60,7 @@ EXPORTS = ["laser_version", "laser_last_error", "laser_launch_count", "laser_poo
            "laser_pool_info", "laser_draft", "laser_draft_temp", "laser_make_rows", "laser_model_create", "laser_model_free",
            "laser_kv_create", "laser_kv_free", "laser_kv_set_page_table", "laser_kv_set_len",
            "laser_kv_get_len", "laser_kv_set_len_dev", "laser_kv_import", "laser_kv_export",
-           "laser_verify_step", "laser_check", "laser_profile_enable", "laser_profile_read", "laser_accept_commit", "laser_accept_commit_noalloc",
+           "laser_verify_step", "laser_verify_step_tree", "laser_check", "laser_profile_enable", "laser_profile_read", "laser_accept_commit", "laser_accept_commit_noalloc",
            "laser_generate"]
 
 lib.laser_version.restype = C.c_char_p
@@ -292,6 +292,20 @@ def verify_step(model: Model, kv: KV, seq_ids, tokens, n_rows, logits=None, stre
     _chk(lib.laser_verify_step(model.handle, kv.handle, _ptr(_dev(seq_ids, torch.int32)),
                                _ptr(_dev(tokens, torch.int32)), _ptr(_dev(n_rows, torch.int32)),
                                C.c_int32(B), _ptr(_dev(logits, torch.float32)), _stream(stream)))
+    return logits
+
+
+def verify_step_tree(model: Model, kv: KV, seq_ids, tokens, parents, n_rows, logits=None, stream=None) -> torch.Tensor:
+    """laser_verify_step_tree: parents int32[B, K+1], parents[b, i] = row of row i's parent."""
+    B = seq_ids.shape[0]
+    R = model.cfg["max_draft"] + 1
+    assert tokens.shape == (B, R) and parents.shape == (B, R), (tokens.shape, parents.shape, B, R)
+    if logits is None:
+        logits = torch.empty(B, R, model.cfg["vocab"], dtype=torch.float32, device=tokens.device)
+    _chk(lib.laser_verify_step_tree(model.handle, kv.handle, _ptr(_dev(seq_ids, torch.int32)),
+                                    _ptr(_dev(tokens, torch.int32)), _ptr(_dev(parents, torch.int32)),
+                                    _ptr(_dev(n_rows, torch.int32)), C.c_int32(B), _ptr(_dev(logits, torch.float32)),
+                                    _stream(stream)))
     return logits
 
 

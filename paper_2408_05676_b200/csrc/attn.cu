@@ -45,7 +45,8 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
                   const int32_t* __restrict__ seq_ids, const int32_t* __restrict__ row_ctx,
                   const int32_t* __restrict__ row_n, int Rs, int H, int Hkv,
                   const int32_t* __restrict__ page_table, int pages_per_seq, int layer_row0,
-                  bf16* __restrict__ out, int32_t* __restrict__ status, const void* next_w, size_t next_bytes) {
+                  bf16* __restrict__ out, int32_t* __restrict__ status, const void* next_w, size_t next_bytes,
+                  const unsigned long long* __restrict__ row_mask) {
   constexpr int HALVES = DH / 64;                 // 64-element (128-byte) column blocks per row
   constexpr int SUB = 16 * 128;                   // bytes of one 16-token x 64-element sub-tile
   constexpr int STAGE = 2 * HALVES * SUB;         // K then V
@@ -138,6 +139,9 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
   // last key each of this lane's two rows may see; inactive rows copy the last active row
   const int lim0 = ctx + min(row0 + g, nr - 1), lim1 = ctx + min(row0 + g + 8, nr - 1);
+  // token tree: of the step's own rows a row sees those of its mask (ancestors and itself)
+  const unsigned long long vis0 = row_mask ? row_mask[size_t(b) * Rs + min(row0 + g, nr - 1)] : 0ull;
+  const unsigned long long vis1 = row_mask ? row_mask[size_t(b) * Rs + min(row0 + g + 8, nr - 1)] : 0ull;
 
   for (int p = warp; p < n_pg; p += kConsumers) {
     const int s = p % kStages;
@@ -166,8 +170,14 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         const int key = key0 + t * 8 + c;
-        if (key > lim0) sc[t][c] = -INFINITY;
-        if (key > lim1) sc[t][2 + c] = -INFINITY;
+        if (row_mask) {
+          const int rel = key - ctx;   // >= 0: one of this step's rows (or the padding of the last page)
+          if (rel >= 0 && (rel >= 64 || !((vis0 >> rel) & 1ull))) sc[t][c] = -INFINITY;
+          if (rel >= 0 && (rel >= 64 || !((vis1 >> rel) & 1ull))) sc[t][2 + c] = -INFINITY;
+        } else {
+          if (key > lim0) sc[t][c] = -INFINITY;
+          if (key > lim1) sc[t][2 + c] = -INFINITY;
+        }
         mx0 = fmaxf(mx0, sc[t][c]);
         mx1 = fmaxf(mx1, sc[t][2 + c]);
       }
@@ -247,7 +257,7 @@ bool attention_tma_supported(const laser_model* m, const laser_kv* kv) {
   return kv->has_pages_map && (m->cfg.head_dim == 64 || m->cfg.head_dim == 128);
 }
 
-laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const int32_t* seq_ids, int B,
+laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const int32_t* seq_ids, int B, bool tree,
                                   const void* next_w, size_t next_bytes, cudaStream_t stream) {
   const int dh = m->cfg.head_dim, H = m->cfg.n_heads, Hkv = m->cfg.n_kv_heads, Rs = m->rows_per_seq;
   const int64_t rows_per_layer = int64_t(kv->n_pages) * 2 * Hkv * 16;
@@ -265,14 +275,15 @@ laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const
   cfg.numAttrs = 1;
   const __nv_bfloat16* q = m->q;
   const int32_t *rc = m->row_ctx, *rn = m->row_n, *pt = kv->page_table;
+  const unsigned long long* mask = tree ? m->row_mask : nullptr;
   if (dh == 128) {
     LASER_CUDA(cudaFuncSetAttribute(attn_paged_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     LASER_CUDA(cudaLaunchKernelEx(&cfg, attn_paged_kernel<128>, kv->pages_map, q, seq_ids, rc, rn, Rs, H, Hkv, pt,
-                                  kv->pages_per_seq, layer_row0, m->attn, m->status, next_w, next_bytes));
+                                  kv->pages_per_seq, layer_row0, m->attn, m->status, next_w, next_bytes, mask));
   } else {
     LASER_CUDA(cudaFuncSetAttribute(attn_paged_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     LASER_CUDA(cudaLaunchKernelEx(&cfg, attn_paged_kernel<64>, kv->pages_map, q, seq_ids, rc, rn, Rs, H, Hkv, pt,
-                                  kv->pages_per_seq, layer_row0, m->attn, m->status, next_w, next_bytes));
+                                  kv->pages_per_seq, layer_row0, m->attn, m->status, next_w, next_bytes, mask));
   }
   count_launch();
   LASER_CUDA(cudaGetLastError());

@@ -18,8 +18,11 @@ using bf16 = __nv_bfloat16;
 constexpr size_t kL2PrefetchBytes = size_t(48) << 20;
 
 // ---- row bookkeeping -------------------------------------------------------------------
-// One thread per row: position, cache slot, capacity check, rotary angles (fp64 -> fp32).
+// One block per row: position, cache slot, capacity check, rotary angles (fp64 -> fp32).
+// With `parents` (token tree, Section 3.3) a row's position is ctx + its depth, its cache slot
+// stays ctx + row index, and row_mask gets the rows it attends to (its ancestors and itself).
 __global__ void prep_rows_kernel(const int32_t* __restrict__ seq_ids, const int32_t* __restrict__ n_rows,
+                                 const int32_t* __restrict__ parents, unsigned long long* __restrict__ row_mask,
                                  int B, int Rs, int R_pad, const int32_t* __restrict__ seq_len,
                                  int max_seqs, int capacity, int half, double theta, int head_dim,
                                  int32_t* __restrict__ row_pos, int32_t* __restrict__ row_seq,
@@ -28,6 +31,9 @@ __global__ void prep_rows_kernel(const int32_t* __restrict__ seq_ids, const int3
   const int r = blockIdx.x;
   const int b = r / Rs, i = r % Rs;
   int pos = -1, seq = 0;
+  __shared__ int s_rpos;
+  int rpos = 0;                      // position the rotary embedding uses
+  unsigned long long mask = 0ull;
   if (r < B * Rs) {
     seq = seq_ids[b];
     int nr = min(max(n_rows[b], 0), Rs);
@@ -43,13 +49,28 @@ __global__ void prep_rows_kernel(const int32_t* __restrict__ seq_ids, const int3
       }
     }
     if (i < nr) pos = ctx + i;
+    rpos = max(pos, 0);
+    if (parents && i < nr && threadIdx.x == 0) {
+      int depth = 0, j = i;
+      mask = 1ull << i;
+      while (j > 0) {                // parents are earlier rows: at most i steps
+        const int pj = parents[b * Rs + j];
+        if (pj < 0 || pj >= j) { atomicCAS(status, 0, LASER_ERR_INVALID_ARG); break; }
+        j = pj;
+        mask |= 1ull << j;
+        ++depth;
+      }
+      rpos = ctx + depth;
+    }
     if (i == 0 && threadIdx.x == 0) { row_ctx[b] = ctx; row_n[b] = nr; }
   }
-  if (threadIdx.x == 0) { row_pos[r] = pos; row_seq[r] = seq; }
+  if (threadIdx.x == 0) { row_pos[r] = pos; row_seq[r] = seq; s_rpos = rpos; if (row_mask) row_mask[r] = mask; }
+  __syncthreads();
+  rpos = s_rpos;
   for (int j = threadIdx.x; j < half; j += blockDim.x) {
     const double inv_freq = pow(theta, -2.0 * double(j) / double(head_dim));
     double s, c;
-    sincos(double(max(pos, 0)) * inv_freq, &s, &c);
+    sincos(double(rpos) * inv_freq, &s, &c);
     rope[(size_t(r) * half + j) * 2] = float(c);
     rope[(size_t(r) * half + j) * 2 + 1] = float(s);
   }
@@ -94,7 +115,8 @@ __global__ void __launch_bounds__(128)
 attention_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ seq_ids,
                  const int32_t* __restrict__ row_ctx, const int32_t* __restrict__ row_n, int Rs, int H,
                  int Hkv, int dh, const int32_t* __restrict__ page_table, int pages_per_seq,
-                 const bf16* __restrict__ pages_layer, size_t page_elems, bf16* __restrict__ out) {
+                 const bf16* __restrict__ pages_layer, size_t page_elems, bf16* __restrict__ out,
+                 const unsigned long long* __restrict__ row_mask) {
   extern __shared__ float smem[];
   float* s_q = smem;            // [dh]
   float* s_sc = smem + dh;      // [ctx + rows]
@@ -114,7 +136,9 @@ attention_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ seq_ids
     __syncthreads();
     for (int d = tid; d < dh; d += 128) s_q[d] = __bfloat162float(q[r * H * dh + size_t(h) * dh + d]) * scale;
     __syncthreads();
-    const int n = ctx + i + 1;
+    // chain: the cache and rows 0..i; token tree: the cache and the rows of the mask
+    const int n = row_mask ? ctx + nr : ctx + i + 1;
+    const unsigned long long vis = row_mask ? row_mask[r] : ~0ull;
     float mx = -INFINITY;
     for (int j = tid; j < n; j += 128) {
       const bf16* kp = pages_layer + size_t(pt[j / 16]) * page_elems + size_t(hk) * 16 * dh + size_t(j % 16) * dh;
@@ -125,6 +149,7 @@ attention_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ seq_ids
 #pragma unroll
         for (int x = 0; x < 8; ++x) s += s_q[d + x] * __bfloat162float(e[x]);
       }
+      if (j >= ctx && !((vis >> (j - ctx)) & 1ull)) s = -INFINITY;
       s_sc[j] = s;
       mx = fmaxf(mx, s);
     }
@@ -305,6 +330,7 @@ LASER_API laser_status laser_model_create(const laser_model_cfg* cfg, const lase
   LASER_TRY(model_alloc(m, &m->row_seq, Rp));
   LASER_TRY(model_alloc(m, &m->row_ctx, size_t(cfg->max_batch)));
   LASER_TRY(model_alloc(m, &m->row_n, size_t(cfg->max_batch)));
+  LASER_TRY(model_alloc(m, &m->row_mask, size_t(m->R_pad)));
   LASER_TRY(model_alloc(m, &m->status, size_t(1)));
   guard.p = nullptr;
   *out = m;
@@ -428,8 +454,24 @@ LASER_API laser_status laser_check(laser_model* m, void* stream) {
   return LASER_OK;
 }
 
+static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
+                                const int32_t* parents, const int32_t* n_rows, int32_t B, float* logits, void* stream_);
+
 LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
-                                         const int32_t* n_rows, int32_t B, float* logits, void* stream_) {
+                                         const int32_t* n_rows, int32_t B, float* logits, void* stream) {
+  return verify_impl(m, kv, seq_ids, tokens, nullptr, n_rows, B, logits, stream);
+}
+
+LASER_API laser_status laser_verify_step_tree(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
+                                              const int32_t* parents, const int32_t* n_rows, int32_t B, float* logits,
+                                              void* stream) {
+  LASER_REQUIRE(parents, "null argument");
+  LASER_REQUIRE(m && m->rows_per_seq <= 64, "a token tree has at most 64 rows (K + 1 = %d)", m ? m->rows_per_seq : 0);
+  return verify_impl(m, kv, seq_ids, tokens, parents, n_rows, B, logits, stream);
+}
+
+static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
+                                const int32_t* parents, const int32_t* n_rows, int32_t B, float* logits, void* stream_) {
   LASER_REQUIRE(m && kv && seq_ids && tokens && n_rows && logits, "null argument");
   LASER_REQUIRE(B >= 1 && B <= m->cfg.max_batch, "B = %d outside [1, max_batch = %d]", B, m->cfg.max_batch);
   LASER_REQUIRE(kv->n_layers == m->cfg.n_layers && kv->n_kv_heads == m->cfg.n_kv_heads && kv->head_dim == m->cfg.head_dim,
@@ -442,7 +484,8 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
 
   // Every row of the workspace is (re)marked: a GEMM's last token tile may reach past this call's
   // rows, and whatever it finds there must be inactive (no cache write) and finite.
-  prep_rows_kernel<<<m->R_pad, 64, 0, stream>>>(seq_ids, n_rows, B, Rs, Rp, kv->seq_len, kv->max_seqs, capacity, dh / 2,
+  const bool tree = parents != nullptr;
+  prep_rows_kernel<<<m->R_pad, 64, 0, stream>>>(seq_ids, n_rows, parents, tree ? m->row_mask : nullptr, B, Rs, Rp, kv->seq_len, kv->max_seqs, capacity, dh / 2,
                                           double(c.rope_theta), dh, m->row_pos, m->row_seq, m->row_ctx, m->row_n,
                                           m->rope, m->status);
   const __nv_bfloat16* first_gain = c.n_layers > 0 ? m->attn_norm[0] : m->final_norm;
@@ -477,11 +520,11 @@ LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int
     {
       ProfScope ps(m, 1, stream);
       if (use_tma_attn) {
-        LASER_TRY(attention_tma_launch(m, kv, l, seq_ids, B, m->wo[l], head_bytes(size_t(d) * m->dq * 2), stream));
+        LASER_TRY(attention_tma_launch(m, kv, l, seq_ids, B, tree, m->wo[l], head_bytes(size_t(d) * m->dq * 2), stream));
       } else {
         attention_kernel<<<dim3(B, H), 128, attn_smem, stream>>>(m->q, seq_ids, m->row_ctx, m->row_n, Rs, H, Hkv, dh,
                                                                 kv->page_table, kv->pages_per_seq, pages_l,
-                                                                kv->page_elems(), m->attn);
+                                                                kv->page_elems(), m->attn, tree ? m->row_mask : nullptr);
         count_launch();
       }
     }

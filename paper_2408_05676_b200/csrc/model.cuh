@@ -25,6 +25,7 @@ struct laser_model {
   int32_t* row_seq = nullptr;      // [R_pad] cache slot of the row
   int32_t* row_ctx = nullptr;      // [max_batch] committed length of each sequence of the step
   int32_t* row_n = nullptr;        // [max_batch] effective rows of each sequence
+  unsigned long long* row_mask = nullptr;  // [R_pad] token tree: rows of its sequence a row attends to (bit j = row j)
   int32_t* status = nullptr;       // first device-side error of the stream, 0 = none
   void* gemm_state = nullptr;      // tensor-map cache of the tensor-core GEMM
   // optional per-class kernel timing (class 0 = GEMM, 1 = attention)
@@ -83,7 +84,7 @@ void gemm_state_free(laser_model* m);
 // TMA-fed paged attention (head_dim 64 or 128 and a cache small enough for 32-bit row
 // coordinates); the verify forward falls back to a plain kernel otherwise.
 bool attention_tma_supported(const laser_model* m, const laser_kv* kv);
-laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const int32_t* seq_ids, int B,
+laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const int32_t* seq_ids, int B, bool tree,
                                   const void* next_w, size_t next_bytes, cudaStream_t stream);
 
 }  // namespace laser
