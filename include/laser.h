@@ -255,6 +255,31 @@ laser_status laser_accept_commit(laser_kv* kv, const int32_t* seq_ids, const flo
                                  int32_t V, const laser_params* p, int32_t* n_accept,
                                  int32_t* out_tokens, int32_t* n_out, void* stream);
 
+/* ---- Verification of a token tree (Section 3.4: "if a predecessor node is rejected, all of its
+ * successor nodes will be skipped ... ultimately accepting the verified branch with the maximum
+ * length") ---------------------------------------------------------------------------------------
+ * tokens / parents / n_rows as for laser_verify_step_tree, logits its result.  Node i is verified
+ * when its parent is (row 0 always is) and tokens[b,i] passes p->mode on the row of its parent.
+ * The verified node of greatest depth wins, the first in depth-first order among equals.
+ *   n_accept    dev int32[B]       depth of the winner = accepted drafts a
+ *   out_tokens  dev int32[B, K+1]  the a tokens of its path, then arg max of its own row, then -1
+ *   n_out       dev int32[B]       a + 1 (0 for an inactive sequence)
+ *   path_rows   dev int32[B, K+1]  rows of the accepted path, root excluded, then -1
+ * kv non-null: the K and V of the accepted rows move from cache slot len + row to len + 1 .. len + a
+ * and the lengths advance by n_out (laser_kv_compact_path, then the update).  kv null: verdict only.
+ * Errors: INVALID_ARG (K + 1 > 64, mode, topk), OOM, CUDA. */
+laser_status laser_accept_tree(laser_kv* kv, const int32_t* seq_ids, const float* logits,
+                               const int32_t* tokens, const int32_t* parents, const int32_t* n_rows,
+                               int32_t B, int32_t V, const laser_params* p, int32_t* n_accept,
+                               int32_t* out_tokens, int32_t* n_out, int32_t* path_rows, void* stream);
+
+/* Cache compaction after tree verification (Section 3.3: the rows of a tree are not consecutive
+ * positions).  For sequence seq_ids[b] with committed length len: slot len + path_rows[b,j] is
+ * copied to slot len + j + 1 for j = 0 .. n_accept[b]-1, in every layer, K and V.  path_rows is
+ * [B, row_stride], rows ascending (as laser_accept_tree writes them).  Lengths are not changed. */
+laser_status laser_kv_compact_path(laser_kv* kv, const int32_t* seq_ids, const int32_t* path_rows,
+                                   const int32_t* n_accept, int32_t B, int32_t row_stride, void* stream);
+
 /* Same result as laser_accept_commit, for callers that must not allocate device memory.
  * (The paper has no counterpart; this exists for integration.)  Some hosts of this library
  * cannot call cudaMalloc on the decoding path: a serving engine that reserved all of HBM for

@@ -60,7 +60,7 @@ EXPORTS = ["laser_version", "laser_last_error", "laser_launch_count", "laser_poo
            "laser_pool_info", "laser_draft", "laser_draft_temp", "laser_make_rows", "laser_model_create", "laser_model_free",
            "laser_kv_create", "laser_kv_free", "laser_kv_set_page_table", "laser_kv_set_len",
            "laser_kv_get_len", "laser_kv_set_len_dev", "laser_kv_import", "laser_kv_export",
-           "laser_verify_step", "laser_verify_step_tree", "laser_check", "laser_profile_enable", "laser_profile_read", "laser_accept_commit", "laser_accept_commit_noalloc",
+           "laser_verify_step", "laser_verify_step_tree", "laser_check", "laser_profile_enable", "laser_profile_read", "laser_accept_commit", "laser_accept_commit_noalloc", "laser_accept_tree", "laser_kv_compact_path",
            "laser_generate"]
 
 lib.laser_version.restype = C.c_char_p
@@ -352,6 +352,23 @@ def accept_commit(kv: Optional[KV], seq_ids, logits, tokens, n_rows, params: Par
                                  _ptr(_dev(n_rows, torch.int32)), C.c_int32(B), C.c_int32(V), C.byref(params),
                                  _ptr(n_accept), _ptr(out_tokens), _ptr(n_out), _stream(stream)))
     return n_accept, out_tokens, n_out
+
+
+def accept_tree(kv: Optional[KV], seq_ids, logits, tokens, parents, n_rows, params: Params, stream=None):
+    """laser_accept_tree; returns n_accept, out_tokens, n_out, path_rows (device tensors)."""
+    B, R, V = logits.shape
+    dev = logits.device
+    n_accept = torch.empty(B, dtype=torch.int32, device=dev)
+    out_tokens = torch.empty(B, R, dtype=torch.int32, device=dev)
+    n_out = torch.empty(B, dtype=torch.int32, device=dev)
+    path_rows = torch.empty(B, R, dtype=torch.int32, device=dev)
+    _chk(lib.laser_accept_tree(kv.handle if kv is not None else C.c_void_p(0),
+                               _ptr(_dev(seq_ids, torch.int32)) if seq_ids is not None else C.c_void_p(0),
+                               _ptr(_dev(logits, torch.float32)), _ptr(_dev(tokens, torch.int32)),
+                               _ptr(_dev(parents, torch.int32)), _ptr(_dev(n_rows, torch.int32)), C.c_int32(B),
+                               C.c_int32(V), C.byref(params), _ptr(n_accept), _ptr(out_tokens), _ptr(n_out),
+                               _ptr(path_rows), _stream(stream)))
+    return n_accept, out_tokens, n_out, path_rows
 
 
 def generate(model: Model, kv: KV, pool: Optional[Pool], prompts: Sequence[np.ndarray], group_id: Sequence[int],

@@ -107,3 +107,105 @@ def test_bad_parent_is_reported(L):
     L.verify_step_tree(m, kv, dev_i32([0]), dev_i32(tokens), dev_i32(parents), dev_i32([Rs]))
     with pytest.raises(L.LaserError):
         L.check(m)
+
+
+@pytest.mark.parametrize("mode,topk,p", [(A.STRICT, 1, 0.0), (A.RELAXED, 2, 0.1), (A.RELAXED, 3, 0.02),
+                                         (A.TOPK, 2, 0.0), (A.TOPP, 1, 0.3)])
+def test_accept_tree_matches_oracle(L, mode, topk, p):
+    """Bit-exact tree verification on synthesised logits that reach every branch of the rules (exact
+    ties included): random trees whose tokens are the parent row's rank-1/2/3 or random tokens."""
+    from paper_2408_05676_b200.synth import make_accept_case
+    rng = np.random.default_rng(31 + mode)
+    deepest = 0
+    for (B, K, V) in [(37, 8, 1000), (5, 15, 32000), (64, 3, 517), (3, 63, 777)]:
+        logits, _, n_rows = make_accept_case(B, K, V, seed=5 + K)
+        n_rows[0] = K + 1
+        if B > 4:
+            n_rows[3] = 0
+        tokens = rng.integers(0, V, size=(B, K + 1)).astype(np.int32)
+        parents = np.full((B, K + 1), -1, np.int32)
+        for b in range(B):
+            par = random_tree(rng, K) if b % 5 else list(range(K))          # every fifth is a chain
+            parents[b, 1:] = par
+            for i in range(1, K + 1):
+                order = np.argsort(-logits[b, par[i - 1]], kind="stable")
+                c = rng.random()
+                if c < 0.9:
+                    tokens[b, i] = order[0] if c < 0.55 else (order[1] if c < 0.8 else order[2])
+        prm = L.make_params(K=K, mode=mode, topk=topk, p=p)
+        for rep in range(2):        # twice: the arrival counters are left clean
+            na, ot, no, pr = L.accept_tree(None, None, torch.from_numpy(logits).cuda(), dev_i32(tokens), dev_i32(parents),
+                                           dev_i32(n_rows), prm)
+            na, ot, no, pr = na.cpu().numpy(), ot.cpu().numpy(), no.cpu().numpy(), pr.cpu().numpy()
+            for b in range(B):
+                nr = int(n_rows[b])
+                if nr == 0:
+                    assert na[b] == 0 and no[b] == 0 and (ot[b] == -1).all() and (pr[b] == -1).all()
+                    continue
+                a, em, path = T.accept_tree(logits[b], tokens[b], parents[b, 1:nr].tolist(), nr, mode, topk,
+                                            float(np.float32(p)))
+                assert na[b] == a and no[b] == a + 1, (b, na[b], a)
+                assert ot[b, :a + 1].tolist() == em and (ot[b, a + 1:] == -1).all()
+                assert pr[b, :a].tolist() == path and (pr[b, a:] == -1).all()
+        deepest = max(deepest, int(na.max()))
+    assert deepest >= 2
+
+
+def test_tree_step_commits_the_accepted_path(L):
+    """Forward, verification and compaction together: after the commit the cache holds the accepted
+    path at consecutive positions, as the oracle's does, and a following plain step agrees."""
+    cfg = synth.model_cfg("tiny")
+    Wc = synth.make_weights(cfg, seed=0, gain_jitter=0.1)
+    B = 4
+    m = L.model_create(cfg, weights_to(Wc, "cuda"), max_batch=B)
+    kv = L.kv_create(m, B, B * 8)
+    okv = O.KVCache(cfg, B, 128)
+    seq_ids = [2, 0, 3, 1]
+    ctx = [40, 0, 15, 31]
+    _fill_both(L, cfg, kv, okv, seq_ids, ctx, seed=3)
+    Rs = cfg["max_draft"] + 1
+    rng = np.random.default_rng(12)
+    prm = L.make_params(K=cfg["max_draft"], mode=A.TOPK, topk=cfg["vocab"] // 2)     # accepts about half the nodes
+    for step in range(3):
+        tokens = np.zeros((B, Rs), np.int32)
+        parents = np.full((B, Rs), -1, np.int32)
+        n_rows = np.full(B, Rs, np.int32)
+        pars = []
+        for b in range(B):
+            tokens[b] = synth.make_prompt(Rs, cfg["vocab"], 10 * step + b)
+            pars.append(random_tree(rng, Rs - 1))
+            parents[b, 1:] = pars[b]
+        logits = L.verify_step_tree(m, kv, dev_i32(seq_ids), dev_i32(tokens), dev_i32(parents), dev_i32(n_rows))
+        na, ot, no, pr = L.accept_tree(kv, dev_i32(seq_ids), logits, dev_i32(tokens), dev_i32(parents), dev_i32(n_rows), prm)
+        L.check(m)
+        lg = logits.cpu().numpy()
+        O.forward(Wc, cfg, okv, seq_ids, [tokens[b] for b in range(B)], parents=pars)
+        total = 0
+        for b, s in enumerate(seq_ids):
+            # follow the library's decisions (its logits), move the oracle's cache the same way
+            a, em, path = T.accept_tree(lg[b], tokens[b], pars[b], Rs, A.TOPK, cfg["vocab"] // 2, 0.0)
+            assert int(na[b]) == a and pr[b, :a].tolist() == path
+            c = int(okv.ctx[s])
+            for d, row in enumerate(path, 1):
+                okv.k[:, s, c + d] = okv.k[:, s, c + row]
+                okv.v[:, s, c + d] = okv.v[:, s, c + row]
+            okv.ctx[s] += a + 1
+            total += a
+            for l in (0, cfg["n_layers"] - 1):
+                k, v = L.kv_export(kv, s, l, c, a + 1)
+                wk = okv.k[l, s, c:c + a + 1].reshape(a + 1, -1).float()
+                wv = okv.v[l, s, c:c + a + 1].reshape(a + 1, -1).float()
+                assert (k.cpu().float() - wk).abs().max() <= 2.0 ** -7 * max(1.0, float(wk.abs().max()))
+                assert (v.cpu().float() - wv).abs().max() <= 2.0 ** -7 * max(1.0, float(wv.abs().max()))
+        assert (L.kv_get_len(kv, seq_ids) == np.asarray([okv.ctx[s] for s in seq_ids])).all()
+        assert total > 0
+    # a plain chain step on top of the compacted caches still matches the oracle
+    rows = [synth.make_prompt(3, cfg["vocab"], 77 + b) for b in range(B)]
+    tokens = np.full((B, Rs), -1, np.int32)
+    for b in range(B):
+        tokens[b, :3] = rows[b]
+    got = L.verify_step(m, kv, dev_i32(seq_ids), dev_i32(tokens), dev_i32(np.full(B, 3, np.int32))).cpu().double()
+    want = O.forward(Wc, cfg, okv, seq_ids, rows)
+    err = max(float((got[b, :3] - want[b]).abs().max()) for b in range(B))
+    print("after compaction: max-abs logit error", err)
+    assert err <= TOL
