@@ -97,6 +97,8 @@ typedef struct {
   int32_t eos_id;     /* stop after emitting this token; -1 = none                         */
   int32_t temp_branches; /* laser_generate: non-zero = also draft from the sequence's own prompt and
                             generated tokens (temporary branch, Section 3.2; needs max_occ in 1..64) */
+  int32_t tree;          /* laser_generate: non-zero = draft a token tree and verify it with tree
+                            attention (Section 3.3; needs K <= 32 and max_occ in 1..64)            */
 } laser_params;
 
 typedef struct {
@@ -165,6 +167,33 @@ laser_status laser_draft_temp(const laser_pool* pool, const int32_t* tails, cons
                               const int32_t* group_id, const int32_t* hist, const int32_t* hist_len,
                               int64_t hist_stride, int32_t B, const laser_params* p,
                               int32_t* draft, int32_t* draft_len, int32_t* match_n, void* stream);
+
+/* ---- Tree-based drafting: T_t = Retrieve(D, tail, K) as a token tree (Section 3.3) -------------
+ * The sub-tree of the group's trie under the matched tail: a node is a sequence of continuation
+ * tokens, its frequency the number of occurrences of the tail followed by that sequence inside
+ * one document.  When the sub-tree has more than K nodes the K most frequent are kept (ties: the
+ * shallower node, then the smaller token path), which keeps every kept node's parent.  The kept
+ * nodes are listed depth-first, children by (frequency descending, token id ascending): the
+ * pseudo-sequence S_t.  Its first branch is what laser_draft would return, as far as it is kept.
+ * The suffix length n shrinks from n_max as in laser_draft (a tree counts by its nodes).
+ *   hist, hist_len, hist_stride   temporary branch as in laser_draft_temp, or null / null / 0
+ *   draft          dev int32[B, K] out: node tokens in depth-first order, padded with -1
+ *   draft_parents  dev int32[B, K] out: row of each node's parent, where row 0 is the root (the
+ *                  pending token) and node j is row j + 1; padded with -1
+ *   draft_len      dev int32[B] out: nodes;  match_n dev int32[B] out
+ * Occurrences: the first p->max_occ (1..64), the history's first.
+ * Errors: INVALID_ARG (K outside 1..32, max_occ outside 1..64, n range). */
+laser_status laser_draft_tree(const laser_pool* pool, const int32_t* tails, const int32_t* tail_len,
+                              const int32_t* group_id, const int32_t* hist, const int32_t* hist_len,
+                              int64_t hist_stride, int32_t B, const laser_params* p, int32_t* draft,
+                              int32_t* draft_parents, int32_t* draft_len, int32_t* match_n, void* stream);
+
+/* Rows of a tree step: laser_make_rows plus parents[b,0] = -1, parents[b,1+j] = draft_parents[b,j]
+ * for j < draft_len[b], rest -1 (the layout laser_verify_step_tree and laser_accept_tree read). */
+laser_status laser_make_rows_tree(const int32_t* last_token, const int32_t* draft,
+                                  const int32_t* draft_parents, const int32_t* draft_len, int32_t B,
+                                  int32_t K, int32_t* tokens, int32_t* parents, int32_t* n_rows,
+                                  void* stream);
 
 /* Builds the verify rows from the drafts: tokens[b,0] = last_token[b],
  * tokens[b,1..] = draft[b,:draft_len[b]], rest -1; n_rows[b] = 1 + draft_len[b], or 0

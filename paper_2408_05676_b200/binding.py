@@ -45,7 +45,7 @@ class Weights(C.Structure):
 
 class Params(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("K", "n_min", "n_max", "min_draft", "max_occ", "mode", "topk")] + \
-               [("p", C.c_float), ("max_new", C.c_int32), ("eos_id", C.c_int32), ("temp_branches", C.c_int32)]
+               [("p", C.c_float), ("max_new", C.c_int32), ("eos_id", C.c_int32), ("temp_branches", C.c_int32), ("tree", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -57,7 +57,7 @@ class Stats(C.Structure):
 
 
 EXPORTS = ["laser_version", "laser_last_error", "laser_launch_count", "laser_pool_build", "laser_pool_free",
-           "laser_pool_info", "laser_draft", "laser_draft_temp", "laser_make_rows", "laser_model_create", "laser_model_free",
+           "laser_pool_info", "laser_draft", "laser_draft_temp", "laser_draft_tree", "laser_make_rows", "laser_make_rows_tree", "laser_model_create", "laser_model_free",
            "laser_kv_create", "laser_kv_free", "laser_kv_set_page_table", "laser_kv_set_len",
            "laser_kv_get_len", "laser_kv_set_len_dev", "laser_kv_import", "laser_kv_export",
            "laser_verify_step", "laser_verify_step_tree", "laser_check", "laser_profile_enable", "laser_profile_read", "laser_accept_commit", "laser_accept_commit_noalloc", "laser_accept_tree", "laser_kv_compact_path",
@@ -99,8 +99,8 @@ def _stream(stream) -> C.c_void_p:
 
 
 def make_params(K=8, n_min=1, n_max=4, min_draft=1, max_occ=64, mode=MODE_STRICT, topk=2, p=0.1,
-                max_new=0, eos_id=-1, temp_branches=0) -> Params:
-    return Params(K, n_min, n_max, min_draft, max_occ, mode, topk, p, max_new, eos_id, temp_branches)
+                max_new=0, eos_id=-1, temp_branches=0, tree=0) -> Params:
+    return Params(K, n_min, n_max, min_draft, max_occ, mode, topk, p, max_new, eos_id, temp_branches, tree)
 
 
 def version() -> str:
@@ -172,6 +172,37 @@ def draft_temp(pool: Pool, tails, tail_len, group_id, hist, hist_len, params: Pa
                               C.c_int64(hist.shape[1] if hist.dim() == 2 else 0), C.c_int32(B), C.byref(params),
                               _ptr(draft_out), _ptr(draft_len), _ptr(match_n), _stream(stream)))
     return draft_out, draft_len, match_n
+
+
+def draft_tree(pool: Pool, tails, tail_len, group_id, params: Params, hist=None, hist_len=None, stream=None):
+    """laser_draft_tree; returns draft, draft_parents, draft_len, match_n (device tensors)."""
+    B = tail_len.shape[0]
+    dev = tails.device
+    draft_out = torch.empty(B, params.K, dtype=torch.int32, device=dev)
+    par_out = torch.empty(B, params.K, dtype=torch.int32, device=dev)
+    draft_len = torch.empty(B, dtype=torch.int32, device=dev)
+    match_n = torch.empty(B, dtype=torch.int32, device=dev)
+    stride = 0
+    if hist is not None:
+        hist, hist_len = _dev(hist, torch.int32), _dev(hist_len, torch.int32)
+        stride = hist.shape[1]
+    _chk(lib.laser_draft_tree(pool.handle, _ptr(_dev(tails, torch.int32)), _ptr(_dev(tail_len, torch.int32)),
+                              _ptr(_dev(group_id, torch.int32)), _ptr(hist), _ptr(hist_len), C.c_int64(stride),
+                              C.c_int32(B), C.byref(params), _ptr(draft_out), _ptr(par_out), _ptr(draft_len),
+                              _ptr(match_n), _stream(stream)))
+    return draft_out, par_out, draft_len, match_n
+
+
+def make_rows_tree(last_token, draft_t, draft_parents, draft_len, K: int, stream=None):
+    B = last_token.shape[0]
+    dev = last_token.device
+    tokens = torch.empty(B, K + 1, dtype=torch.int32, device=dev)
+    parents = torch.empty(B, K + 1, dtype=torch.int32, device=dev)
+    n_rows = torch.empty(B, dtype=torch.int32, device=dev)
+    _chk(lib.laser_make_rows_tree(_ptr(_dev(last_token, torch.int32)), _ptr(_dev(draft_t, torch.int32)),
+                                  _ptr(_dev(draft_parents, torch.int32)), _ptr(_dev(draft_len, torch.int32)),
+                                  C.c_int32(B), C.c_int32(K), _ptr(tokens), _ptr(parents), _ptr(n_rows), _stream(stream)))
+    return tokens, parents, n_rows
 
 
 def make_rows(last_token, draft_t, draft_len, K: int, tokens=None, n_rows=None, stream=None):
@@ -369,6 +400,14 @@ def accept_tree(kv: Optional[KV], seq_ids, logits, tokens, parents, n_rows, para
                                C.c_int32(V), C.byref(params), _ptr(n_accept), _ptr(out_tokens), _ptr(n_out),
                                _ptr(path_rows), _stream(stream)))
     return n_accept, out_tokens, n_out, path_rows
+
+
+def kv_compact_path(kv: KV, seq_ids, path_rows, n_accept, stream=None) -> None:
+    """laser_kv_compact_path: path_rows int32[B, stride] as laser_accept_tree writes them."""
+    B = n_accept.shape[0]
+    _chk(lib.laser_kv_compact_path(kv.handle, _ptr(_dev(seq_ids, torch.int32)), _ptr(_dev(path_rows, torch.int32)),
+                                   _ptr(_dev(n_accept, torch.int32)), C.c_int32(B), C.c_int32(path_rows.shape[1]),
+                                   _stream(stream)))
 
 
 def generate(model: Model, kv: KV, pool: Optional[Pool], prompts: Sequence[np.ndarray], group_id: Sequence[int],

@@ -119,6 +119,7 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
   LASER_REQUIRE(p->max_new >= 1, "max_new = %d", p->max_new);
   LASER_REQUIRE(pool == nullptr || (p->K >= 1 && p->n_max >= 1 && p->n_max <= 8), "drafting needs K >= 1 and n_max in [1, 8]");
   LASER_REQUIRE(!p->temp_branches || pool != nullptr, "temporary branches are drafted beside a pool");
+  LASER_REQUIRE(!p->tree || pool != nullptr, "tree drafting needs a pool");
   cudaStream_t stream = as_stream(stream_);
   const int K = p->K, Rs = K + 1, n_max = pool ? p->n_max : 1;
   int max_prompt = 0;
@@ -135,7 +136,7 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
   GenState g{};
   g.max_total = max_prompt + p->max_new + Rs;
   int32_t *tokens, *n_rows, *tails, *tail_len, *last, *draft, *draft_len, *match_n, *seq_ids, *gid;
-  int32_t *n_accept, *out_tokens, *n_out, *d_out;
+  int32_t *n_accept, *out_tokens, *n_out, *d_out, *draft_par, *parents, *path_rows;
   float* logits;
   LASER_TRY(buf.get(&g.seq_tok, size_t(B) * g.max_total));
   LASER_TRY(buf.get(&g.seq_len, size_t(B)));
@@ -155,6 +156,9 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
   LASER_TRY(buf.get(&match_n, size_t(B)));
   LASER_TRY(buf.get(&seq_ids, size_t(B)));
   LASER_TRY(buf.get(&gid, size_t(B)));
+  LASER_TRY(buf.get(&draft_par, size_t(B) * std::max(K, 1)));
+  LASER_TRY(buf.get(&parents, size_t(B) * Rs));
+  LASER_TRY(buf.get(&path_rows, size_t(B) * Rs));
   LASER_TRY(buf.get(&n_accept, size_t(B)));
   LASER_TRY(buf.get(&out_tokens, size_t(B) * Rs));
   LASER_TRY(buf.get(&n_out, size_t(B)));
@@ -204,7 +208,11 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
     count_launch();
     if (pool) {
       // temporary branch: the sequence's prompt and generated tokens (seq_tok) are searched as well
-      if (p->temp_branches)
+      if (p->tree)
+        LASER_TRY(laser_draft_tree(pool, tails, tail_len, gid, p->temp_branches ? g.seq_tok : nullptr,
+                                   p->temp_branches ? g.seq_len : nullptr, p->temp_branches ? g.max_total : 0, B, p, draft,
+                                   draft_par, draft_len, match_n, stream));
+      else if (p->temp_branches)
         LASER_TRY(laser_draft_temp(pool, tails, tail_len, gid, g.seq_tok, g.seq_len, g.max_total, B, p, draft, draft_len,
                                    match_n, stream));
       else
@@ -213,13 +221,23 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
       no_draft_kernel<<<ceil_div(B * std::max(K, 1), 128), 128, 0, stream>>>(B, K, draft, draft_len);
       count_launch();
     }
-    LASER_TRY(laser_make_rows(last, draft, draft_len, B, K, tokens, n_rows, stream));
+    const bool tree = pool && p->tree;
+    if (tree) LASER_TRY(laser_make_rows_tree(last, draft, draft_par, draft_len, B, K, tokens, parents, n_rows, stream));
+    else LASER_TRY(laser_make_rows(last, draft, draft_len, B, K, tokens, n_rows, stream));
     LASER_CUDA(cudaEventRecord(ev.e[1], stream));
-    LASER_TRY(laser_verify_step(m, kv, seq_ids, tokens, n_rows, B, logits, stream));
+    if (tree) LASER_TRY(laser_verify_step_tree(m, kv, seq_ids, tokens, parents, n_rows, B, logits, stream));
+    else LASER_TRY(laser_verify_step(m, kv, seq_ids, tokens, n_rows, B, logits, stream));
     ++verify_calls;
     LASER_CUDA(cudaEventRecord(ev.e[2], stream));
-    LASER_TRY(laser_accept_commit(nullptr, nullptr, logits, tokens, n_rows, B, m->cfg.vocab, &acc, n_accept, out_tokens,
-                                  n_out, stream));
+    if (tree) {
+      // verdict, then the accepted path's K/V to consecutive slots (the lengths advance in step_append)
+      LASER_TRY(laser_accept_tree(nullptr, nullptr, logits, tokens, parents, n_rows, B, m->cfg.vocab, &acc, n_accept,
+                                  out_tokens, n_out, path_rows, stream));
+      LASER_TRY(laser_kv_compact_path(kv, seq_ids, path_rows, n_accept, B, Rs, stream));
+    } else {
+      LASER_TRY(laser_accept_commit(nullptr, nullptr, logits, tokens, n_rows, B, m->cfg.vocab, &acc, n_accept, out_tokens,
+                                    n_out, stream));
+    }
     step_append_kernel<<<ceil_div(B, 128), 128, 0, stream>>>(g, B, Rs, p->max_new, p->eos_id, n_rows, n_accept,
                                                             out_tokens, n_out, d_out, kv->seq_len);
     count_launch();

@@ -375,6 +375,201 @@ draft_temp_kernel(PoolView pv, DraftArgs a, TempArgs t) {
   if (lane == 0) { a.draft_len[q] = best_len; a.match_n[q] = best_len ? best_n : 0; }
 }
 
+// Tree-based drafting (Section 3.3): the sub-tree under the matched tail, cut to its K most
+// frequent nodes, listed depth-first.  One warp per query.  The occurrences (history first if
+// given, then the group's, at most max_occ <= 64) each carry a continuation of up to K tokens; a
+// trie node is a pair (occurrence o, depth d) = the first d tokens of o's continuation, owned by
+// the first occurrence that has that prefix.  Pairwise common-prefix lengths give every node's
+// frequency; nodes are taken best first by (frequency descending, depth ascending, token path
+// ascending) -- along one occurrence that is by increasing depth, so each occurrence offers one
+// candidate per round -- and the kept nodes are ranked into depth-first order, children by
+// (frequency descending, token ascending).
+constexpr int kTreeK = 32;   // nodes of a drafted tree (one lane ranks one node)
+
+__global__ void __launch_bounds__(32)
+draft_tree_kernel(PoolView pv, DraftArgs a, TempArgs t, int32_t* __restrict__ draft_parents) {
+  __shared__ uint32_t s_occ[64];
+  __shared__ int32_t s_cont[64][kTreeK];
+  __shared__ uint8_t s_len[64], s_own[64];         // continuation length; first depth the occurrence owns
+  __shared__ uint8_t s_lcp[64][64];
+  __shared__ uint8_t s_freq[64][kTreeK];           // frequency of node (o, d) at [o][d-1]
+  __shared__ int s_sel_o[kTreeK], s_sel_d[kTreeK], s_rank[kTreeK];
+  const int lane = threadIdx.x, q = blockIdx.x;
+  if (q >= a.B) return;
+  int32_t* out = a.draft + size_t(q) * a.K;
+  int32_t* outp = draft_parents + size_t(q) * a.K;
+  const int K = a.K;
+  const int g = a.group_id[q];
+  const bool has_group = g >= 0 && g < pv.G;
+  const int64_t lo = has_group ? pv.goff[g] : 0, hi = has_group ? pv.goff[g + 1] : 0;
+  const int32_t* h = t.hist ? t.hist + size_t(q) * t.hist_stride : nullptr;
+  const int hl = t.hist ? max(t.hist_len[q], 0) : 0;
+  const int cap = a.max_occ;
+  int best_len = 0, best_n = 0;
+  const int tl = min(max(a.tail_len[q], 0), a.n_max);
+  for (int n = tl; n >= a.n_min; --n) {
+    int32_t tn[kMaxN];
+    bool bad = false;
+    uint64_t key = key_begin(g, n);
+    for (int j = 0; j < n; ++j) {
+      tn[j] = a.tails[size_t(q) * a.n_max + a.n_max - n + j];
+      bad |= tn[j] < 0;
+      key = key_push(key, tn[j]);
+    }
+    if (bad) continue;
+    // ---- occurrences ----
+    int n_occ = 0;
+    for (int base = 0; base + 1 < hl && n_occ < cap; base += 32) {
+      const int idx = base + lane;
+      bool ok = idx >= n - 1 && idx + 1 < hl;
+      for (int j = 0; ok && j < n; ++j) ok = h[idx - n + 1 + j] == tn[j];
+      const unsigned ball = __ballot_sync(0xffffffffu, ok);
+      const int slot = n_occ + __popc(ball & ((1u << lane) - 1));
+      if (ok && slot < 64) s_occ[slot] = uint32_t(idx) | 0x80000000u;
+      n_occ += __popc(ball);
+    }
+    n_occ = min(n_occ, cap);
+    uint32_t start = 0, count = 0;
+    if (has_group && n_occ < cap && probe(pv.table[n], pv.mask[n], key_end(key), lane, start, count)) {
+      const uint32_t* plist = pv.positions[n] + start;
+      for (uint32_t base = 0; base < count && n_occ < cap; base += 32) {
+        const uint32_t idx = base + lane;
+        const int64_t p = idx < count ? int64_t(plist[idx]) : -1;
+        const bool ok = idx < count && is_occurrence(pv.tok, lo, hi, p, tn, n);
+        const unsigned ball = __ballot_sync(0xffffffffu, ok);
+        const int slot = n_occ + __popc(ball & ((1u << lane) - 1));
+        if (ok && slot < 64) s_occ[slot] = uint32_t(p);
+        n_occ += __popc(ball);
+      }
+      n_occ = min(n_occ, cap);
+    }
+    if (n_occ == 0) continue;
+    __syncwarp();
+    // ---- continuations ----
+    for (int o = lane; o < n_occ; o += 32) {
+      const uint32_t e = s_occ[o];
+      int len = 0;
+      for (int j = 1; j <= K; ++j) {
+        int32_t tok;
+        if (e & 0x80000000u) { const int idx = int(e & 0x7fffffffu) + j; tok = idx < hl ? h[idx] : -1; }
+        else { const int64_t p = int64_t(e) + j; tok = p < hi ? pv.tok[p] : -1; }
+        if (tok < 0) break;
+        s_cont[o][len++] = tok;
+      }
+      s_len[o] = uint8_t(len);
+    }
+    __syncwarp();
+    // ---- pairwise common-prefix lengths ----
+    for (int pr = lane; pr < n_occ * n_occ; pr += 32) {
+      const int o = pr / n_occ, o2 = pr % n_occ;
+      const int lim = min(int(s_len[o]), int(s_len[o2]));
+      int l = 0;
+      while (l < lim && s_cont[o][l] == s_cont[o2][l]) ++l;
+      s_lcp[o][o2] = uint8_t(l);
+    }
+    __syncwarp();
+    // ---- node frequencies; the depth from which an occurrence owns its nodes ----
+    for (int o = lane; o < n_occ; o += 32) {
+      uint8_t hist_l[kTreeK + 1];
+      for (int d = 0; d <= K; ++d) hist_l[d] = 0;
+      int shared_before = 0;
+      for (int o2 = 0; o2 < n_occ; ++o2) {
+        const int l = s_lcp[o][o2];
+        ++hist_l[l];
+        if (o2 < o) shared_before = max(shared_before, l);
+      }
+      int run = 0;
+      for (int d = int(s_len[o]); d >= 1; --d) { run += hist_l[d]; s_freq[o][d - 1] = uint8_t(run); }
+      s_own[o] = uint8_t(shared_before + 1);
+    }
+    __syncwarp();
+    // ---- best-first selection: each occurrence offers its shallowest untaken own node ----
+    int nd0 = lane < n_occ ? int(s_own[lane]) : 255, nd1 = lane + 32 < n_occ ? int(s_own[lane + 32]) : 255;
+    int m = 0;
+    auto pack = [&](int o, int d) -> unsigned {   // smaller = better; ties are resolved by the token path below
+      const unsigned f = s_freq[o][d - 1];
+      return ((255u - f) << 16) | (unsigned(d) << 8) | unsigned(o);
+    };
+    auto path_less = [&](int o, int o2, int d) -> bool {   // same frequency and depth, different nodes
+      const int l = s_lcp[o][o2];
+      return s_cont[o][l] < s_cont[o2][l];
+    };
+    auto node_better = [&](unsigned x, unsigned y) -> bool {
+      if (y == 0xffffffffu) return x != 0xffffffffu;
+      if (x == 0xffffffffu) return false;
+      if ((x >> 8) != (y >> 8)) return (x >> 8) < (y >> 8);
+      const int o = int(x & 255u), o2 = int(y & 255u), d = int((x >> 8) & 255u);
+      if (o == o2) return false;
+      return path_less(o, o2, d);
+    };
+    while (m < K) {
+      unsigned c0 = (nd0 <= (lane < n_occ ? int(s_len[lane]) : 0)) ? pack(lane, nd0) : 0xffffffffu;
+      const unsigned c1 = (nd1 <= (lane + 32 < n_occ ? int(s_len[lane + 32]) : 0)) ? pack(lane + 32, nd1) : 0xffffffffu;
+      if (node_better(c1, c0)) c0 = c1;
+      for (int off = 16; off; off >>= 1) {
+        const unsigned other = __shfl_xor_sync(0xffffffffu, c0, off);
+        if (node_better(other, c0)) c0 = other;
+      }
+      if (c0 == 0xffffffffu) break;
+      const int o = int(c0 & 255u), d = int((c0 >> 8) & 255u);
+      if (lane == 0) { s_sel_o[m] = o; s_sel_d[m] = d; }
+      if (o == lane) ++nd0;
+      if (o == lane + 32) ++nd1;
+      ++m;
+    }
+    __syncwarp();
+    if (m > best_len) {
+      // ---- depth-first rank of every kept node (lane k ranks node k) ----
+      int rank = 0;
+      const int ok_ = lane < m ? s_sel_o[lane] : 0, dk = lane < m ? s_sel_d[lane] : 0;
+      if (lane < m) {
+        for (int j = 0; j < m; ++j) {
+          if (j == lane) continue;
+          const int oj = s_sel_o[j], dj = s_sel_d[j];
+          const int l = min(int(s_lcp[oj][ok_]), min(dj, dk));
+          bool before;
+          if (l == dj) before = true;                 // j is an ancestor of this node
+          else if (l == dk) before = false;           // this node is an ancestor of j
+          else {                                      // they part at depth l + 1: compare those siblings
+            const int fj = s_freq[oj][l], fk = s_freq[ok_][l];
+            before = fj > fk || (fj == fk && s_cont[oj][l] < s_cont[ok_][l]);
+          }
+          rank += before;
+        }
+        s_rank[lane] = rank;
+      }
+      __syncwarp();
+      if (lane < m) {
+        int parent_row = 0;
+        if (dk > 1)
+          for (int j = 0; j < m; ++j)
+            if (s_sel_d[j] == dk - 1 && int(s_lcp[s_sel_o[j]][ok_]) >= dk - 1) { parent_row = s_rank[j] + 1; break; }
+        out[rank] = s_cont[ok_][dk - 1];
+        outp[rank] = parent_row;
+      }
+      best_len = m; best_n = n;
+    }
+    __syncwarp();
+    if (best_len >= max(a.min_draft, 1)) break;
+  }
+  for (int j = best_len + lane; j < K; j += 32) { out[j] = -1; outp[j] = -1; }
+  if (lane == 0) { a.draft_len[q] = best_len; a.match_n[q] = best_len ? best_n : 0; }
+}
+
+__global__ void make_tree_rows_kernel(const int32_t* __restrict__ last, const int32_t* __restrict__ draft,
+                                      const int32_t* __restrict__ dpar, const int32_t* __restrict__ dlen, int B, int K,
+                                      int32_t* __restrict__ tokens, int32_t* __restrict__ parents,
+                                      int32_t* __restrict__ n_rows) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= B * (K + 1)) return;
+  const int b = i / (K + 1), j = i % (K + 1);
+  const int32_t lt = last[b];
+  const int m = lt < 0 ? 0 : min(max(dlen[b], 0), K);
+  tokens[i] = lt < 0 ? -1 : (j == 0 ? lt : (j <= m ? draft[b * K + j - 1] : -1));
+  parents[i] = (lt >= 0 && j >= 1 && j <= m) ? dpar[b * K + j - 1] : -1;
+  if (j == 0) n_rows[b] = lt < 0 ? 0 : 1 + m;
+}
+
 // Large-run path: one CTA per query, votes through a shared-memory histogram over the
 // vocabulary.  Occurrences are streamed from the run at every depth; one is alive at depth
 // j if its tokens match the tail and its continuation agrees with the draft so far.
@@ -678,6 +873,49 @@ LASER_API laser_status laser_draft_temp(const laser_pool* pool, const int32_t* t
               draft, draft_len, match_n, nullptr};
   TempArgs t{hist, hist_len, hist_stride};
   draft_temp_kernel<<<ceil_div(B, kDraftWarps), kDraftWarps * 32, 0, stream>>>(pv, a, t);
+  count_launch();
+  LASER_CUDA(cudaGetLastError());
+  return LASER_OK;
+}
+
+LASER_API laser_status laser_draft_tree(const laser_pool* pool, const int32_t* tails, const int32_t* tail_len,
+                                        const int32_t* group_id, const int32_t* hist, const int32_t* hist_len,
+                                        int64_t hist_stride, int32_t B, const laser_params* p, int32_t* draft,
+                                        int32_t* draft_parents, int32_t* draft_len, int32_t* match_n, void* stream_) {
+  using namespace laser;
+  LASER_REQUIRE(pool && tails && tail_len && group_id && p && draft && draft_parents && draft_len && match_n, "null argument");
+  LASER_REQUIRE((hist == nullptr) == (hist_len == nullptr), "hist and hist_len come together");
+  LASER_REQUIRE(B >= 0 && hist_stride >= 0, "B = %d, hist_stride = %lld", B, (long long)hist_stride);
+  LASER_REQUIRE(p->K >= 1 && p->K <= kTreeK, "K = %d outside [1, %d]", p->K, kTreeK);
+  LASER_REQUIRE(p->n_min >= pool->n_min && p->n_max <= pool->n_max && p->n_min <= p->n_max,
+                "suffix range [%d, %d] outside the pool's [%d, %d]", p->n_min, p->n_max, pool->n_min, pool->n_max);
+  LASER_REQUIRE(p->max_occ >= 1 && p->max_occ <= 64 && p->min_draft >= 0,
+                "max_occ = %d: tree drafting keeps 1..64 occurrences", p->max_occ);
+  if (B == 0) return LASER_OK;
+  PoolView pv{};
+  pv.tok = pool->tokens; pv.goff = pool->group_offsets; pv.G = pool->n_groups;
+  for (int n = pool->n_min; n <= pool->n_max; ++n) {
+    pv.table[n] = pool->level[n].table; pv.mask[n] = pool->level[n].mask;
+    pv.positions[n] = pool->level[n].positions;
+  }
+  DraftArgs a{tails, tail_len, group_id, B, p->K, p->n_min, p->n_max, p->min_draft, p->max_occ,
+              draft, draft_len, match_n, nullptr};
+  TempArgs t{hist, hist_len, hist_stride};
+  draft_tree_kernel<<<B, 32, 0, as_stream(stream_)>>>(pv, a, t, draft_parents);
+  count_launch();
+  LASER_CUDA(cudaGetLastError());
+  return LASER_OK;
+}
+
+LASER_API laser_status laser_make_rows_tree(const int32_t* last_token, const int32_t* draft, const int32_t* draft_parents,
+                                            const int32_t* draft_len, int32_t B, int32_t K, int32_t* tokens,
+                                            int32_t* parents, int32_t* n_rows, void* stream) {
+  using namespace laser;
+  LASER_REQUIRE(last_token && draft && draft_parents && draft_len && tokens && parents && n_rows, "null argument");
+  LASER_REQUIRE(B >= 0 && K >= 0, "B = %d, K = %d", B, K);
+  if (B == 0) return LASER_OK;
+  make_tree_rows_kernel<<<ceil_div(B * (K + 1), 256), 256, 0, as_stream(stream)>>>(last_token, draft, draft_parents, draft_len,
+                                                                                  B, K, tokens, parents, n_rows);
   count_launch();
   LASER_CUDA(cudaGetLastError());
   return LASER_OK;

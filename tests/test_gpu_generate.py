@@ -10,6 +10,7 @@ from oracle import accept as A
 from oracle import forward as O
 from oracle import generate as G
 from oracle import retrieval as R
+from oracle import tree as T
 from paper_2408_05676_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -52,7 +53,7 @@ def setup(L):
     return cfg, Wc, m, kv, pool, offs, prompts
 
 
-def _teacher_forced(cfg, Wc, pool, offs, prompts, gid, out, prm, mode, k, p, temp=False):
+def _teacher_forced(cfg, Wc, pool, offs, prompts, gid, out, prm, mode, k, p, temp=False, tree=False):
     """Replays the library's committed tokens through the oracle.  Every step the oracle drafts
     and verifies from the library's own history; its emitted tokens must equal the library's
     next tokens unless the deciding logits are within NEAR_TIE."""
@@ -64,11 +65,18 @@ def _teacher_forced(cfg, Wc, pool, offs, prompts, gid, out, prm, mode, k, p, tem
         seq, at = list(map(int, prompts[b])), 0
         while at < len(out[b]):
             lo, hi = int(offs[gid[b]]), int(offs[gid[b] + 1])
-            d, _ = R.draft_one(pool, lo, hi, np.asarray(seq[-prm.n_max:]), prm.K, prm.n_min, prm.n_max,
-                               prm.min_draft, prm.max_occ, np.asarray(seq) if temp else None)
-            rows = np.asarray([seq[-1]] + d, np.int32)
-            lg = O.forward(Wc, cfg, kvo, [0], [rows])[0].float().numpy()
-            a, em = A.accept_one(lg, rows, len(rows), mode, k, p)
+            if tree:
+                d, par, _ = T.draft_tree_one(pool, lo, hi, np.asarray(seq[-prm.n_max:]), prm.K, prm.n_min, prm.n_max,
+                                             prm.min_draft, prm.max_occ, np.asarray(seq) if temp else None)
+                rows = np.asarray([seq[-1]] + d, np.int32)
+                lg = O.forward(Wc, cfg, kvo, [0], [rows], parents=[par])[0].float().numpy()
+                a, em, path = T.accept_tree(lg, rows, par, len(rows), mode, k, p)
+            else:
+                d, _ = R.draft_one(pool, lo, hi, np.asarray(seq[-prm.n_max:]), prm.K, prm.n_min, prm.n_max,
+                                   prm.min_draft, prm.max_occ, np.asarray(seq) if temp else None)
+                rows = np.asarray([seq[-1]] + d, np.int32)
+                lg = O.forward(Wc, cfg, kvo, [0], [rows])[0].float().numpy()
+                a, em = A.accept_one(lg, rows, len(rows), mode, k, p)
             em = em[:len(out[b]) - at]
             got = out[b][at:at + len(em)]
             steps += 1
@@ -87,6 +95,17 @@ def _teacher_forced(cfg, Wc, pool, offs, prompts, gid, out, prm, mode, k, p, tem
                 else:
                     within_tol.append(float(min(gaps)))
                 em = got[:j + 1]       # follow the library's history
+            if tree:
+                # the oracle's cache follows the tokens actually kept: the path (a prefix of it after a
+                # disagreement, found again by its tokens), moved to consecutive slots
+                c, row = int(kvo.ctx[0]), 0
+                for dpt, tok in enumerate(em[:-1], 1):
+                    nxt = [i for i in range(1, len(rows)) if par[i - 1] == row and int(rows[i]) == tok]
+                    if not nxt:
+                        break
+                    row = nxt[0]
+                    kvo.k[:, 0, c + dpt] = kvo.k[:, 0, c + row]
+                    kvo.v[:, 0, c + dpt] = kvo.v[:, 0, c + row]
             kvo.ctx[0] += len(em)
             seq.extend(em)
             at += len(em)
@@ -154,6 +173,37 @@ def test_temporary_branches(L, setup):
     assert near <= max(2, steps // 20)
     with pytest.raises(L.LaserError):      # the temporary-branch draft keeps a capped occurrence list
         L.generate(m, kv, h, tprompts, gid, L.make_params(K=8, n_min=1, n_max=3, max_occ=0, max_new=8, temp_branches=1))
+
+
+def test_tree_drafting(L, setup):
+    """Token trees verified with tree attention: lossless under strict verification, no more steps
+    than chain drafting, every step in agreement with the tree oracle (with and without temporary
+    branches), cache lengths as after plain decoding."""
+    cfg, Wc, m, kv, pool, offs, prompts = setup
+    h = L.pool_build(pool, offs, 1, 3)
+    gid = [0, 1, 2, 3]
+    greedy = L.generate(m, kv, None, prompts, gid, L.make_params(K=8, max_new=64))
+    chain = L.generate(m, kv, h, prompts, gid, L.make_params(K=8, n_min=1, n_max=3, max_occ=64, max_new=64))
+    for temp in (0, 1):
+        prm = L.make_params(K=8, n_min=1, n_max=3, max_occ=64, max_new=64, tree=1, temp_branches=temp)
+        tree = L.generate(m, kv, h, prompts, gid, prm)
+        assert tree["out"] == greedy["out"] and tree["emitted"] == 4 * 64
+        assert (L.kv_get_len(kv, [0, 1, 2, 3]) == 63 + 64).all()
+        exact, near, steps = _teacher_forced(cfg, Wc, pool, offs, prompts, gid, tree["out"], prm, A.STRICT, 1, 0.0,
+                                             temp=bool(temp), tree=True)
+        print("tree (temp", temp, "): steps", steps, "exact", exact, "near-tie", near, "accepted/step",
+              tree["accepted"] / tree["steps"], "chain steps", chain["steps"])
+        assert near <= max(2, steps // 20)
+        if not temp:
+            assert tree["steps"] <= chain["steps"]
+    # relaxed verification of a tree
+    prm = L.make_params(K=8, n_min=1, n_max=3, max_occ=64, mode=L.MODE_RELAXED, topk=2, p=1e-4, max_new=48, tree=1)
+    rel = L.generate(m, kv, h, prompts, gid, prm)
+    assert rel["accepted"] > 0 and rel["emitted"] == 4 * 48
+    exact, near, steps = _teacher_forced(cfg, Wc, pool, offs, prompts, gid, rel["out"], prm, A.RELAXED, 2,
+                                         float(np.float32(1e-4)), tree=True)
+    print("tree relaxed: steps", steps, "exact", exact, "near-tie", near)
+    assert near <= max(2, steps // 10)
 
 
 def test_eos_and_argument_checks(L, setup):

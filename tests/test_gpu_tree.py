@@ -209,3 +209,102 @@ def test_tree_step_commits_the_accepted_path(L):
     err = max(float((got[b, :3] - want[b]).abs().max()) for b in range(B))
     print("after compaction: max-abs logit error", err)
     assert err <= TOL
+
+
+def _tree_oracle_batch(pool_np, offs, tails, tl, gid, K, n_min, n_max, min_draft, max_occ, hists=None):
+    B = len(tl)
+    d = np.full((B, K), -1, np.int32)
+    pr = np.full((B, K), -1, np.int32)
+    ln, mn = np.zeros(B, np.int32), np.zeros(B, np.int32)
+    w = tails.shape[1]
+    for b in range(B):
+        g = int(gid[b])
+        lo, hi = (int(offs[g]), int(offs[g + 1])) if 0 <= g < len(offs) - 1 else (0, 0)
+        tk, pp, n = T.draft_tree_one(pool_np, lo, hi, tails[b, w - int(tl[b]):], K, n_min, n_max, min_draft, max_occ,
+                                     None if hists is None else hists[b])
+        d[b, :len(tk)], pr[b, :len(pp)], ln[b], mn[b] = tk, pp, len(tk), n
+    return d, pr, ln, mn
+
+
+def test_draft_tree_hand_examples(L):
+    gold = os.path.join(os.path.dirname(__file__), "golden", "tree_hand_examples.txt")
+    ints = lambda s: [int(x) for x in s.split(",")] if s else []
+    for line in open(gold):
+        if line.startswith("#") or not line.strip():
+            continue
+        f = [x.strip() for x in line.split("|")]
+        pool_np, tail = np.asarray(ints(f[0]), np.int32), ints(f[1])
+        K, n_min, n_max, min_draft, max_occ = map(int, f[2:7])
+        tails = np.full((1, n_max), -1, np.int32)
+        t = tail[-n_max:]
+        tails[0, n_max - len(t):] = t
+        offs = np.asarray([0, len(pool_np)], np.int64)
+        pool = L.pool_build(pool_np, offs, n_min, n_max)
+        prm = L.make_params(K=K, n_min=n_min, n_max=n_max, min_draft=min_draft, max_occ=max_occ or 64)
+        d, pr, dl, mn = L.draft_tree(pool, dev_i32(tails), dev_i32([len(t)]), dev_i32([0]), prm)
+        n = len(ints(f[7]))
+        assert int(dl[0]) == n and int(mn[0]) == int(f[9])
+        assert d[0, :n].tolist() == ints(f[7]) and pr[0, :n].tolist() == ints(f[8])
+        assert (d[0, n:] == -1).all() and (pr[0, n:] == -1).all()
+        pool.free()
+
+
+@pytest.mark.parametrize("vocab,K,max_occ,temp,seed", [(3, 8, 64, False, 1), (4, 5, 7, False, 2), (6, 32, 64, False, 3),
+                                                       (3, 8, 64, True, 4), (5, 16, 20, True, 5), (40, 8, 64, True, 6)])
+def test_draft_tree_random(L, vocab, K, max_occ, temp, seed):
+    rng = np.random.default_rng(seed)
+    G = 4
+    toks, offs = [], [0]
+    for g in range(G):
+        ln = int(rng.integers(1, 700))
+        t = rng.integers(0, vocab, size=ln)
+        t[rng.random(ln) < 0.05] = -1
+        toks.extend(t.tolist())
+        offs.append(len(toks))
+    pool_np, offs = np.asarray(toks, np.int32), np.asarray(offs, np.int64)
+    n_min, n_max = 1, 4
+    pool = L.pool_build(pool_np, offs, n_min, n_max)
+    B = 120
+    tails, tl = np.full((B, n_max), -1, np.int32), np.zeros(B, np.int32)
+    hists = []
+    for b in range(B):
+        hl = int(rng.choice([0, 1, 5, 33, 64, 200]))
+        h = rng.integers(0, vocab, size=hl).astype(np.int32)
+        hists.append(h)
+        if temp and hl and rng.random() < 0.8:
+            t = h[-n_max:]
+        else:
+            t = rng.integers(0, vocab, size=int(rng.integers(0, n_max + 1))).astype(np.int32)
+        tails[b, n_max - len(t):] = t
+        tl[b] = len(t)
+    gid = rng.integers(0, G, size=B).astype(np.int32)
+    stride = max(1, max(len(h) for h in hists))
+    hist = np.zeros((B, stride), np.int32)
+    hlen = np.zeros(B, np.int32)
+    for b, h in enumerate(hists):
+        hist[b, :len(h)] = h
+        hlen[b] = len(h)
+    for min_draft in (1, K):
+        prm = L.make_params(K=K, n_min=n_min, n_max=n_max, min_draft=min_draft, max_occ=max_occ)
+        d, pr, dl, mn = L.draft_tree(pool, dev_i32(tails), dev_i32(tl), dev_i32(gid), prm,
+                                     dev_i32(hist) if temp else None, dev_i32(hlen) if temp else None)
+        wd, wp, wl, wn = _tree_oracle_batch(pool_np, offs, tails, tl, gid, K, n_min, n_max, min_draft, max_occ,
+                                            hists if temp else None)
+        assert (dl.cpu().numpy() == wl).all() and (mn.cpu().numpy() == wn).all()
+        assert (d.cpu().numpy() == wd).all()
+        assert (pr.cpu().numpy() == wp).all()
+    assert (wl == K).mean() > 0.2 and (wl > 0).mean() > 0.5
+    # rows for the verify step
+    last = rng.integers(0, vocab, size=B).astype(np.int32)
+    last[5] = -1
+    tk, pa, nr = L.make_rows_tree(dev_i32(last), d, pr, dl, K)
+    tk, pa, nr = tk.cpu().numpy(), pa.cpu().numpy(), nr.cpu().numpy()
+    for b in range(B):
+        if last[b] < 0:
+            assert nr[b] == 0 and (tk[b] == -1).all() and (pa[b] == -1).all()
+            continue
+        n = int(wl[b])
+        assert nr[b] == n + 1 and tk[b, 0] == last[b] and pa[b, 0] == -1
+        assert tk[b, 1:n + 1].tolist() == wd[b, :n].tolist() and pa[b, 1:n + 1].tolist() == wp[b, :n].tolist()
+        assert (tk[b, n + 1:] == -1).all() and (pa[b, n + 1:] == -1).all()
+    pool.free()
