@@ -154,7 +154,22 @@ def build_workload(L, dev, cfg):
         new_offs.append(new_offs[-1] + n)
     pool = np.concatenate(parts)
     offs = np.asarray(new_offs, dtype=np.int64)
-    return dict(cfg=cfg, W=W, model=model, kv=kv, seq_ids=seq_ids, lens=lens, last=last_np, tails=tails, gid=gid,
+    # second pool for tree drafting: three differently corrupted copies of each continuation per group,
+    # so that the sub-tree under the tail branches where they disagree
+    parts3, offs3 = [], [0]
+    alt = [drafts, synth.corrupt_drafts(greedy, second, cfg["vocab"], seed=9),
+           synth.corrupt_drafts(greedy, second, cfg["vocab"], seed=10)]
+    base, boffs = synth.make_zipf_pool(POOL_TOKENS, POOL_GROUPS, vocab=cfg["vocab"], seed=42)
+    for g in range(POOL_GROUPS):
+        parts3.append(base[boffs[g]:boffs[g + 1]])
+        n = int(boffs[g + 1] - boffs[g])
+        if g in doc_of:
+            for dr in alt:
+                doc = np.concatenate([[synth.SENTINEL], tails[doc_of[g]], dr[doc_of[g]]]).astype(np.int32)
+                parts3.append(doc)
+                n += len(doc)
+        offs3.append(offs3[-1] + n)
+    return dict(pool3=np.concatenate(parts3), offs3=np.asarray(offs3, dtype=np.int64), cfg=cfg, W=W, model=model, kv=kv, seq_ids=seq_ids, lens=lens, last=last_np, tails=tails, gid=gid,
                 drafts=drafts, greedy=greedy, pool=pool, offs=offs)
 
 
@@ -231,6 +246,47 @@ def run_ours(args):
 
     res = {name: timed(prm, args.steps, args.warmup, sample_clocks=(name == "strict")) for name, prm in modes.items()}
     main = res["strict"]
+
+    # tree-based drafting (Section 3.3) against chain drafting, both on the pool with three variants per
+    # continuation: same verify forward (tree attention), tree verification, cache compaction
+    pool3 = L.pool_build(wl["pool3"], wl["offs3"], 1, N_MAX)
+    tree_out = {}
+
+    def tree_step(prm):
+        L.kv_set_len_dev(kv, lens)
+        d, pr, dl, _ = L.draft_tree(pool3, d_tails, d_tl, d_gid, prm)
+        tk, pa, nr = L.make_rows_tree(d_last, d, pr, dl, K)
+        L.verify_step_tree(model, kv, seq_ids, tk, pa, nr, logits)
+        tree_out["r"] = L.accept_tree(kv, seq_ids, logits, tk, pa, nr, prm)
+
+    def chain3_step(prm):
+        L.kv_set_len_dev(kv, lens)
+        L.draft(pool3, d_tails, d_tl, d_gid, prm, draft, dlen, mn)
+        L.make_rows(d_last, draft, dlen, K, tokens, n_rows)
+        L.verify_step(model, kv, seq_ids, tokens, n_rows, logits)
+        L.accept_commit(kv, seq_ids, logits, tokens, n_rows, prm, out=outs)
+
+    def timed_fn(fn, result):
+        for _ in range(max(3, args.warmup)):
+            fn(strict)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            fn(strict)
+        e1.record()
+        barrier()
+        ms, _ = replicas.reduce_step(dist, e0.elapsed_time(e1) / args.steps, 0, torch.device(dev))
+        na, no = result()
+        return dict(ms_per_step=ms, tokens_per_s=world * no / (ms * 1e-3), accepted_drafts_per_step=na / B,
+                    emitted_per_step=no / B)
+
+    tree_res = dict(
+        note="pool with three corrupted variants of each continuation; strict verification",
+        tree=timed_fn(tree_step, lambda: (int(tree_out["r"][0].sum()), int(tree_out["r"][2].sum()))),
+        chain=timed_fn(chain3_step, lambda: (int(outs[0].sum()), int(outs[2].sum()))))
+    L.check(model)
+    step(strict)        # leave the buffers as the headline step does
     value = world * main["tokens"] / (main["ms"] * 1e-3)
 
     def verify_pass(profile):
@@ -308,6 +364,7 @@ def run_ours(args):
                      "frac": gemm_gbs / peaks["hbm_gbs"], "traffic": GEMM_DRAM_TRAFFIC_PER_STEP if args.layers == 32 else None,
                      "traffic_note": "ncu dram read+write summed over the 129 launches of a step (per-launch figures in profiles/gemm_tc_kernel_7b_rows144.md, scaled from a 2-layer capture); includes up to 48 MB of next-kernel L2 prefetch per launch, counted twice under ncu's serialised replay",
                      "algorithmic_bytes_per_step": ab["weights"], "ms_per_step": gemm_ms, "launches_per_step": gemm_n // args.steps},
+        "tree_drafting": tree_res,
         "verify_step": {"ms": verify_ms, "algorithmic_bytes": ab["total"],
                         "achieved_gbs": ab["total"] / (verify_ms * 1e-3) / 1e9,
                         "frac_of_measured_hbm": ab["total"] / (verify_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
