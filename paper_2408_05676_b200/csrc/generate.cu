@@ -194,6 +194,7 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
     LASER_TRY(laser_verify_step(m, kv, seq_ids, tokens, n_rows, B, logits, stream));
     prefill_advance_kernel<<<ceil_div(B, 128), 128, 0, stream>>>(g, B, n_rows, kv->seq_len);
     count_launch(2);
+    if ((it & 15) == 15) LASER_TRY(laser_check(m, stream));   // do not keep launching after a device-side error
   }
   LASER_CUDA(cudaEventRecord(ev.e[1], stream));
   LASER_CUDA(cudaStreamSynchronize(stream));
@@ -201,6 +202,7 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
 
   laser_params acc = *p;
   int64_t verify_calls = 0;
+  int32_t h_status = 0;
   const int max_steps = p->max_new + 1;
   for (int step = 0; step < max_steps && h_active > 0; ++step) {
     LASER_CUDA(cudaEventRecord(ev.e[0], stream));
@@ -243,7 +245,9 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
     count_launch();
     LASER_CUDA(cudaEventRecord(ev.e[3], stream));
     LASER_CUDA(cudaMemcpyAsync(&h_active, g.n_active, 4, cudaMemcpyDeviceToHost, stream));
+    LASER_CUDA(cudaMemcpyAsync(&h_status, m->status, 4, cudaMemcpyDeviceToHost, stream));
     LASER_CUDA(cudaStreamSynchronize(stream));
+    if (h_status != 0) break;   // a device-side error (capacity, a wait that ran out): stop at once, laser_check reports it
     LASER_CUDA(cudaEventElapsedTime(&ms, ev.e[0], ev.e[1])); ms_draft += ms;
     LASER_CUDA(cudaEventElapsedTime(&ms, ev.e[1], ev.e[2])); ms_verify += ms;
     LASER_CUDA(cudaEventElapsedTime(&ms, ev.e[2], ev.e[3])); ms_accept += ms;
