@@ -25,6 +25,7 @@
 // copies, still joins the cluster barriers, frees its tensor memory and exits.
 #include <map>
 #include <tuple>
+#include <type_traits>
 
 #include "model.cuh"
 #include "tma.cuh"
@@ -39,7 +40,6 @@ constexpr int kBK = 64;           // K elements per stage = one 128-byte swizzle
 constexpr int kMaxStages = 6;
 constexpr int kMaxNT = 192;       // token rows per tile: accumulator staging must fit shared memory
 constexpr int kSmemBudget = 110 * 1024;  // shared memory of one CTA: two CTAs per SM
-constexpr int kBatch = 3, kPre = 3;      // epilogue: columns per group, groups whose operands are prefetched
 
 // Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows 128 B apart, groups
 // of 8 rows 1024 B apart.
@@ -302,11 +302,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = tmem_slot;
 
-  // epilogue operands live in registers of warps 2-5 from kernel start to the epilogue
-  const int ew = warp - 2, nfeat = n0 + 4 * lane;
+  const int nfeat = n0 + 4 * lane;
   const LaneCtx lc = make_lane_ctx<EPI>(e, n0, lane, N);
-  uint2 gain4 = make_uint2(0u, 0u);
-  float4 pg0[kPre][kBatch], pg1[kPre][kBatch];
+  uint2 gain4 = make_uint2(0u, 0u);   // gains of the next norm: a weight, not a result of the kernel before
+  if (EPI == EPI_RESID && nfeat < N) gain4 = *reinterpret_cast<const uint2*>(e.gain_next + nfeat);
   auto fetch_operands = [&](int jj, float4& g0, float4& g1) {
     g0 = make_float4(0.f, 0.f, 0.f, 0.f); g1 = g0;
     const int r = r0 + krank * slice + jj;
@@ -401,11 +400,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       }
       s_rstd[j] = rstd; s_pos[j] = pos; s_page[j] = page;
     }
-    if (EPI == EPI_RESID && nfeat < N) gain4 = *reinterpret_cast<const uint2*>(e.gain_next + nfeat);
-#pragma unroll
-    for (int k = 0; k < kPre; ++k)
-#pragma unroll
-      for (int b = 0; b < kBatch; ++b) fetch_operands((ew + 4 * k) * kBatch + b, pg0[k][b], pg1[k][b]);
     // part 2: accumulator from tensor memory to shared memory, token-major [NT][128]
     const int quarter = warp & 3;  // a warp may only touch its own 32 TMEM lanes
     const bool ok = mbar_wait(smem_u32(&acc_bar), 0, &abort_flag);
@@ -464,56 +458,54 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         else epi_swiglu(e, r, live, wtile * 64, lane, acc[b], rstd);
       }
     }
-  } else if (warp >= 2) {
-    // part 3: sum the partial columns this CTA owns (ranks in order 0..splits-1) and finish them.
-    // One group = kBatch columns: all partial columns of a group are requested first
-    // (independent loads), then summed and finished.  Warp w takes groups w, w+4, w+8, ...
-    uint32_t rank_base[8];
+  } else {
+    // part 3: sum the partial columns this CTA owns (ranks in order 0..splits-1) and finish them, all
+    // six warps, group g by warp g % 6.  A group is as many columns as give about twelve loads in
+    // flight per lane: every partial column of the group and its epilogue operands are requested
+    // first (independent loads, one round trip through distributed shared memory), then summed in
+    // rank order and finished.
+    auto reduce_rows = [&](auto s_tag, auto rb_tag) {
+      constexpr int S = decltype(s_tag)::value, RB = decltype(rb_tag)::value;
+      uint32_t rank_base[S];
 #pragma unroll
-    for (int rk = 0; rk < 8; ++rk)
-      rank_base[rk] = splits > 1 ? map_to_rank(tiles, uint32_t(PAIR ? 2 * min(rk, splits - 1) + half : min(rk, splits - 1))) : tiles;
-    auto finish_group = [&](int jb, const float4 (&g0)[kBatch], const float4 (&g1)[kBatch]) {
-      float4 acc[kBatch];
+      for (int q = 0; q < S; ++q) rank_base[q] = S > 1 ? map_to_rank(tiles, uint32_t(PAIR ? 2 * q + half : q)) : tiles;
+      for (int jb = warp * RB; jb < own; jb += (kTcThreads / 32) * RB) {
+        float4 part[RB][S], g0[RB], g1[RB];
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {   // ranks 0-3, then 4-7: at most 12 loads in flight
-        float4 part[kBatch][4];
+        for (int b = 0; b < RB; ++b) {
+          const int jj = min(jb + b, own - 1);
 #pragma unroll
-        for (int b = 0; b < kBatch; ++b)
+          for (int q = 0; q < S; ++q)
+            part[b][q] = ld_cluster_f4(rank_base[q] + uint32_t(((krank * slice + jj) * kBM + 4 * lane) * 4));
+        }
 #pragma unroll
-          for (int q = 0; q < 4; ++q)
-            if (half * 4 + q < splits && jb + b < own)
-              part[b][q] = ld_cluster_f4(rank_base[half * 4 + q] + uint32_t(((krank * slice + jb + b) * kBM + 4 * lane) * 4));
+        for (int b = 0; b < RB; ++b) fetch_operands(jb + b, g0[b], g1[b]);
 #pragma unroll
-        for (int b = 0; b < kBatch; ++b)
+        for (int b = 0; b < RB; ++b) {
+          float4 acc = part[b][0];
 #pragma unroll
-          for (int q = 0; q < 4; ++q)
-            if (half * 4 + q < splits && jb + b < own) {
-              if (half == 0 && q == 0) acc[b] = part[b][0];
-              else { acc[b].x += part[b][q].x; acc[b].y += part[b][q].y; acc[b].z += part[b][q].z; acc[b].w += part[b][q].w; }
-            }
-        if (splits <= 4) break;
-      }
-#pragma unroll
-      for (int b = 0; b < kBatch; ++b) {
-        const int jj = jb + b;
-        const int j = jj < own ? krank * slice + jj : 0, r = r0 + j;
-        const bool live = jj < own && r < e.R_rows;   // the last token tile may overhang the buffers
-        if (jj >= own) acc[b] = make_float4(0.f, 0.f, 0.f, 0.f);
-        const float rstd = s_rstd[j];
-        if (EPI == EPI_PLAIN) epi_plain(e, lc, r, live, acc[b], rstd, N);
-        else if (EPI == EPI_RESID) epi_resid(e, lc, r, live, lane, acc[b], N, wtile, g0[b], gain4);
-        else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, live, wtile * 64, lane, acc[b], rstd);
-        else epi_qkv(e, lc, r, live, acc[b], rstd, s_pos[j], s_page[j], g0[b], g1[b]);
+          for (int q = 1; q < S; ++q) { acc.x += part[b][q].x; acc.y += part[b][q].y; acc.z += part[b][q].z; acc.w += part[b][q].w; }
+          const int jj = jb + b;
+          const int j = jj < own ? krank * slice + jj : 0, r = r0 + j;
+          const bool live = jj < own && r < e.R_rows && !abort_flag;   // the last token tile may overhang the buffers
+          const float rstd = s_rstd[j];
+          if (EPI == EPI_PLAIN) epi_plain(e, lc, r, live, acc, rstd, N);
+          else if (EPI == EPI_RESID) epi_resid(e, lc, r, live, lane, acc, N, wtile, g0[b], gain4);
+          else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, live, wtile * 64, lane, acc, rstd);
+          else epi_qkv(e, lc, r, live, acc, rstd, s_pos[j], s_page[j], g0[b], g1[b]);
+        }
       }
     };
-#pragma unroll
-    for (int k = 0; k < kPre; ++k)
-      if ((ew + 4 * k) * kBatch < own) finish_group((ew + 4 * k) * kBatch, pg0[k], pg1[k]);
-    for (int jb = (ew + 4 * kPre) * kBatch; jb < own; jb += 4 * kBatch) {
-      float4 g0[kBatch], g1[kBatch];
-#pragma unroll
-      for (int b = 0; b < kBatch; ++b) fetch_operands(jb + b, g0[b], g1[b]);
-      finish_group(jb, g0, g1);
+    using std::integral_constant;
+    switch (splits) {
+      case 1: reduce_rows(integral_constant<int, 1>{}, integral_constant<int, 6>{}); break;
+      case 2: reduce_rows(integral_constant<int, 2>{}, integral_constant<int, 6>{}); break;
+      case 3: reduce_rows(integral_constant<int, 3>{}, integral_constant<int, 4>{}); break;
+      case 4: reduce_rows(integral_constant<int, 4>{}, integral_constant<int, 3>{}); break;
+      case 5: reduce_rows(integral_constant<int, 5>{}, integral_constant<int, 2>{}); break;
+      case 6: reduce_rows(integral_constant<int, 6>{}, integral_constant<int, 2>{}); break;
+      case 7: reduce_rows(integral_constant<int, 7>{}, integral_constant<int, 2>{}); break;
+      default: reduce_rows(integral_constant<int, 8>{}, integral_constant<int, 1>{}); break;
     }
   }
   __syncwarp();
