@@ -635,7 +635,10 @@ laser_status gemm_fused(laser_model* m, const __nv_bfloat16* A, const __nv_bfloa
   const int n_wtiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
   // Two weight tiles share one 256-row MMA of a CTA pair (each CTA then stages only half of the
   // token rows) when the tiles come in pairs.
-  const bool pair = g_force_pair != 0 && n_wtiles % 2 == 0;
+  // All GEMMs of a model run the same MMA form (m->pair_mma): kernels of consecutive launches share
+  // SMs under programmatic dependent launch, and a step that alternated between one-CTA and two-CTA
+  // tensor-memory allocation stopped making progress when it was tried.
+  const bool pair = g_force_pair != 0 && m->pair_mma && n_wtiles % 2 == 0;
   const int splits = pick_splits(R_pad, N, K, epi, pair);
   const TcShape sh = tc_shape(R_pad, pair);
   const CUtensorMap *tw = nullptr, *ta = nullptr;
