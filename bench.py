@@ -31,7 +31,7 @@ WORKLOAD = "verify-step-7b: batch 16, ctx 512 (16-token pages), 1+8 rows/seq, dr
 B, K, CTX, N_MAX = 16, 8, 512, 4
 POOL_TOKENS, POOL_GROUPS = 5_000_000, 1000
 # read + write MB of the QKV, O, gate/up and down launches of a layer x 32 + the LM head, from the ncu capture
-GEMM_DRAM_TRAFFIC_PER_STEP = int((105.7 + 76.6 + 219.9 + 132.2) * 32e6 + 267.8e6)
+GEMM_DRAM_TRAFFIC_PER_STEP = int((105.5 + 76.8 + 217.4 + 138.3) * 32e6 + 267.6e6)
 SAMPLE_LAYERS = 4          # layers the CPU baseline really runs (time is extrapolated to all)
 
 

@@ -16,11 +16,12 @@
 //              shared-memory stages; weight tiles are requested before the dependency wait,
 //              since they do not depend on the previous kernel;
 //   warp 1     MMA issuer: tcgen05.mma into a TMEM accumulator, tcgen05.commit frees stages;
-//   warps 2-5  epilogue: move the finished accumulator to shared memory (the free stages),
-//              then, after a cluster barrier, sum the partial tiles of the cluster through
+//   warps 2-5  move the finished accumulator to shared memory (the free stages); then, after a
+//              cluster barrier, all six warps sum the partial tiles of the cluster through
 //              distributed shared memory in rank order (run-to-run identical, no partial sums
-//              in global memory) for the token columns this CTA owns and apply the fused
-//              epilogue, whose global operands were requested at kernel start.
+//              in global memory) for the token columns this CTA owns and apply the fused epilogue.
+// Option PAIR: the CTAs of cluster ranks 2i, 2i+1 run one 256-row MMA together (cta_group::2),
+// each staging its own 128 weight rows and half of the token rows.
 // Every mbarrier wait is bounded: on expiry the CTA records LASER_ERR_TIMEOUT, drains its
 // copies, still joins the cluster barriers, frees its tensor memory and exits.
 #include <map>
@@ -545,10 +546,12 @@ laser_status tensor_map(GemmState* st, const void* ptr, int rows, int cols, int 
 struct TcShape { int n_ttiles, NT, stages, tmem_cols; size_t smem; };
 }  // namespace
 // Tuning aids: non-zero values override the modelled split count / the stage count;
-// g_force_pair: 0 = single-CTA MMA only, 1 = two-CTA MMA wherever the shape allows it.
+// g_force_pair: 0 (default) = single-CTA MMA; 1 = two-CTA MMA (cta_group::2) for models whose matrices all
+// have an even number of weight tiles.  Both forms measure the same step time; the single-CTA form is the
+// default because it keeps tensor-memory allocation local to an SM.
 int g_force_splits = 0;
 int g_force_stages = 0;
-int g_force_pair = 1;
+int g_force_pair = 0;
 namespace {
 
 TcShape tc_shape(int R_pad, bool pair) {
