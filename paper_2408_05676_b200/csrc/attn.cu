@@ -53,13 +53,14 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
   constexpr int QLD = DH + 8;                     // padded row of the Q tile (elements)
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint64_t full_bar[kStages], empty_bar[kStages];
-  __shared__ float s_m[kConsumers][16], s_l[kConsumers][16];
+  __shared__ float s_m[kConsumers][16], s_l[kConsumers][16], s_wgt[kConsumers][16];
   __shared__ int abort_flag;
 
-  // programmatic dependent launch: let the next kernel start its prologue, then wait for the
-  // kernel that produced Q and the new K/V rows
+  // Programmatic dependent launch: let the next kernel start its prologue.  The kernel before this
+  // one produces Q and the K/V of the step's own rows; pages that lie wholly below the committed
+  // length were written by earlier steps, so the producer requests those before it waits for that
+  // kernel, and the wait and the Q tile overlap their flight.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int b = blockIdx.x, h = blockIdx.y, mt = blockIdx.z;
   const int hk = h / (H / Hkv);
   const int nr = row_n[b], ctx = row_ctx[b];
@@ -67,6 +68,7 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
   const int row0 = mt * 16;
   bf16* obase = out + (size_t(b) * Rs + row0) * H * DH + size_t(h) * DH;
   if (row0 >= nr) {  // nothing active in this tile: zero its rows
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int idx = tid; idx < 16 * DH; idx += kAttnThreads) {
       const int r = idx / DH, d = idx % DH;
       if (row0 + r < Rs) obase[size_t(r) * H * DH + d] = __float2bfloat16(0.f);
@@ -87,22 +89,17 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
     mbar_fence_init();
     tma_prefetch_map(&kvmap);
   }
-  // Q tile: rows of this sequence, zero beyond the active ones
-  for (int idx = tid; idx < 16 * (DH / 8); idx += kAttnThreads) {
-    const int r = idx / (DH / 8), c = idx % (DH / 8);
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (row0 + r < nr) v = *reinterpret_cast<const uint4*>(q + (size_t(b) * Rs + row0 + r) * H * DH + size_t(h) * DH + c * 8);
-    *reinterpret_cast<uint4*>(q_ptr + r * QLD + c * 8) = v;
-  }
-  __syncthreads();
+  __syncthreads();   // barriers initialised
 
   if (warp == kConsumers) {  // producer
     if (lane == 0) {
       const int32_t* pt = page_table + size_t(seq_ids[b]) * pages_per_seq;
+      const int n_early = min(min(ctx >> 4, n_pg), kStages);   // whole pages of older tokens that fit the ring
       bool ok = true;
       int issued = 0;
       for (int p = 0; p < n_pg && ok; ++p) {
         const int s = p % kStages;
+        if (p == n_early) asm volatile("griddepcontrol.wait;" ::: "memory");   // from here on: pages the kernel before may write
         if (p >= kStages) ok = mbar_wait(smem_u32(&empty_bar[s]), ((p / kStages) - 1) & 1, &abort_flag);
         if (!ok) break;
         const uint32_t bar = smem_u32(&full_bar[s]);
@@ -128,6 +125,15 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
   }
 
   // ---- consumers ----
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Q tile: rows of this sequence, zero beyond the active ones
+  for (int idx = tid; idx < 16 * (DH / 8); idx += kConsumers * 32) {
+    const int r = idx / (DH / 8), c = idx % (DH / 8);
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (row0 + r < nr) v = *reinterpret_cast<const uint4*>(q + (size_t(b) * Rs + row0 + r) * H * DH + size_t(h) * DH + c * 8);
+    *reinterpret_cast<uint4*>(q_ptr + r * QLD + c * 8) = v;
+  }
+  asm volatile("bar.sync 1, 128;" ::: "memory");
   const int g = lane >> 2, qd = lane & 3;
   const float sl2 = rsqrtf(float(DH)) * 1.4426950408889634f;
   // Q fragments are re-read from shared memory for every page: keeping them in registers
@@ -232,21 +238,36 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
     *reinterpret_cast<float2*>(s_o + (warp * 16 + g + 8) * DH + t * 8 + 2 * qd) = make_float2(o[t][2], o[t][3]);
   }
   asm volatile("bar.sync 1, 128;" ::: "memory");
-  for (int idx = tid; idx < 16 * DH; idx += kConsumers * 32) {
-    const int r = idx / DH, d = idx % DH;
-    if (row0 + r >= Rs) continue;
+  // weight of each warp's partial result per row, normalisation included: e_w / sum_w e_w l_w
+  if (tid < 16 * kConsumers) {
+    const int r = tid % 16, wsel = tid / 16;
     float mt_ = -INFINITY;
 #pragma unroll
     for (int w = 0; w < kConsumers; ++w) mt_ = fmaxf(mt_, s_m[w][r]);
-    float num = 0.f, den = 0.f;
+    float den = 0.f, mine = 0.f;
 #pragma unroll
     for (int w = 0; w < kConsumers; ++w) {
       const float e = s_m[w][r] == -INFINITY ? 0.f : exp2f((s_m[w][r] - mt_) * sl2);
-      num += e * s_o[(w * 16 + r) * DH + d];
       den += e * s_l[w][r];
+      if (w == wsel) mine = e;
     }
     const bool live = row0 + r < nr && den > 0.f && !abort_flag;
-    obase[size_t(r) * H * DH + d] = __float2bfloat16(live ? num / den : 0.f);
+    s_wgt[wsel][r] = live ? mine / den : 0.f;
+  }
+  asm volatile("bar.sync 1, 128;" ::: "memory");
+  for (int idx = tid; idx < 16 * (DH / 4); idx += kConsumers * 32) {   // four features per thread
+    const int r = idx / (DH / 4), d = (idx % (DH / 4)) * 4;
+    if (row0 + r >= Rs) continue;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int w = 0; w < kConsumers; ++w) {
+      const float e = s_wgt[w][r];
+      const float4 x = *reinterpret_cast<const float4*>(s_o + (w * 16 + r) * DH + d);
+      acc.x += e * x.x; acc.y += e * x.y; acc.z += e * x.z; acc.w += e * x.w;
+    }
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+    *reinterpret_cast<uint2*>(obase + size_t(r) * H * DH + d) =
+        make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
   }
   if (tid == 0 && abort_flag) atomicCAS(status, 0, LASER_ERR_TIMEOUT);
 }
