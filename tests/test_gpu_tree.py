@@ -308,3 +308,45 @@ def test_draft_tree_random(L, vocab, K, max_occ, temp, seed):
         assert tk[b, 1:n + 1].tolist() == wd[b, :n].tolist() and pa[b, 1:n + 1].tolist() == wp[b, :n].tolist()
         assert (tk[b, n + 1:] == -1).all() and (pa[b, n + 1:] == -1).all()
     pool.free()
+
+
+def test_13b_shape_17_rows_chain_and_tree(L):
+    """The 13B layer shape (d 5120, 40 heads of 128, f 13824) with K = 16: 17 rows per sequence, i.e. two
+    16-row tiles in the attention kernel (the second holding one row), 9 sequences = 153 rows in the GEMMs.
+    Two layers, so that the fp64 oracle stays cheap; chain rows and a token tree, both against the oracle."""
+    cfg = synth.model_cfg("13b", n_layers=2, max_draft=16, vocab=8192)
+    Wc = synth.make_weights(cfg, seed=1)
+    B, Rs = 9, 17
+    m = L.model_create(cfg, weights_to(Wc, "cuda"), max_batch=B)
+    kv = L.kv_create(m, B, B * 16)
+    okv = O.KVCache(cfg, B, 256)
+    rng = np.random.default_rng(6)
+    seq_ids = list(range(B))
+    ctx = [int(x) for x in rng.integers(0, 200, size=B)]
+    _fill_both(L, cfg, kv, okv, seq_ids, ctx, seed=21)
+    for tree in (False, True):
+        tokens = np.full((B, Rs), -1, np.int32)
+        parents = np.full((B, Rs), -1, np.int32)
+        n_rows = np.zeros(B, np.int32)
+        rows, pars = [], []
+        for b in range(B):
+            nr = Rs if b < 3 else int(rng.integers(1, Rs + 1))
+            r = synth.make_prompt(nr, cfg["vocab"], 300 + b + 50 * tree)
+            par = random_tree(rng, nr - 1) if tree else list(range(nr - 1))
+            tokens[b, :nr], parents[b, 1:nr], n_rows[b] = r, par, nr
+            rows.append(r)
+            pars.append(par)
+        if tree:
+            logits = L.verify_step_tree(m, kv, dev_i32(seq_ids), dev_i32(tokens), dev_i32(parents), dev_i32(n_rows))
+        else:
+            logits = L.verify_step(m, kv, dev_i32(seq_ids), dev_i32(tokens), dev_i32(n_rows))
+        L.check(m)
+        want = O.forward(Wc, cfg, okv.clone(), seq_ids, rows, parents=pars if tree else None)
+        # at this width rounding the GEMM operands to bf16 alone moves the logits by more than 2e-2: the
+        # yardstick is the fp64 oracle whose only change is that rounding (25 % slack for other rounding points)
+        yard = O.forward(Wc, cfg, okv, seq_ids, rows, parents=pars if tree else None, mirror_bf16=True)
+        got = logits.cpu().double()
+        err = max(float((got[b, :n_rows[b]] - want[b]).abs().max()) for b in range(B))
+        yerr = max(float((yard[b] - want[b]).abs().max()) for b in range(B))
+        print("13B shape, tree" if tree else "13B shape, chain", "max-abs logit error", err, "bf16-operand oracle", yerr)
+        assert err <= 1.25 * yerr and err < 0.15
