@@ -4,10 +4,9 @@ A synthetic analogue of the paper's pool-size study (Section 3.1, Figure 2) and 
 column of its ablation (Table 3): the same token stream is indexed once as a single group (global pool)
 and once as groups of about 5 k tokens (customised pools), at several total sizes.  Reported per
 configuration: index build time and bytes, device time of laser_draft for 4096 queries (chain and tree
-form), hit rate and mean draft length.  With --scan the linear scan of one group per query (what a
-pool without an index costs; the test oracle's definition, run on the host) is timed on a sample.
+form), hit rate and mean draft length.
 
-    python -m paper_2408_05676_b200.pool_sweep [--sizes 1,5,20,50] [--scan]
+    python -m paper_2408_05676_b200.pool_sweep [--sizes 1,5,20,50]
 
 Prints one JSON line per configuration.  The streams are the Zipf/template recipe of synth.py; real
 datasets and embeddings are not available here, so acceptance quality is not part of this sweep.
@@ -38,7 +37,7 @@ def _time_ms(fn, reps: int = 10) -> float:
     return e0.elapsed_time(e1) / reps
 
 
-def run(sizes_m, scan: bool, n_queries: int = 4096, K: int = 16) -> None:
+def run(sizes_m, n_queries: int = 4096, K: int = 16) -> None:
     dev = "cuda"
     for size_m in sizes_m:
         n = int(size_m * 1e6)
@@ -71,14 +70,6 @@ def run(sizes_m, scan: bool, n_queries: int = 4096, K: int = 16) -> None:
                        tree_draft_us_per_4096_queries=round(ms_tree * 1e3, 1),
                        hit_rate=round(float((dl > 0).mean()), 3), mean_draft=round(float(dl.mean()), 2),
                        mean_tree_nodes=round(float(out["t"][2].float().mean()), 2))
-            if scan:
-                from oracle import retrieval as R      # the definition, run on the host: a scan of the group
-                sample = range(0, n_queries, max(1, n_queries // 16))
-                t0 = time.time()
-                for q in sample:
-                    lo, hi = int(offs[gid[q]]), int(offs[gid[q] + 1])
-                    R.draft_one(pool, lo, hi, tails[q], K, 1, 4, 1, 64)
-                rec["host_scan_ms_per_query"] = round((time.time() - t0) * 1e3 / len(sample), 3)
             print(json.dumps(rec), flush=True)
             h.free()
 
@@ -86,6 +77,5 @@ def run(sizes_m, scan: bool, n_queries: int = 4096, K: int = 16) -> None:
 if __name__ == "__main__":
     ap = argparse.ArgumentParser()
     ap.add_argument("--sizes", default="1,5,20,50", help="total pool sizes in millions of tokens")
-    ap.add_argument("--scan", action="store_true", help="also time the host-side linear scan (imports the test oracle)")
     a = ap.parse_args()
-    run([float(x) for x in a.sizes.split(",")], a.scan)
+    run([float(x) for x in a.sizes.split(",")])

@@ -206,3 +206,39 @@ def test_generation_7b_batch64_chain_and_tree(L):
         assert gap < 0.3
     print("greedy    %6.2f s  decode %7.1f tokens/s" % (t_greedy, B * NEW / ((greedy["ms_total"] - greedy["ms_prefill"]) * 1e-3)))
     assert results["chain"]["steps"] < greedy["steps"] // 2
+
+
+def test_scan_time_grows_with_the_group_the_index_does_not(L):
+    """The paper's motivation for customised pools (Section 3.1): retrieval that walks the pool gets slower
+    as the pool grows.  The oracle's linear scan shows it on the host (time per query, 5 k-token groups
+    against one 20 M-token pool); the hashed index answers 4096 queries in the same time for both."""
+    n = 20_000_000
+    pool, offs = synth.make_zipf_pool(n, n // 5000, vocab=32000, seed=42)
+    tails, tail_len, gid = synth.make_queries(pool, offs, 4096, n_tail=4, seed=44)
+    prm = L.make_params(K=16, n_min=1, n_max=4, max_occ=64)
+    res = {}
+    for name, o, g in (("customised", offs, gid), ("global", np.asarray([0, n], np.int64), np.zeros(4096, np.int32))):
+        h = L.pool_build(pool, o, 1, 4)
+        d_t, d_l, d_g = dev_i32(tails), dev_i32(tail_len), dev_i32(g)
+        for _ in range(3):
+            out = L.draft(h, d_t, d_l, d_g, prm)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(10):
+            out = L.draft(h, d_t, d_l, d_g, prm)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 100.0
+        sample = list(range(0, 4096, 512))
+        t0 = time.time()
+        want = [R.draft_one(pool, int(o[g[q]]), int(o[g[q] + 1]), tails[q], 16, 1, 4, 1, 64) for q in sample]
+        scan_ms = (time.time() - t0) * 1e3 / len(sample)
+        got_d, got_l = out[0].cpu().numpy(), out[1].cpu().numpy()
+        for q, (d, _) in zip(sample, want):
+            assert got_l[q] == len(d) and got_d[q, :len(d)].tolist() == d
+        print("%-10s laser_draft %.1f us per 4096 queries; host scan %.2f ms per query" % (name, us, scan_ms))
+        res[name] = (us, scan_ms)
+        h.free()
+    assert res["global"][1] > 20 * res["customised"][1]       # the scan pays for the pool size
+    assert res["global"][0] < 3 * res["customised"][0]        # the index does not
