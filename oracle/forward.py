@@ -58,14 +58,23 @@ def rope(x: torch.Tensor, pos: torch.Tensor, theta: float) -> torch.Tensor:
     return torch.cat([x1 * c - x2 * s, x2 * c + x1 * s], dim=-1)
 
 
+# The activations a bf16-operand implementation hands to a matrix product (the A operands): per
+# layer the attention-norm output, the rotated queries, the attention output, the FFN-norm output
+# and the SwiGLU output; after the last layer the final-norm output.
+MIRROR_SITES_PER_LAYER = 5
+MIRROR_SITES_FINAL = 1
+
+
 def _r(x: torch.Tensor, mirror: bool) -> torch.Tensor:
-    """Debug aid: round an activation to bf16 where a bf16 tensor-core path would."""
+    """Yardstick mode: round an activation to bf16 (nearest-even) where a bf16-operand
+    implementation would hand it to a matrix product; identity otherwise."""
     return x.to(torch.bfloat16).to(F64) if mirror else x
 
 
 def forward(W: Dict, cfg: Dict, kv: KVCache, seq_ids: Sequence[int],
             tokens: Sequence[np.ndarray], mirror_bf16: bool = False,
-            parents: Optional[Sequence[Sequence[int]]] = None) -> List[torch.Tensor]:
+            parents: Optional[Sequence[Sequence[int]]] = None,
+            hidden_out: Optional[List[torch.Tensor]] = None) -> List[torch.Tensor]:
     """One forward over the new rows of each listed sequence.
 
     tokens[j] holds the rows of sequence seq_ids[j]: the pending token followed by its
@@ -74,6 +83,11 @@ def forward(W: Dict, cfg: Dict, kv: KVCache, seq_ids: Sequence[int],
     acceptance step's job).  Returns one fp64 logits tensor [rows, vocab] per sequence.
     parents[j][i-1] (optional) = row of row i's parent in sequence j's token tree (row 0 is the
     root); without it the rows are a chain.
+    mirror_bf16 = True gives the yardstick of a bf16-operand implementation: the same forward with
+    the matrix-product A operands (MIRROR_SITES_PER_LAYER per layer, MIRROR_SITES_FINAL after the
+    last) rounded to bf16 and nothing else changed.
+    hidden_out (optional list) receives the residual stream [all rows, d_model] entering layer 0
+    and leaving every layer (observation only).
     """
     H, Hkv, dh = cfg["n_heads"], cfg["n_kv_heads"], cfg["head_dim"]
     eps, theta = cfg["rms_eps"], cfg["rope_theta"]
@@ -98,6 +112,8 @@ def forward(W: Dict, cfg: Dict, kv: KVCache, seq_ids: Sequence[int],
         if kv.ctx[s] + r > kv.capacity:
             raise ValueError("KV capacity exceeded")
     x = W["tok_emb"][flat].to(F64)
+    if hidden_out is not None:
+        hidden_out.append(x.clone())
     rep = H // Hkv
     for l, lw in enumerate(W["layers"]):
         h = _r(rmsnorm(x, lw["attn_norm"].to(F64), eps), mirror_bf16)
@@ -125,6 +141,8 @@ def forward(W: Dict, cfg: Dict, kv: KVCache, seq_ids: Sequence[int],
         up = h2 @ lw["w_up"].to(F64).T
         act = _r(gate * torch.sigmoid(gate) * up, mirror_bf16)  # SwiGLU: silu(gate) * up
         x = x + act @ lw["w_down"].to(F64).T
+        if hidden_out is not None:
+            hidden_out.append(x.clone())
     hn = _r(rmsnorm(x, W["final_norm"].to(F64), eps), mirror_bf16)
     logits = hn @ W["lm_head"].to(F64).T
     return [logits[starts[j]:starts[j + 1]] for j in range(len(rows))]

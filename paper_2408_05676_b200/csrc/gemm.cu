@@ -20,8 +20,6 @@
 //              cluster barrier, all six warps sum the partial tiles of the cluster through
 //              distributed shared memory in rank order (run-to-run identical, no partial sums
 //              in global memory) for the token columns this CTA owns and apply the fused epilogue.
-// Option PAIR: the CTAs of cluster ranks 2i, 2i+1 run one 256-row MMA together (cta_group::2),
-// each staging its own 128 weight rows and half of the token rows.
 // Every mbarrier wait is bounded: on expiry the CTA records LASER_ERR_TIMEOUT, drains its
 // copies, still joins the cluster barriers, frees its tensor memory and exits.
 #include <map>
@@ -60,26 +58,6 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// ---- two-CTA forms: the CTAs of ranks 2i and 2i+1 of a cluster run one 256-row MMA together ----
-__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// arrives on the barrier at the same shared-memory offset in every CTA named by the rank mask
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint32_t rank_mask) {
-  asm volatile(
-      "{\n.reg .b16 m;\ncvt.u16.u32 m, %1;\n"
-      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n}"
-      ::"r"(bar), "r"(rank_mask) : "memory");
-}
-// tile load whose completion bytes are counted on a barrier of the pair's first CTA
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t leader_bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(leader_bar) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -253,7 +231,7 @@ __device__ __forceinline__ void epi_qkv(const GemmEpilogue& e, const LaneCtx& c,
 }
 
 
-template <int EPI, bool PAIR>
+template <int EPI>
 __global__ void __launch_bounds__(kTcThreads, 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, const GemmEpilogue e,
                int N, int NT, int total_kb, int kb_per_split, int splits, int stages, int tmem_cols,
@@ -267,13 +245,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its prologue
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
-  // PAIR: the cluster holds 2 x splits CTAs, rank = 2 x (K range) + (half of a 256-row weight tile);
-  // each CTA stages its own 128 weight rows and half of the token rows.
-  const uint32_t w_bytes = kBM * 128, a_bytes = uint32_t(PAIR ? NT / 2 : NT) * 128, stage_bytes = w_bytes + a_bytes;
+  const uint32_t w_bytes = kBM * 128, a_bytes = uint32_t(NT) * 128, stage_bytes = w_bytes + a_bytes;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int csize = PAIR ? 2 * splits : splits, crank = blockIdx.x % csize, ttile = blockIdx.x / csize;
-  const int half = PAIR ? (crank & 1) : 0, krank = PAIR ? (crank >> 1) : crank;
-  const int wtile = PAIR ? 2 * blockIdx.y + half : blockIdx.y;
+  const int krank = blockIdx.x % splits, ttile = blockIdx.x / splits;   // cluster rank = K range
+  const int wtile = blockIdx.y;
   const int r0 = ttile * NT, n0 = wtile * kBM;
   const int kb0 = krank * kb_per_split;
   const int nkb = max(0, min(kb_per_split, total_kb - kb0));
@@ -289,17 +264,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     tma_prefetch_map(&tmA);
   }
   if (warp == 1) {
-    if (PAIR) {  // issued by the same warp of both CTAs of the pair
-      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(tmem_cols) : "memory");
-      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-    } else {
-      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(tmem_cols) : "memory");
-      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (PAIR) cluster_sync_all();   // the partner's copies count on this CTA's barriers: they must exist first
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = tmem_slot;
 
@@ -322,15 +291,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 
   if (warp == 0) {
     if (lane == 0) {  // ---- TMA producer ----
-      // PAIR: both CTAs' copies complete on the first CTA's barrier, which expects the bytes of both
-      const uint32_t full0 = PAIR ? map_to_rank(smem_u32(&full_bar[0]), uint32_t(crank & ~1)) : smem_u32(&full_bar[0]);
-      auto load = [&](uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
-        if (PAIR) tma_load_2d_pair(dst, tm, x, y, bar); else tma_load_2d(dst, tm, x, y, bar);
-      };
-      auto expect = [&](int s) {
-        if (!PAIR) mbar_expect_tx(smem_u32(&full_bar[s]), stage_bytes);
-        else if (half == 0) mbar_expect_tx(smem_u32(&full_bar[s]), 2 * stage_bytes);
-      };
+      const uint32_t full0 = smem_u32(&full_bar[0]);
+      auto load = [&](uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) { tma_load_2d(dst, tm, x, y, bar); };
+      auto expect = [&](int s) { mbar_expect_tx(smem_u32(&full_bar[s]), stage_bytes); };
       auto load_w = [&](int kb) {
         const int s = kb % stages, k = (kb0 + kb) * kBK;
         const uint32_t dst = tiles + uint32_t(s) * stage_bytes, bar = full0 + uint32_t(s) * 8;
@@ -339,7 +302,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       };
       auto load_a = [&](int kb) {
         const int s = kb % stages;
-        load(tiles + uint32_t(s) * stage_bytes + w_bytes, &tmA, (kb0 + kb) * kBK, r0 + half * (NT / 2), full0 + uint32_t(s) * 8);
+        load(tiles + uint32_t(s) * stage_bytes + w_bytes, &tmA, (kb0 + kb) * kBK, r0, full0 + uint32_t(s) * 8);
       };
       // The weights do not depend on the kernel before this one: fill the ring with weight
       // tiles first, and only then wait for the previous kernel's results (the activations).
@@ -357,13 +320,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         load_w(kb);
         load_a(kb);
       }
-      if (!ok && half == 0)  // drain copies still in flight (the partner's too) before the CTAs may exit
+      if (!ok)  // drain copies still in flight before the CTA may exit
         for (int j = max(0, kb - stages); j < kb; ++j) mbar_drain(smem_u32(&full_bar[j % stages]), (j / stages) & 1);
     }
   } else if (warp == 1) {
-    if (lane == 0 && half == 0) {  // ---- MMA issuer (PAIR: the first CTA issues for both) ----
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(NT >> 3) << 17) | (uint32_t((PAIR ? 2 * kBM : kBM) >> 4) << 24);
-      const uint32_t pair_mask = 3u << (crank & ~1);
+    if (lane == 0) {  // ---- MMA issuer ----
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(NT >> 3) << 17) | (uint32_t(kBM >> 4) << 24);
       bool ok = true;
       for (int kb = 0; kb < nkb && ok; ++kb) {
         const int s = kb % stages;
@@ -374,12 +336,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const uint64_t wdesc = umma_desc(w_addr), adesc = umma_desc(w_addr + w_bytes);
 #pragma unroll
         for (int k = 0; k < kBK / 16; ++k)  // 16 bf16 = 32 bytes further along K inside the swizzle span
-          if (PAIR) umma_bf16_pair(tmem_acc, wdesc + uint64_t(k * 2), adesc + uint64_t(k * 2), idesc, (kb | k) != 0);
-          else umma_bf16(tmem_acc, wdesc + uint64_t(k * 2), adesc + uint64_t(k * 2), idesc, (kb | k) != 0);
-        if (PAIR) umma_commit_pair(smem_u32(&empty_bar[s]), pair_mask); else umma_commit(smem_u32(&empty_bar[s]));
+          umma_bf16(tmem_acc, wdesc + uint64_t(k * 2), adesc + uint64_t(k * 2), idesc, (kb | k) != 0);
+        umma_commit(smem_u32(&empty_bar[s]));
       }
       // arrives when every MMA issued so far has finished
-      if (PAIR) umma_commit_pair(smem_u32(&acc_bar), pair_mask); else umma_commit(smem_u32(&acc_bar));
+      umma_commit(smem_u32(&acc_bar));
     }
   } else {
     // ---- epilogue warps, part 1: everything that can be done before the accumulator is ready ----
@@ -469,7 +430,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       constexpr int S = decltype(s_tag)::value, RB = decltype(rb_tag)::value;
       uint32_t rank_base[S];
 #pragma unroll
-      for (int q = 0; q < S; ++q) rank_base[q] = S > 1 ? map_to_rank(tiles, uint32_t(PAIR ? 2 * q + half : q)) : tiles;
+      for (int q = 0; q < S; ++q) rank_base[q] = S > 1 ? map_to_rank(tiles, uint32_t(q)) : tiles;
       for (int jb = warp * RB; jb < own; jb += (kTcThreads / 32) * RB) {
         float4 part[RB][S], g0[RB], g1[RB];
 #pragma unroll
@@ -510,11 +471,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
   }
   __syncwarp();
-  if (splits > 1 || PAIR) cluster_sync_all();  // peers may still be reading this CTA's staged tile or tensor memory
+  if (splits > 1) cluster_sync_all();  // peers may still be reading this CTA's staged tile or tensor memory
   __syncthreads();
   if (warp == 1) {
-    if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(tmem_cols) : "memory");
-    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(tmem_cols) : "memory");
   }
   if (threadIdx.x == 0 && abort_flag) atomicCAS(status, 0, LASER_ERR_TIMEOUT);
 }
@@ -545,20 +505,16 @@ laser_status tensor_map(GemmState* st, const void* ptr, int rows, int cols, int 
 
 struct TcShape { int n_ttiles, NT, stages, tmem_cols; size_t smem; };
 }  // namespace
-// Tuning aids: non-zero values override the modelled split count / the stage count;
-// g_force_pair: 0 (default) = single-CTA MMA; 1 = two-CTA MMA (cta_group::2) for models whose matrices all
-// have an even number of weight tiles.  Both forms measure the same step time; the single-CTA form is the
-// default because it keeps tensor-memory allocation local to an SM.
+// Tuning aids: non-zero values override the modelled split count / the stage count.
 int g_force_splits = 0;
 int g_force_stages = 0;
-int g_force_pair = 0;
 namespace {
 
-TcShape tc_shape(int R_pad, bool pair) {
+TcShape tc_shape(int R_pad) {
   TcShape s;
   s.n_ttiles = ceil_div(R_pad, kMaxNT);
   s.NT = ceil_div(ceil_div(R_pad, s.n_ttiles), 16) * 16;
-  const int stage_bytes = kBM * 128 + (pair ? s.NT / 2 : s.NT) * 128;
+  const int stage_bytes = kBM * 128 + s.NT * 128;
   s.stages = std::max(2, std::min(kMaxStages, kSmemBudget / stage_bytes));
   if (g_force_stages) s.stages = std::max(2, std::min(s.stages, g_force_stages));
   s.tmem_cols = 32;
@@ -567,18 +523,17 @@ TcShape tc_shape(int R_pad, bool pair) {
   return s;
 }
 
-template <int EPI, bool PAIR>
+template <int EPI>
 laser_status launch_epi(const CUtensorMap& tw, const CUtensorMap& ta, const GemmEpilogue& e, int N, const TcShape& sh,
                         int n_wtiles, int total_kb, int kbps, int splits, int32_t* status, cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = PAIR ? dim3(unsigned(sh.n_ttiles * splits * 2), unsigned(n_wtiles / 2), 1)
-                     : dim3(unsigned(sh.n_ttiles * splits), unsigned(n_wtiles), 1);
+  cfg.gridDim = dim3(unsigned(sh.n_ttiles * splits), unsigned(n_wtiles), 1);
   cfg.blockDim = dim3(kTcThreads, 1, 1);
   cfg.dynamicSmemBytes = sh.smem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = unsigned(PAIR ? 2 * splits : splits);
+  attr[0].val.clusterDim.x = unsigned(splits);
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   // programmatic dependent launch: this kernel may begin while the previous one drains; it
@@ -587,7 +542,7 @@ laser_status launch_epi(const CUtensorMap& tw, const CUtensorMap& ta, const Gemm
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  LASER_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI, PAIR>, tw, ta, e, N, sh.NT, total_kb, kbps, splits, sh.stages,
+  LASER_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI>, tw, ta, e, N, sh.NT, total_kb, kbps, splits, sh.stages,
                                 sh.tmem_cols, status));
   return LASER_OK;
 }
@@ -595,18 +550,10 @@ laser_status launch_epi(const CUtensorMap& tw, const CUtensorMap& ta, const Gemm
 laser_status prepare(GemmState* st) {
   if (st->ready) return LASER_OK;
   const int bytes = kSmemBudget + 2048;
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
   st->ready = true;
   return LASER_OK;
 }
@@ -615,12 +562,11 @@ laser_status prepare(GemmState* st) {
 // fastest with roughly 200 CTAs (of the 296 resident slots), whatever the matrix: 1 for 172 or
 // 250 weight tiles, 2 for 96, 6 for 32.  Fewer CTAs leave SMs idle, more add start-up and
 // cluster-reduction cost faster than they shorten the K loop.
-int pick_splits(int R_pad, int N, int K, int epi, bool pair) {
+int pick_splits(int R_pad, int N, int K, int epi) {
   const int n_wtiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
-  const int tiles = n_wtiles * tc_shape(R_pad, pair).n_ttiles, total_kb = ceil_div(K, kBK);
+  const int tiles = n_wtiles * tc_shape(R_pad).n_ttiles, total_kb = ceil_div(K, kBK);
   int s = g_force_splits ? g_force_splits : int(208.0 / tiles + 0.5);
-  // clusters of up to 12 CTAs schedule well (they need the non-portable size attribute), larger ones do not
-  s = std::max(1, std::min(s, std::min(total_kb, pair ? 6 : 8)));
+  s = std::max(1, std::min(s, std::min(total_kb, 8)));   // portable cluster size
   while (s > 1 && ceil_div(total_kb, s) * (s - 1) >= total_kb) --s;   // no rank without K blocks
   return s;
 }
@@ -636,21 +582,13 @@ laser_status gemm_fused(laser_model* m, const __nv_bfloat16* A, const __nv_bfloa
   GemmState* st = get_state(m);
   LASER_TRY(prepare(st));
   const int n_wtiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
-  // Two weight tiles share one 256-row MMA of a CTA pair (each CTA then stages only half of the
-  // token rows) when the tiles come in pairs.
-  // All GEMMs of a model run the same MMA form (m->pair_mma): kernels of consecutive launches share
-  // SMs under programmatic dependent launch, and a step that alternated between one-CTA and two-CTA
-  // tensor-memory allocation stopped making progress when it was tried.
-  const bool pair = g_force_pair != 0 && m->pair_mma && n_wtiles % 2 == 0;
-  const int splits = pick_splits(R_pad, N, K, epi, pair);
-  const TcShape sh = tc_shape(R_pad, pair);
+  const int splits = pick_splits(R_pad, N, K, epi);
+  const TcShape sh = tc_shape(R_pad);
   const CUtensorMap *tw = nullptr, *ta = nullptr;
   LASER_TRY(tensor_map(st, W, N, K, 64, &tw));
-  LASER_TRY(tensor_map(st, A, m->R_pad, K, pair ? sh.NT / 2 : sh.NT, &ta));
+  LASER_TRY(tensor_map(st, A, m->R_pad, K, sh.NT, &ta));
   const int total_kb = ceil_div(K, kBK), kbps = ceil_div(total_kb, splits);
-#define LASER_GEMM_LAUNCH(E)                                                                                            \
-  if (pair) LASER_TRY((launch_epi<E, true>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, m->status, stream)));  \
-  else LASER_TRY((launch_epi<E, false>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, m->status, stream)));
+#define LASER_GEMM_LAUNCH(E) LASER_TRY((launch_epi<E>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, m->status, stream)));
   switch (epi) {
     case EPI_PLAIN: LASER_GEMM_LAUNCH(EPI_PLAIN) break;
     case EPI_RESID: LASER_GEMM_LAUNCH(EPI_RESID) break;

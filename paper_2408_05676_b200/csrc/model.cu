@@ -298,11 +298,6 @@ LASER_API laser_status laser_model_create(const laser_model_cfg* cfg, const lase
   m->dq = cfg->n_heads * cfg->head_dim;
   m->dkv = cfg->n_kv_heads * cfg->head_dim;
   m->dqkv = m->dq + 2 * m->dkv;
-  {  // the two-CTA MMA needs weight tiles in pairs, in every matrix of the model
-    auto even = [](int tiles) { return tiles % 2 == 0; };
-    m->pair_mma = even(ceil_div(m->dqkv, 128)) && even(ceil_div(cfg->d_model, 128)) && even(ceil_div(cfg->d_ffn, 64)) &&
-                  even(ceil_div(cfg->vocab, 128));
-  }
   m->tok_emb = static_cast<const bf16*>(w->tok_emb);
   m->lm_head = static_cast<const bf16*>(w->lm_head);
   m->final_norm = static_cast<const bf16*>(w->final_norm);

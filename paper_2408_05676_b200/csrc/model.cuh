@@ -28,7 +28,6 @@ struct laser_model {
   unsigned long long* row_mask = nullptr;  // [R_pad] token tree: rows of its sequence a row attends to (bit j = row j)
   int32_t* status = nullptr;       // first device-side error of the stream, 0 = none
   void* gemm_state = nullptr;      // tensor-map cache of the tensor-core GEMM
-  bool pair_mma = true;            // every weight matrix has an even number of 128-row tiles: two-CTA MMA throughout
   // optional per-class kernel timing (class 0 = GEMM, 1 = attention)
   bool profile = false;
   std::vector<cudaEvent_t> prof_events[2];  // begin/end pairs

@@ -15,8 +15,11 @@ from paper_2408_05676_b200 import synth
 
 pytestmark = pytest.mark.gpu
 NEAR_TIE = 1e-3          # margin below which a different decision counts as a near-tie
-LOGIT_TOL = 2e-2         # allowed max-abs logit error of the bf16 path; a deciding gap below
-                         # 2 * LOGIT_TOL can legitimately flip and is counted, not failed
+LOGIT_TOL = 2e-2         # allowed max-abs logit error of the bf16 path: a deciding gap below 2 * LOGIT_TOL
+                         # can flip although both sides are within tolerance.  Such steps are counted and
+                         # bounded on their own (at most MAX_WITHIN_TOL per run), never folded into the
+                         # near-ties; a wider gap is a hard mismatch and fails
+MAX_WITHIN_TOL = 1
 
 
 @pytest.fixture(scope="module")
@@ -56,7 +59,8 @@ def setup(L):
 def _teacher_forced(cfg, Wc, pool, offs, prompts, gid, out, prm, mode, k, p, temp=False, tree=False):
     """Replays the library's committed tokens through the oracle.  Every step the oracle drafts
     and verifies from the library's own history; its emitted tokens must equal the library's
-    next tokens unless the deciding logits are within NEAR_TIE."""
+    next tokens unless the deciding logits are within NEAR_TIE.  Returns (steps, exact, near-ties below
+    NEAR_TIE, decisions flipped inside twice the logit tolerance); hard mismatches assert."""
     near, exact, steps = 0, 0, 0
     within_tol = []
     for b in range(len(prompts)):
@@ -109,7 +113,7 @@ def _teacher_forced(cfg, Wc, pool, offs, prompts, gid, out, prm, mode, k, p, tem
             kvo.ctx[0] += len(em)
             seq.extend(em)
             at += len(em)
-    return exact, near + len(within_tol), steps
+    return steps, exact, near, len(within_tol)
 
 
 def test_strict_equals_greedy_and_oracle(L, setup):
@@ -123,9 +127,10 @@ def test_strict_equals_greedy_and_oracle(L, setup):
     assert spec["out"] == greedy["out"]                      # lossless
     assert spec["emitted"] == 4 * 64 and spec["steps"] < greedy["steps"]
     assert (L.kv_get_len(kv, [0, 1, 2, 3]) == 63 + 64).all()
-    exact, near, steps = _teacher_forced(cfg, Wc, pool, offs, prompts, gid, spec["out"], prm, A.STRICT, 1, 0.0)
-    print("strict: steps", steps, "exact", exact, "near-tie", near, "accepted/step", spec["accepted"] / spec["steps"])
-    assert near <= max(2, steps // 20)
+    steps, exact, near, wtol = _teacher_forced(cfg, Wc, pool, offs, prompts, gid, spec["out"], prm, A.STRICT, 1, 0.0)
+    print("strict: steps", steps, "exact", exact, "near-tie(<1e-3)", near, "within 2x tolerance", wtol, "hard 0",
+          "accepted/step", spec["accepted"] / spec["steps"])
+    assert exact + near + wtol == steps and near <= max(2, steps // 20) and wtol <= MAX_WITHIN_TOL
 
 
 def test_relaxed_matches_oracle_under_teacher_forcing(L, setup):
@@ -142,10 +147,10 @@ def test_relaxed_matches_oracle_under_teacher_forcing(L, setup):
     prm = L.make_params(K=8, n_min=1, n_max=3, max_occ=64, mode=L.MODE_RELAXED, topk=2, p=p_low, max_new=48)
     rel = L.generate(m, kv, h, prompts, gid, prm)
     assert rel["accepted"] > 0 and rel["emitted"] == 4 * 48
-    exact, near, steps = _teacher_forced(cfg, Wc, pool, offs, prompts, gid, rel["out"], prm, A.RELAXED, 2,
-                                         float(np.float32(p_low)))
-    print("relaxed: steps", steps, "exact", exact, "near-tie", near)
-    assert near <= max(2, steps // 10)
+    steps, exact, near, wtol = _teacher_forced(cfg, Wc, pool, offs, prompts, gid, rel["out"], prm, A.RELAXED, 2,
+                                               float(np.float32(p_low)))
+    print("relaxed: steps", steps, "exact", exact, "near-tie(<1e-3)", near, "within 2x tolerance", wtol, "hard 0")
+    assert exact + near + wtol == steps and near <= max(2, steps // 10) and wtol <= MAX_WITHIN_TOL
 
 
 def test_temporary_branches(L, setup):
@@ -166,11 +171,11 @@ def test_temporary_branches(L, setup):
     temp = L.generate(m, kv, h, tprompts, gid, prm)
     assert temp["out"] == greedy["out"] and temp["emitted"] == 4 * 48          # lossless
     assert temp["drafted"] > plain["drafted"]                                  # the history adds drafts
-    exact, near, steps = _teacher_forced(cfg, Wc, pool, offs, tprompts, gid, temp["out"], prm, A.STRICT, 1, 0.0,
-                                         temp=True)
-    print("temp: steps", steps, "exact", exact, "near-tie", near, "drafted", temp["drafted"], "plain", plain["drafted"],
-          "accepted", temp["accepted"])
-    assert near <= max(2, steps // 20)
+    steps, exact, near, wtol = _teacher_forced(cfg, Wc, pool, offs, tprompts, gid, temp["out"], prm, A.STRICT, 1, 0.0,
+                                               temp=True)
+    print("temp: steps", steps, "exact", exact, "near-tie(<1e-3)", near, "within 2x tolerance", wtol, "hard 0",
+          "drafted", temp["drafted"], "plain", plain["drafted"], "accepted", temp["accepted"])
+    assert exact + near + wtol == steps and near <= max(2, steps // 20) and wtol <= MAX_WITHIN_TOL
     with pytest.raises(L.LaserError):      # the temporary-branch draft keeps a capped occurrence list
         L.generate(m, kv, h, tprompts, gid, L.make_params(K=8, n_min=1, n_max=3, max_occ=0, max_new=8, temp_branches=1))
 
@@ -189,21 +194,21 @@ def test_tree_drafting(L, setup):
         tree = L.generate(m, kv, h, prompts, gid, prm)
         assert tree["out"] == greedy["out"] and tree["emitted"] == 4 * 64
         assert (L.kv_get_len(kv, [0, 1, 2, 3]) == 63 + 64).all()
-        exact, near, steps = _teacher_forced(cfg, Wc, pool, offs, prompts, gid, tree["out"], prm, A.STRICT, 1, 0.0,
-                                             temp=bool(temp), tree=True)
-        print("tree (temp", temp, "): steps", steps, "exact", exact, "near-tie", near, "accepted/step",
-              tree["accepted"] / tree["steps"], "chain steps", chain["steps"])
-        assert near <= max(2, steps // 20)
+        steps, exact, near, wtol = _teacher_forced(cfg, Wc, pool, offs, prompts, gid, tree["out"], prm, A.STRICT, 1, 0.0,
+                                                   temp=bool(temp), tree=True)
+        print("tree (temp", temp, "): steps", steps, "exact", exact, "near-tie(<1e-3)", near, "within 2x tolerance", wtol,
+              "hard 0", "accepted/step", tree["accepted"] / tree["steps"], "chain steps", chain["steps"])
+        assert exact + near + wtol == steps and near <= max(2, steps // 20) and wtol <= MAX_WITHIN_TOL
         if not temp:
             assert tree["steps"] <= chain["steps"]
     # relaxed verification of a tree
     prm = L.make_params(K=8, n_min=1, n_max=3, max_occ=64, mode=L.MODE_RELAXED, topk=2, p=1e-4, max_new=48, tree=1)
     rel = L.generate(m, kv, h, prompts, gid, prm)
     assert rel["accepted"] > 0 and rel["emitted"] == 4 * 48
-    exact, near, steps = _teacher_forced(cfg, Wc, pool, offs, prompts, gid, rel["out"], prm, A.RELAXED, 2,
-                                         float(np.float32(1e-4)), tree=True)
-    print("tree relaxed: steps", steps, "exact", exact, "near-tie", near)
-    assert near <= max(2, steps // 10)
+    steps, exact, near, wtol = _teacher_forced(cfg, Wc, pool, offs, prompts, gid, rel["out"], prm, A.RELAXED, 2,
+                                               float(np.float32(1e-4)), tree=True)
+    print("tree relaxed: steps", steps, "exact", exact, "near-tie(<1e-3)", near, "within 2x tolerance", wtol, "hard 0")
+    assert exact + near + wtol == steps and near <= max(2, steps // 10) and wtol <= MAX_WITHIN_TOL
 
 
 def test_eos_and_argument_checks(L, setup):

@@ -136,3 +136,124 @@ def test_rope_properties():
     r = O.rope(x, p, 1e4)[1, 0]
     assert abs(r[1] - (x[1, 0, 1] * math.cos(ang) - x[1, 0, 9] * math.sin(ang))) < 1e-12
     assert abs(r[9] - (x[1, 0, 9] * math.cos(ang) + x[1, 0, 1] * math.sin(ang))) < 1e-12
+
+
+# ---- the bf16-operand yardstick (mirror_bf16 = True) -------------------------------------------------
+
+def _bf(t):
+    return t.bfloat16().double()
+
+
+def _hand_mirror_forward(W, cfg, toks, round_sites=True, extra_site=False, skip_site=0):
+    """Whole-sequence, cache-free composition from library routines that rounds to bf16 exactly the
+    six kinds of matrix-product operands the yardstick names (norm output, rotated Q, attention output,
+    FFN-norm output, SwiGLU output, final-norm output) - and K, V by the cache contract."""
+    r = _bf if round_sites else (lambda t: t)
+    ident = lambda t: t
+    H, Hkv, dh = cfg["n_heads"], cfg["n_kv_heads"], cfg["head_dim"]
+    T = len(toks)
+    x = W["tok_emb"].double()[torch.as_tensor(toks, dtype=torch.long)]
+    inv = 1.0 / (cfg["rope_theta"] ** (torch.arange(0, dh, 2, dtype=torch.float64) / dh))
+    rot = torch.polar(torch.ones(T, dh // 2, dtype=torch.float64),
+                      torch.arange(T, dtype=torch.float64)[:, None] * inv[None, :])
+
+    def rope_c(t):
+        z = torch.complex(t[..., :dh // 2], t[..., dh // 2:]) * rot[:, None, :]
+        return torch.cat([z.real, z.imag], dim=-1)
+
+    for lw in W["layers"]:
+        h = r(F.rms_norm(x, (x.shape[-1],), lw["attn_norm"].double(), cfg["rms_eps"]))            # site 1
+        q = r(rope_c(F.linear(h, lw["wq"].double()).view(T, H, dh)))                               # site 2
+        k = _bf(rope_c(F.linear(h, lw["wk"].double()).view(T, Hkv, dh)))
+        v = _bf(F.linear(h, lw["wv"].double()).view(T, Hkv, dh))
+        k = k.repeat_interleave(H // Hkv, dim=1)
+        v = v.repeat_interleave(H // Hkv, dim=1)
+        a = F.scaled_dot_product_attention(q.transpose(0, 1), k.transpose(0, 1), v.transpose(0, 1),
+                                           is_causal=True).transpose(0, 1).reshape(T, H * dh)
+        x = x + F.linear((ident if skip_site == 3 else r)(a), lw["wo"].double())                   # site 3
+        h = r(F.rms_norm(x, (x.shape[-1],), lw["ffn_norm"].double(), cfg["rms_eps"]))             # site 4
+        gate = F.linear(h, lw["w_gate"].double())
+        if extra_site:
+            gate = _bf(gate)                                                                       # not a site
+        act = r(F.silu(gate) * F.linear(h, lw["w_up"].double()))                                   # site 5
+        x = x + F.linear(act, lw["w_down"].double())
+    return F.linear(r(F.rms_norm(x, (x.shape[-1],), W["final_norm"].double(), cfg["rms_eps"])),   # final site
+                    W["lm_head"].double())
+
+
+def test_mirror_with_identity_rounding_is_the_exact_forward_bit_for_bit(monkeypatch):
+    W = synth.make_weights(CFG, seed=21, std=0.2, gain_jitter=0.3)
+    toks = synth.make_prompt(11, CFG["vocab"], 6)
+    exact = O.forward(W, CFG, O.KVCache(CFG, 1, 16), [0], [toks])[0]
+    monkeypatch.setattr(O, "_r", lambda x, mirror: x)
+    kv = O.KVCache(CFG, 1, 16)
+    got = O.forward(W, CFG, kv, [0], [toks], mirror_bf16=True)[0]
+    assert torch.equal(got, exact)
+
+
+def test_mirror_rounds_exactly_the_named_operand_sites(monkeypatch):
+    calls = []
+    real = O._r
+
+    def spy(x, mirror):
+        calls.append((tuple(x.shape), bool(mirror)))
+        return real(x, mirror)
+
+    monkeypatch.setattr(O, "_r", spy)
+    W = synth.make_weights(CFG, seed=22, std=0.2)
+    toks = synth.make_prompt(7, CFG["vocab"], 7)
+    O.forward(W, CFG, O.KVCache(CFG, 1, 8), [0], [toks], mirror_bf16=True)
+    L, d, f = CFG["n_layers"], CFG["d_model"], CFG["d_ffn"]
+    assert O.MIRROR_SITES_PER_LAYER == 5 and O.MIRROR_SITES_FINAL == 1
+    assert len(calls) == L * O.MIRROR_SITES_PER_LAYER + O.MIRROR_SITES_FINAL
+    assert all(m for _, m in calls)
+    per_layer = [(7, d), (7, CFG["n_heads"], CFG["head_dim"]), (7, CFG["n_heads"] * CFG["head_dim"]), (7, d), (7, f)]
+    assert [s for s, _ in calls] == per_layer * L + [(7, d)]
+
+
+def test_mirror_equals_a_hand_composition_that_rounds_those_sites_only():
+    for n_layers in (1, 2):
+        cfg = dict(CFG, n_layers=n_layers)
+        W = synth.make_weights(cfg, seed=23, std=0.2, gain_jitter=0.3)
+        toks = synth.make_prompt(19, cfg["vocab"], 8)
+        kv = O.KVCache(cfg, 1, 32)
+        got, i = [], 0
+        for chunk in (6, 1, 9, 3):
+            got.append(O.forward(W, cfg, kv, [0], [toks[i:i + chunk]], mirror_bf16=True)[0])
+            kv.ctx[0] += chunk
+            i += chunk
+        got = torch.cat(got)
+        want = _hand_mirror_forward(W, cfg, toks)
+        assert (got - want).abs().max() < 1e-9
+        # the rounding is really there (a mirror that rounds nothing would equal the exact forward),
+        # it is small, and a composition with one site fewer or one more is told apart
+        exact = _hand_mirror_forward(W, cfg, toks, round_sites=False)
+        gap = float((want - exact).abs().max())
+        assert 1e-4 < gap < 0.2
+        kv2 = O.KVCache(cfg, 1, 32)
+        ex2 = O.forward(W, cfg, kv2, [0], [toks])[0]
+        assert (ex2 - exact).abs().max() < 1e-9
+        assert (got - _hand_mirror_forward(W, cfg, toks, extra_site=True)).abs().max() > 1e-5
+        assert (got - _hand_mirror_forward(W, cfg, toks, skip_site=3)).abs().max() > 1e-5
+
+
+def test_mirror_stays_within_the_logit_tolerance_on_the_tiny_shape():
+    cfg = synth.model_cfg("tiny")
+    W = synth.make_weights(cfg, seed=0)
+    toks = synth.make_prompt(24, cfg["vocab"], 2000)
+    a = O.forward(W, cfg, O.KVCache(cfg, 1, 32), [0], [toks])[0]
+    b = O.forward(W, cfg, O.KVCache(cfg, 1, 32), [0], [toks], mirror_bf16=True)[0]
+    err = float((a - b).abs().max())
+    assert 0 < err < 2e-2
+
+
+def test_hidden_out_observes_the_residual_stream_without_changing_the_result():
+    W = synth.make_weights(CFG, seed=24, std=0.2)
+    toks = synth.make_prompt(5, CFG["vocab"], 9)
+    hs = []
+    a = O.forward(W, CFG, O.KVCache(CFG, 1, 8), [0], [toks], hidden_out=hs)[0]
+    b = O.forward(W, CFG, O.KVCache(CFG, 1, 8), [0], [toks])[0]
+    assert torch.equal(a, b) and len(hs) == CFG["n_layers"] + 1
+    assert torch.equal(hs[0], W["tok_emb"].double()[torch.as_tensor(toks, dtype=torch.long)])
+    last = O.rmsnorm(hs[-1], W["final_norm"].double(), CFG["rms_eps"]) @ W["lm_head"].double().T
+    assert (last - a).abs().max() < 1e-12
