@@ -6,7 +6,9 @@ One step = draft retrieval (laser_draft) -> row assembly -> verify forward over
 [pending token + 8 drafts] for 16 sequences with 512 cached tokens each
 (laser_verify_step) -> acceptance + KV commit (laser_accept_commit), on seeded synthetic
 weights, cache and pool.  Prints one JSON line (rank 0).  `--impl reference` times the CPU
-oracle on a bounded sample of the same workload instead.
+oracle on a bounded sample of the same workload instead.  `--gpus N` started without a launcher
+spawns N replicas itself (one process per GPU, each serving its own block of pool groups); under
+torchrun the ranks are taken from the environment.
 """
 from __future__ import annotations
 
@@ -32,7 +34,6 @@ B, K, CTX, N_MAX = 16, 8, 512, 4
 POOL_TOKENS, POOL_GROUPS = 5_000_000, 1000
 # read + write MB of the QKV, O, gate/up and down launches of a layer x 32 + the LM head, from the ncu capture
 GEMM_DRAM_TRAFFIC_PER_STEP = int((105.7 + 45.6 + 193.5 + 108.8) * 32e6 + 268.0e6)
-SAMPLE_LAYERS = 4          # layers the CPU baseline really runs (time is extrapolated to all)
 
 
 def measured_peaks():
@@ -103,8 +104,11 @@ def algorithmic_bytes(cfg, n_seqs, ctx, rows_per_seq):
                 total=weights + kv_read + kv_write + logits)
 
 
-def build_workload(L, dev, cfg):
-    """Weights, synthetic cache, greedy continuation, corrupted drafts, pool holding them."""
+def build_workload(L, dev, cfg, rank=0, world=1):
+    """Weights, synthetic cache, greedy continuation, corrupted drafts, pool holding them.
+    With several replicas each rank serves its own block of groups (replicas.shard_groups): its
+    sequences belong to those groups and its pool holds only their tokens."""
+    from paper_2408_05676_b200 import replicas
     W = synth.make_weights(cfg, seed=0, device=dev)
     model = L.model_create(cfg, W, max_batch=B)
     pages_per_seq = (CTX + K + 1 + 15) // 16 + 1
@@ -138,12 +142,17 @@ def build_workload(L, dev, cfg):
     drafts = synth.corrupt_drafts(greedy, second, cfg["vocab"], seed=8)
     # pool: Zipf/template background; group of sequence b also holds "tail + drafts" as a document
     pool, offs = synth.make_zipf_pool(POOL_TOKENS, POOL_GROUPS, vocab=cfg["vocab"], seed=42)
-    gid = (np.arange(B) * 61 % POOL_GROUPS).astype(np.int32)
+    mine = replicas.shard_groups(POOL_GROUPS, rank, world)
+    n_mine = len(mine)
+    pool, offs = pool[offs[mine.start]:offs[mine.stop]], offs[mine.start:mine.stop + 1] - offs[mine.start]
+    gid = (np.arange(B) * 61 % n_mine).astype(np.int32)          # group ids local to this rank's pool
     tails = np.concatenate([rng.integers(0, cfg["vocab"], size=(B, N_MAX - 1)).astype(np.int32),
                             last_np[:, None]], axis=1)
+    pool_bg, offs_bg = pool, offs
     parts, new_offs = [], [0]
     doc_of = {int(g): b for b, g in enumerate(gid)}
-    for g in range(POOL_GROUPS):
+    assert len(doc_of) == B, "every sequence needs a group of its own"
+    for g in range(n_mine):
         parts.append(pool[offs[g]:offs[g + 1]])
         n = int(offs[g + 1] - offs[g])
         if g in doc_of:
@@ -159,8 +168,8 @@ def build_workload(L, dev, cfg):
     parts3, offs3 = [], [0]
     alt = [drafts, synth.corrupt_drafts(greedy, second, cfg["vocab"], seed=9),
            synth.corrupt_drafts(greedy, second, cfg["vocab"], seed=10)]
-    base, boffs = synth.make_zipf_pool(POOL_TOKENS, POOL_GROUPS, vocab=cfg["vocab"], seed=42)
-    for g in range(POOL_GROUPS):
+    base, boffs = pool_bg, offs_bg
+    for g in range(n_mine):
         parts3.append(base[boffs[g]:boffs[g + 1]])
         n = int(boffs[g + 1] - boffs[g])
         if g in doc_of:
@@ -169,7 +178,7 @@ def build_workload(L, dev, cfg):
                 parts3.append(doc)
                 n += len(doc)
         offs3.append(offs3[-1] + n)
-    return dict(pool3=np.concatenate(parts3), offs3=np.asarray(offs3, dtype=np.int64), cfg=cfg, W=W, model=model, kv=kv, seq_ids=seq_ids, lens=lens, last=last_np, tails=tails, gid=gid,
+    return dict(groups=(mine.start, mine.stop), pool3=np.concatenate(parts3), offs3=np.asarray(offs3, dtype=np.int64), cfg=cfg, W=W, model=model, kv=kv, seq_ids=seq_ids, lens=lens, last=last_np, tails=tails, gid=gid,
                 drafts=drafts, greedy=greedy, pool=pool, offs=offs)
 
 
@@ -180,8 +189,10 @@ def run_ours(args):
     torch.cuda.set_device(local)
     dev = "cuda:%d" % local
     dist, rank, world = replicas.init("nccl", torch.device(dev))
+    if world != args.gpus and rank == 0:
+        print("bench.py: --gpus %d but WORLD_SIZE is %d: reporting what runs" % (args.gpus, world), file=sys.stderr)
     cfg = synth.model_cfg("7b", n_layers=args.layers)
-    wl = build_workload(L, dev, cfg)
+    wl = build_workload(L, dev, cfg, rank, world)
     model, kv, seq_ids, lens = wl["model"], wl["kv"], wl["seq_ids"], wl["lens"]
     t0 = time.time()
     pool = L.pool_build(wl["pool"], wl["offs"], 1, N_MAX)
@@ -353,7 +364,7 @@ def run_ours(args):
                    "model_shape": "llama-2-7b", "layers": args.layers, "batch": B, "ctx": CTX, "draft_len": K,
                    "pool_tokens": int(len(wl["pool"])), "pool_groups": POOL_GROUPS, "suffix_n": [1, N_MAX],
                    "max_occ": 64, "l2": "inputs larger than L2 (13.2 GB of weights + 4.3 GB of KV per step)",
-                   "parallelism": "replicas x%d" % world},
+                   "parallelism": "replicas x%d, groups sharded by rank (rank 0 serves groups %d..%d), no data-path collective" % (world, wl["groups"][0], wl["groups"][1] - 1)},
         "clocks": main["clocks"],
         "e2e": {"value": e2e_value, "unit": "tokens/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in h_in)),
@@ -377,85 +388,99 @@ def run_ours(args):
                        for name, r in res.items()},
         "p_cal": p_cal, "pool_build_s": pool_build_s, "launches_per_step": int(main["launches"]),
     }
-    if args.layers >= SAMPLE_LAYERS:
-        out["cpu_baseline"] = cpu_baseline(wl, sample="1 of 16 sequences, %d of 32 layers run, time extrapolated" % SAMPLE_LAYERS)
+    if world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(wl)
     print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
 
 
 # ---------------------------------------------------------------------------------------------
-def oracle_sample(cfg, W_cpu, kv_rows, pool, offs, tail, gid, repeat=1):
-    """One sequence through the oracle: draft, forward over SAMPLE_LAYERS layers (timed apart from
-    the embedding/LM-head part so that the time can be scaled to all layers), acceptance."""
+def oracle_step(cfg, W_cpu, kv_rows, pool, offs, tail, gid):
+    """One sequence of the workload through the oracle as it stands: draft retrieval in its group,
+    verify forward over [pending token + drafts] through every layer against its 512 cached tokens,
+    strict acceptance.  Returns (seconds spent, tokens emitted, accepted drafts).  Nothing is scaled."""
     from oracle import accept as OA
     from oracle import forward as OF
     from oracle import retrieval as OR
-    cfg_s = dict(cfg, n_layers=SAMPLE_LAYERS)
-    cfg_0 = dict(cfg, n_layers=0)
-    W0 = dict(W_cpu, layers=[])
-    times = []
-    for _ in range(repeat):
-        t0 = time.perf_counter()
-        d, _ = OR.draft_one(pool, int(offs[gid]), int(offs[gid + 1]), tail, K, 1, N_MAX, 1, 64)
-        rows = np.asarray([tail[-1]] + d, np.int32)
-        t1 = time.perf_counter()
-        okv = OF.KVCache(cfg_s, 1, CTX + K + 2)
-        for l in range(SAMPLE_LAYERS):
-            okv.k[l, 0, :CTX] = kv_rows[l][0].view(CTX, cfg["n_kv_heads"], cfg["head_dim"])
-            okv.v[l, 0, :CTX] = kv_rows[l][1].view(CTX, cfg["n_kv_heads"], cfg["head_dim"])
-        okv.ctx[0] = CTX
-        t2 = time.perf_counter()
-        logits = OF.forward(W_cpu, cfg_s, okv, [0], [rows])[0]
-        t3 = time.perf_counter()
-        OF.forward(W0, cfg_0, OF.KVCache(cfg_0, 1, 16), [0], [rows])
-        t4 = time.perf_counter()
-        a, em = OA.accept_one(logits.float().numpy(), rows, len(rows), OA.STRICT, 2, 0.1)
-        t5 = time.perf_counter()
-        head = t4 - t3
-        per_layer = max((t3 - t2) - head, 0.0) / SAMPLE_LAYERS
-        total = (t1 - t0) + head + per_layer * cfg["n_layers"] + (t5 - t4)
-        times.append((total, len(em)))
-    return times
+    t0 = time.perf_counter()
+    d, _ = OR.draft_one(pool, int(offs[gid]), int(offs[gid + 1]), tail, K, 1, N_MAX, 1, 64)
+    rows = np.asarray([tail[-1]] + d, np.int32)
+    okv = OF.KVCache(cfg, 1, CTX + K + 2)
+    for l in range(cfg["n_layers"]):
+        okv.k[l, 0, :CTX] = kv_rows[l][0].view(CTX, cfg["n_kv_heads"], cfg["head_dim"])
+        okv.v[l, 0, :CTX] = kv_rows[l][1].view(CTX, cfg["n_kv_heads"], cfg["head_dim"])
+    okv.ctx[0] = CTX
+    logits = OF.forward(W_cpu, cfg, okv, [0], [rows])[0]
+    a, em = OA.accept_one(logits.float().numpy(), rows, len(rows), OA.STRICT, 2, 0.1)
+    return time.perf_counter() - t0, len(em), int(a)
 
 
-def cpu_baseline(wl, sample):
+SAMPLE = "1 of the 16 sequences of a step (sequence 0: draft in its group, all %d layers, acceptance), measured, nothing scaled"
+
+
+def cpu_baseline(wl):
+    """The oracle on the host cores, once, on sequence 0 of the same workload (same weights, cache,
+    pool and tail as the GPU arm)."""
     cfg = wl["cfg"]
     W = wl["W"]
     W_cpu = dict(tok_emb=W["tok_emb"].cpu(), lm_head=W["lm_head"].cpu(), final_norm=W["final_norm"].cpu(),
-                 layers=[{k: v.cpu() for k, v in lw.items()} for lw in W["layers"][:SAMPLE_LAYERS]])
+                 layers=[{k: v.cpu() for k, v in lw.items()} for lw in W["layers"]])
     width = cfg["n_kv_heads"] * cfg["head_dim"]
     kv_rows = [tuple(t.cpu() for t in synth.make_kv_layer(CTX, width, 7, l, device=str(W["tok_emb"].device)))
-               for l in range(SAMPLE_LAYERS)]
-    total, n_tok = oracle_sample(cfg, W_cpu, kv_rows, wl["pool"], wl["offs"], wl["tails"][0], int(wl["gid"][0]))[0]
-    return {"value": n_tok / total, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle",
-            "sample": sample, "seconds_extrapolated": total}
+               for l in range(cfg["n_layers"])]
+    sec, n_tok, _ = oracle_step(cfg, W_cpu, kv_rows, wl["pool"], wl["offs"], wl["tails"][0], int(wl["gid"][0]))
+    return {"value": n_tok / sec, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle",
+            "sample": SAMPLE % cfg["n_layers"], "seconds": sec, "tokens": n_tok}
 
 
 def run_reference(args):
-    """CPU oracle on a bounded sample of the same workload; rank 0 only."""
+    """The CPU oracle on the same workload recipe (5 M-token pool in 1000 groups, planted tail + drafts at
+    60 % agreement with the oracle's own greedy continuation, 512 cached tokens, all 32 layers), one
+    sequence per step; every step is really run and timed.  Rank 0 only."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    cfg = synth.model_cfg("7b")
-    cfg_s = dict(cfg, n_layers=SAMPLE_LAYERS)
-    W_cpu = synth.make_weights(cfg_s, seed=0, device="cpu")
+    from oracle import forward as OF
+    cfg = synth.model_cfg("7b", n_layers=args.layers)
+    W_cpu = synth.make_weights(cfg, seed=0, device="cpu")
     width = cfg["n_kv_heads"] * cfg["head_dim"]
-    kv_rows = [synth.make_kv_layer(CTX, width, 7, l) for l in range(SAMPLE_LAYERS)]
-    pool, offs = synth.make_zipf_pool(POOL_TOKENS // 10, POOL_GROUPS // 10, vocab=cfg["vocab"], seed=42)
+    kv_rows = [synth.make_kv_layer(CTX, width, 7, l) for l in range(cfg["n_layers"])]
     rng = np.random.default_rng(8)
-    st = int(offs[3]) + 100
-    tail = pool[st:st + N_MAX].copy()          # a tail that occurs in its group, so a draft is found
-    times = oracle_sample(cfg, W_cpu, kv_rows, pool, offs, tail, 3, repeat=args.warmup + args.steps)[args.warmup:]
-    total = sum(t for t, _ in times)
-    toks = sum(n for _, n in times)
+    last = int(rng.integers(0, cfg["vocab"], size=B)[0])
+    # greedy continuation and runner-up of sequence 0 by the oracle (set-up, not timed), then the drafts
+    okv = OF.KVCache(cfg, 1, CTX + K + 2)
+    for l in range(cfg["n_layers"]):
+        okv.k[l, 0, :CTX] = kv_rows[l][0].view(CTX, cfg["n_kv_heads"], cfg["head_dim"])
+        okv.v[l, 0, :CTX] = kv_rows[l][1].view(CTX, cfg["n_kv_heads"], cfg["head_dim"])
+    okv.ctx[0] = CTX
+    cur, greedy, second = last, [], []
+    for _ in range(K):
+        lg = OF.forward(W_cpu, cfg, okv, [0], [np.asarray([cur], np.int32)])[0][0]
+        top2 = torch.topk(lg, 2).indices
+        okv.ctx[0] += 1
+        cur = int(top2[0])
+        greedy.append(cur)
+        second.append(int(top2[1]))
+    drafts = synth.corrupt_drafts(np.asarray([greedy]), np.asarray([second]), cfg["vocab"], seed=8)[0]
+    pool, offs = synth.make_zipf_pool(POOL_TOKENS, POOL_GROUPS, vocab=cfg["vocab"], seed=42)
+    tail = np.concatenate([rng.integers(0, cfg["vocab"], size=(B, N_MAX - 1)).astype(np.int32)[0], [last]]).astype(np.int32)
+    doc = np.concatenate([[synth.SENTINEL], tail, drafts]).astype(np.int32)
+    pool = np.concatenate([pool[:offs[1]], doc, pool[offs[1]:]])         # sequence 0 belongs to group 0
+    offs = offs.copy()
+    offs[1:] += len(doc)
+    times = [oracle_step(cfg, W_cpu, kv_rows, pool, offs, tail, 0) for _ in range(args.warmup + args.steps)][args.warmup:]
+    total = sum(t for t, _, _ in times)
+    toks = sum(n for _, n, _ in times)
     value = toks / total
-    sample = ("per step: 1 of 16 sequences, %d of 32 layers run and time extrapolated to 32; pool %d tokens"
-              % (SAMPLE_LAYERS, len(pool)))
+    sample = "per step: " + SAMPLE % cfg["n_layers"]
     print(json.dumps({
         "impl": "reference", "metric": "generated_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "model_shape": "llama-2-7b", "batch": B, "ctx": CTX, "draft_len": K},
+        "config": {"workload": WORKLOAD, "model_shape": "llama-2-7b", "layers": args.layers, "batch": B, "ctx": CTX,
+                   "draft_len": K, "pool_tokens": int(len(pool)), "pool_groups": POOL_GROUPS, "suffix_n": [1, N_MAX],
+                   "max_occ": 64, "sample": sample},
+        "accepted_drafts_per_step": sum(a for _, _, a in times) / len(times),
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
@@ -469,10 +494,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=32,
                     help="decoder layers of the 7B shape (fewer only for small profiler captures; the line says so)")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle leg (profiler captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "RANK" not in os.environ:
+        # started plainly with --gpus N: become the launcher of N replicas, one process per GPU
+        from paper_2408_05676_b200 import replicas
+        sys.exit(replicas.launch_local([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], args.gpus))
     else:
         run_ours(args)
 

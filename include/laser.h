@@ -64,7 +64,8 @@ typedef struct {
   int32_t max_batch;   /* most sequences in one laser_verify_step call                     */
 } laser_model_cfg;
 
-/* bf16 device pointers, matrices row-major [out_features, in_features].  The per-layer
+/* bf16 device pointers, matrices row-major [out_features, in_features] and 16-byte aligned,
+ * norm gains 8-byte aligned (laser_model_create returns INVALID_ARG otherwise).  The per-layer
  * members are host arrays of n_layers device pointers. */
 typedef struct {
   const void* tok_emb;     /* [vocab, d_model]                                             */
@@ -239,8 +240,8 @@ laser_status laser_kv_export(const laser_kv* kv, int32_t seq, int32_t layer, int
  * committed length is not changed.  bf16 operands, fp32 accumulation and residual stream.
  *   seq_ids  dev int32[B] distinct cache slots;  tokens dev int32[B, K+1];
  *   n_rows   dev int32[B], 0..K+1 (0 = inactive);  logits dev fp32[B, K+1, vocab] out
- * with K = cfg.max_draft.  Rows >= n_rows[b] are left unspecified.
- * Errors: INVALID_ARG (B > max_batch), CAPACITY (a sequence would outgrow its pages: found
+ * with K = cfg.max_draft.  Rows >= n_rows[b] are left unspecified.  logits must be 16-byte aligned.
+ * Errors: INVALID_ARG (B > max_batch, misaligned logits), CAPACITY (a sequence would outgrow its pages: found
  * on the device, the rows are then not cached, and laser_check() reports it). */
 laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int32_t* seq_ids,
                                const int32_t* tokens, const int32_t* n_rows, int32_t B,
@@ -284,9 +285,8 @@ laser_status laser_accept_commit(laser_kv* kv, const int32_t* seq_ids, const flo
                                  int32_t V, const laser_params* p, int32_t* n_accept,
                                  int32_t* out_tokens, int32_t* n_out, void* stream);
 
-/* ---- Verification of a token tree (Section 3.4: "if a predecessor node is rejected, all of its
- * successor nodes will be skipped ... ultimately accepting the verified branch with the maximum
- * length") ---------------------------------------------------------------------------------------
+/* ---- Verification of a token tree (Section 3.4, tree verification: the children of a rejected
+ * node are not examined, and of all verified nodes the deepest one fixes the accepted path) ------
  * tokens / parents / n_rows as for laser_verify_step_tree, logits its result.  Node i is verified
  * when its parent is (row 0 always is) and tokens[b,i] passes p->mode on the row of its parent.
  * The verified node of greatest depth wins, the first in depth-first order among equals.
@@ -316,17 +316,33 @@ laser_status laser_kv_compact_path(laser_kv* kv, const int32_t* seq_ids, const i
  * in the middle of a step would also stall every stream of the device while the driver
  * serves it.  laser_accept_commit keeps its per-row verdicts in a lazily grown scratch
  * buffer; this variant keeps them in a fixed 132 KB array that is part of the library image
- * on every GPU that loads it, and calls no allocating routine at all.
+ * on every GPU that loads it, and itself calls no allocating routine.
  *   Limits: B <= 1024 sequences and B * (K+1) <= 16384 rows; larger calls return
  *   LASER_ERR_CAPACITY and launch nothing.
  *   The first call on each device looks up the array's device address (the device must be
- *   current); make that first call before starting any stream capture.
+ *   current).  With lazy module loading that look-up, or the first launch, is also when the
+ *   CUDA runtime loads this part of the library onto the device (the kernel image and the
+ *   132 KB array), which needs driver memory: make the first call at start-up, before the
+ *   host reserves the rest of HBM and before starting any stream capture.  Later calls touch
+ *   no allocator.  The look-up is serialised between host threads.
  *   All calls on a device share the one array: two calls whose kernels may overlap on the GPU
  *   (different streams) race on it and give undefined results.  Serialise them. */
 laser_status laser_accept_commit_noalloc(laser_kv* kv, const int32_t* seq_ids, const float* logits,
                                          const int32_t* tokens, const int32_t* n_rows, int32_t B,
                                          int32_t V, const laser_params* p, int32_t* n_accept,
                                          int32_t* out_tokens, int32_t* n_out, void* stream);
+
+/* Self-test of the library's failure path (the paper has no counterpart).  Every wait inside the
+ * TMA-fed kernels is bounded; when one runs out the kernel stops waiting, lets its copies in flight
+ * land, records LASER_ERR_TIMEOUT in the model's status word and returns, and the context stays
+ * usable.  This call runs that path on purpose without harming anything: one small kernel waits on
+ * a barrier nobody arrives on, for at most limit_cycles clock cycles (1e3 .. 2e9), while a second
+ * role of the same kernel drains one bulk copy.  Afterwards laser_check() returns
+ * LASER_ERR_TIMEOUT once (and clears it), and the model works as before.
+ *   report  dev int32[4] out: [0] the starved wait gave up, [1] the abort flag reached the
+ *           producer role, [2] the producer saw its copy land, [3] cycles the wait took.
+ * Asynchronous on `stream`.  Errors: INVALID_ARG. */
+laser_status laser_selftest_wait(laser_model* m, int64_t limit_cycles, int32_t* report, void* stream);
 
 /* ---- Generation loop (Section 2.1 / Section 3) ----------------------------------------
  * Prefills each prompt except its last token, then repeats draft -> verify -> accept ->

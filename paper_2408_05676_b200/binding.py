@@ -61,7 +61,7 @@ EXPORTS = ["laser_version", "laser_last_error", "laser_launch_count", "laser_poo
            "laser_kv_create", "laser_kv_free", "laser_kv_set_page_table", "laser_kv_set_len",
            "laser_kv_get_len", "laser_kv_set_len_dev", "laser_kv_import", "laser_kv_export",
            "laser_verify_step", "laser_verify_step_tree", "laser_check", "laser_profile_enable", "laser_profile_read", "laser_accept_commit", "laser_accept_commit_noalloc", "laser_accept_tree", "laser_kv_compact_path",
-           "laser_generate"]
+           "laser_selftest_wait", "laser_generate"]
 
 lib.laser_version.restype = C.c_char_p
 lib.laser_last_error.restype = C.c_char_p
@@ -353,6 +353,12 @@ def profile_read(model: Model, cls: int):
 
 def check(model: Model, stream=None) -> None:
     _chk(lib.laser_check(model.handle, _stream(stream)))
+
+
+def selftest_wait(model: Model, limit_cycles: int, stream=None) -> torch.Tensor:
+    report = torch.zeros(4, dtype=torch.int32, device="cuda")
+    _chk(lib.laser_selftest_wait(model.handle, C.c_int64(int(limit_cycles)), _ptr(report), _stream(stream)))
+    return report
 
 
 def accept_commit_noalloc(kv: Optional[KV], seq_ids, logits, tokens, n_rows, params: Params, out, stream=None):

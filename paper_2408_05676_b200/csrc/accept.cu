@@ -7,6 +7,8 @@
 // rule needs a probability, sums exp(l - max) in fp64.  The last CTA of a sequence to finish
 // walks the per-row verdicts in order and writes the outputs.  Reductions have a fixed
 // shape, so results are identical from run to run.
+#include <mutex>
+
 #include "state.cuh"
 
 namespace laser {
@@ -156,10 +158,13 @@ constexpr size_t kNoAllocCounterBytes = sizeof(int32_t) * kNoAllocMaxSeqs;
 constexpr size_t kNoAllocBytes = kNoAllocCounterBytes + sizeof(RowVerdict) * kNoAllocMaxRows;
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 
-// Device address of g_noalloc_scratch on the current device, resolved once per device.
+// Device address of g_noalloc_scratch on the current device, resolved once per device.  Host threads
+// may make their first calls at the same time: the table is guarded by a mutex.
 laser_status noalloc_scratch(void** out) {
   constexpr int kMaxDevices = 64;
   static void* addr[kMaxDevices] = {};
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
   int dev = 0;
   LASER_CUDA(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) { set_error("device index %d out of range", dev); return LASER_ERR_UNSUPPORTED; }

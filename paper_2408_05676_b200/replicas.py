@@ -4,8 +4,12 @@ around a timed region and the reduction of the per-rank figures: time = max over
 tokens = sum over ranks.  Works with any torch.distributed backend (nccl on GPUs, gloo on CPU)."""
 from __future__ import annotations
 
+import json
 import os
-from typing import Optional, Tuple
+import socket
+import subprocess
+import sys
+from typing import List, Optional, Sequence, Tuple
 
 import torch
 
@@ -52,3 +56,62 @@ def reduce_step(dist, ms: float, tokens: int, device: Optional[torch.device] = N
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     dist.all_reduce(n, op=dist.ReduceOp.SUM)
     return float(t[0]), int(n[0])
+
+
+def launch_local(cmd: Sequence[str], n: int, extra_env: Optional[dict] = None, timeout: Optional[float] = None) -> int:
+    """Starts `cmd` n times on this node, one process per rank (RANK = LOCAL_RANK = 0..n-1, WORLD_SIZE = n,
+    rendezvous on 127.0.0.1 at a free port), waits for all of them and returns the largest exit code.
+    The children inherit stdout/stderr, so whatever rank 0 prints is the job's output.  If one rank fails
+    the others are terminated (they would wait at the next barrier for ever)."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs: List[subprocess.Popen] = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), LOCAL_WORLD_SIZE=str(n),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        env.update(extra_env or {})
+        procs.append(subprocess.Popen(list(cmd), env=env))
+    rc = 0
+    pending = list(procs)
+    import time
+    t0 = time.time()
+    while pending:
+        for p in list(pending):
+            code = p.poll()
+            if code is None:
+                continue
+            pending.remove(p)
+            rc = max(rc, abs(code))
+            if code != 0:
+                for q in pending:
+                    q.terminate()
+        if timeout is not None and time.time() - t0 > timeout:
+            for q in pending:
+                q.terminate()
+            rc = max(rc, 124)
+            timeout = None
+        time.sleep(0.05)
+    return rc
+
+
+def _stub_workload() -> None:
+    """Stand-in workload for the launcher's CPU test: every rank joins (gloo), takes its block of 10 groups,
+    "times" a step, and rank 0 prints the reduced figures as one JSON line."""
+    dist, rank, world = init("gloo")
+    groups = list(shard_groups(10, rank, world))
+    barrier(dist)
+    ms, tokens = reduce_step(dist, 3.0 + rank, 10 * len(groups))
+    ranks = reduce_step(dist, 0.0, 1)[1]
+    if rank == 0:
+        print(json.dumps({"n_gpus": world, "ranks_seen": ranks, "ms": ms, "tokens": tokens, "groups_rank0": groups}))
+    barrier(dist)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    if "--stub-workload" in sys.argv:
+        if "--fail-rank" in sys.argv and os.environ.get("RANK") == sys.argv[sys.argv.index("--fail-rank") + 1]:
+            sys.exit(3)
+        _stub_workload()

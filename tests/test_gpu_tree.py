@@ -345,8 +345,11 @@ def test_13b_shape_17_rows_chain_and_tree(L):
         # at this width rounding the GEMM operands to bf16 alone moves the logits by more than 2e-2: the
         # yardstick is the fp64 oracle whose only change is that rounding (25 % slack for other rounding points)
         yard = O.forward(Wc, cfg, okv, seq_ids, rows, parents=pars if tree else None, mirror_bf16=True)
-        got = logits.cpu().double()
-        err = max(float((got[b, :n_rows[b]] - want[b]).abs().max()) for b in range(B))
-        yerr = max(float((yard[b] - want[b]).abs().max()) for b in range(B))
-        print("13B shape, tree" if tree else "13B shape, chain", "max-abs logit error", err, "bf16-operand oracle", yerr)
-        assert err <= 1.25 * yerr and err < 0.15
+        got = torch.cat([logits[b, :n_rows[b]].cpu().double() for b in range(B)])
+        want, yard = torch.cat(want), torch.cat(yard)
+        err, rms = float((got - want).abs().max()), float((got - want).pow(2).mean().sqrt())
+        yerr, yrms = float((yard - want).abs().max()), float((yard - want).pow(2).mean().sqrt())
+        agree = float((got.argmax(-1) == want.argmax(-1)).double().mean())
+        print("13B shape, tree" if tree else "13B shape, chain", "max-abs logit error %.4f rms %.5f" % (err, rms),
+              "| pinned bf16-operand yardstick %.4f rms %.5f" % (yerr, yrms), "| arg-max agreement %.3f over %d rows" % (agree, got.shape[0]))
+        assert err <= 1.25 * yerr and rms <= 1.25 * yrms and agree >= 0.8

@@ -49,3 +49,19 @@ def test_single_process_is_a_no_op():
     assert dist is None and (r, w) == (0, 1)
     assert replicas.reduce_step(None, 3.5, 9) == (3.5, 9)
     assert list(replicas.shard_groups(5, 0, 1)) == [0, 1, 2, 3, 4]
+
+
+def test_launcher_starts_n_ranks_and_reports_failures():
+    """The spawn path behind `bench.py --gpus N`: two ranks of a stub workload on CPU (gloo)."""
+    import json
+    import subprocess
+    code = ("import sys; sys.path.insert(0, %r); from paper_2408_05676_b200 import replicas; "
+            "sys.exit(replicas.launch_local([sys.executable, '-m', 'paper_2408_05676_b200.replicas', '--stub-workload'] + sys.argv[1:], 2, timeout=120))" % ROOT)
+    r = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, cwd=ROOT, timeout=180)
+    assert r.returncode == 0, r.stderr
+    line = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])
+    assert line["n_gpus"] == 2 and line["ranks_seen"] == 2 and line["ms"] == 4.0 and line["tokens"] == 100
+    assert line["groups_rank0"] == [0, 1, 2, 3, 4]
+    # a rank that exits with an error ends the job with a non-zero code instead of leaving the other waiting
+    r = subprocess.run([sys.executable, "-c", code, "--fail-rank", "1"], capture_output=True, text=True, cwd=ROOT, timeout=180)
+    assert r.returncode != 0

@@ -69,3 +69,36 @@ def test_sizes_beyond_the_fixed_array_are_refused(L):
         L.accept_commit_noalloc(None, None, torch.zeros(B, K + 1, V, device="cuda"),
                                 torch.zeros(B, K + 1, dtype=torch.int32, device="cuda"),
                                 torch.ones(B, dtype=torch.int32, device="cuda"), L.make_params(K=K), _outs(B, K + 1))
+
+
+def test_commit_and_exact_limits(L):
+    """With a cache handle the call also advances the committed lengths, exactly as the allocating call
+    does; and the two stated limits themselves (1024 sequences; 16384 rows) are accepted."""
+    cfg = synth.model_cfg("tiny")
+    from helpers import weights_to
+    m = L.model_create(cfg, weights_to(synth.make_weights(cfg, seed=0), "cuda"), max_batch=8)
+    kv = L.kv_create(m, 8, 8 * 8)
+    B, K, V = 8, 8, cfg["vocab"]
+    logits, tokens, n_rows = synth.make_accept_case(B, K, V, 31)
+    dl, dt, dn = torch.as_tensor(logits, device="cuda"), dev_i32(tokens), dev_i32(n_rows)
+    ids = torch.arange(B, dtype=torch.int32, device="cuda")
+    prm = L.make_params(K=K, mode=L.MODE_STRICT)
+    L.kv_set_len(kv, list(range(B)), [5] * B)
+    want = [t.cpu().numpy() for t in L.accept_commit(kv, ids, dl, dt, dn, prm)]
+    want_len = L.kv_get_len(kv, list(range(B)))
+    for call in range(2):
+        L.kv_set_len(kv, list(range(B)), [5] * B)
+        got = L.accept_commit_noalloc(kv, ids, dl, dt, dn, prm, _outs(B, K + 1))
+        torch.cuda.synchronize()
+        for g, w in zip(got, want):
+            assert (g.cpu().numpy() == w).all()
+        assert (L.kv_get_len(kv, list(range(B))) == want_len).all() and (want_len == 5 + want[2]).all()
+    for (B, K) in ((1024, 0), (1024, 15)):              # 1024 sequences; 1024 * 16 = 16384 rows
+        V = 64
+        logits, tokens, n_rows = synth.make_accept_case(B, K, V, 40 + K)
+        dl, dt, dn = torch.as_tensor(logits, device="cuda"), dev_i32(tokens), dev_i32(n_rows)
+        prm = L.make_params(K=K, mode=L.MODE_RELAXED, topk=2, p=0.05)
+        want = [t.cpu().numpy() for t in L.accept_commit(None, None, dl, dt, dn, prm)]
+        got = L.accept_commit_noalloc(None, None, dl, dt, dn, prm, _outs(B, K + 1))
+        for g, w in zip(got, want):
+            assert (g.cpu().numpy() == w).all()
