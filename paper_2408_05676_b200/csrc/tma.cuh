@@ -31,20 +31,25 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false when the limit ran out or another role of the CTA gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit_cycles = kWaitCycles) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
     for (int i = 0; i < 256; ++i)
       if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; return false; }
+    if (clock64() - t0 > limit_cycles) { *abort_flag = 1; return false; }
   }
 }
 // Drain helper for a producer that gave up: wait (bounded) for one copy still in flight.
-__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+// Returns whether the copy landed within the limit.
+__device__ __forceinline__ bool mbar_drain(uint32_t bar, uint32_t parity) {
   const long long t0 = clock64();
-  while (!mbar_try(bar, parity) && clock64() - t0 < kWaitCycles) {}
+  for (;;) {
+    if (mbar_try(bar, parity)) return true;
+    if (clock64() - t0 >= kWaitCycles) return false;
+  }
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
