@@ -38,11 +38,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
     hdrs = glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
     newest_hdr = max(os.path.getmtime(h) for h in hdrs)
     jobs, objs = [], []
+    extra = os.environ.get("LASER_NVCC_EXTRA", "").split()   # e.g. -DNAME for a diagnostic build
     for s in srcs:
         o = os.path.join(OBJ, os.path.basename(s)[:-3] + ".o")
         objs.append(o)
         if force or not os.path.exists(o) or os.path.getmtime(o) < max(os.path.getmtime(s), newest_hdr):
-            jobs.append([_nvcc(), *NVCC_FLAGS, "-c", s, "-o", o] + (["-Xptxas", "-v"] if verbose else []))
+            jobs.append([_nvcc(), *NVCC_FLAGS, *extra, "-c", s, "-o", o] + (["-Xptxas", "-v"] if verbose else []))
 
     def run(cmd):
         r = subprocess.run(cmd, capture_output=True, text=True)

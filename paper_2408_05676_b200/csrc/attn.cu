@@ -45,7 +45,7 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
                   const int32_t* __restrict__ seq_ids, const int32_t* __restrict__ row_ctx,
                   const int32_t* __restrict__ row_n, int Rs, int H, int Hkv,
                   const int32_t* __restrict__ page_table, int pages_per_seq, int layer_row0,
-                  bf16* __restrict__ out, int32_t* __restrict__ status, const void* next_w, size_t next_bytes,
+                  bf16* __restrict__ out, int32_t* __restrict__ status,
                   const unsigned long long* __restrict__ row_mask) {
   constexpr int HALVES = DH / 64;                 // 64-element (128-byte) column blocks per row
   constexpr int SUB = 16 * 128;                   // bytes of one 16-token x 64-element sub-tile
@@ -97,6 +97,7 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
       const int n_early = min(min(ctx >> 4, n_pg), kStages);   // whole pages of older tokens that fit the ring
       bool ok = true;
       int issued = 0;
+      const uint64_t kv_policy = make_policy_evict_first();   // a page is read once per step
       for (int p = 0; p < n_pg && ok; ++p) {
         const int s = p % kStages;
         if (p == n_early) asm volatile("griddepcontrol.wait;" ::: "memory");   // from here on: pages the kernel before may write
@@ -110,16 +111,13 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
         const int rowv = layer_row0 + ((phys * 2 + 1) * Hkv + hk) * 16;
 #pragma unroll
         for (int hf = 0; hf < HALVES; ++hf) {
-          tma_load_2d(dst + hf * SUB, &kvmap, hf * 64, rowk, bar);
-          tma_load_2d(dst + (HALVES + hf) * SUB, &kvmap, hf * 64, rowv, bar);
+          tma_load_2d_hint(dst + hf * SUB, &kvmap, hf * 64, rowk, bar, kv_policy);
+          tma_load_2d_hint(dst + (HALVES + hf) * SUB, &kvmap, hf * 64, rowv, bar, kv_policy);
         }
         issued = p + 1;
       }
       if (!ok)
         for (int p = max(0, issued - kStages); p < issued; ++p) mbar_drain(smem_u32(&full_bar[p % kStages]), (p / kStages) & 1);
-      // all pages requested: warm the L2 with the weights of the projection that follows
-      if (ok) prefetch_l2(next_w, next_bytes, blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z),
-                          gridDim.x * gridDim.y * gridDim.z);
     }
     return;
   }
@@ -279,7 +277,7 @@ bool attention_tma_supported(const laser_model* m, const laser_kv* kv) {
 }
 
 laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const int32_t* seq_ids, int B, bool tree,
-                                  const void* next_w, size_t next_bytes, cudaStream_t stream) {
+                                  cudaStream_t stream) {
   const int dh = m->cfg.head_dim, H = m->cfg.n_heads, Hkv = m->cfg.n_kv_heads, Rs = m->rows_per_seq;
   const int64_t rows_per_layer = int64_t(kv->n_pages) * 2 * Hkv * 16;
   const int layer_row0 = int(rows_per_layer * layer);
@@ -300,11 +298,11 @@ laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const
   if (dh == 128) {
     LASER_CUDA(cudaFuncSetAttribute(attn_paged_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     LASER_CUDA(cudaLaunchKernelEx(&cfg, attn_paged_kernel<128>, kv->pages_map, q, seq_ids, rc, rn, Rs, H, Hkv, pt,
-                                  kv->pages_per_seq, layer_row0, m->attn, m->status, next_w, next_bytes, mask));
+                                  kv->pages_per_seq, layer_row0, m->attn, m->status, mask));
   } else {
     LASER_CUDA(cudaFuncSetAttribute(attn_paged_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     LASER_CUDA(cudaLaunchKernelEx(&cfg, attn_paged_kernel<64>, kv->pages_map, q, seq_ids, rc, rn, Rs, H, Hkv, pt,
-                                  kv->pages_per_seq, layer_row0, m->attn, m->status, next_w, next_bytes, mask));
+                                  kv->pages_per_seq, layer_row0, m->attn, m->status, mask));
   }
   count_launch();
   LASER_CUDA(cudaGetLastError());

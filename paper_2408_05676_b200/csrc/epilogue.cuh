@@ -1,0 +1,128 @@
+// Fused epilogues of the dense contractions of the verify forward: what happens to a finished
+// 128-feature x token-row accumulator tile.  Shared by the per-matrix kernel and the persistent
+// whole-step kernel.  Values that another SM may have written during the running kernel (the
+// residual stream) are read past L1.
+#pragma once
+#include "model.cuh"
+
+namespace laser {
+
+using bf16 = __nv_bfloat16;
+constexpr int kBM = 128;          // weight rows per tile (MMA M)
+constexpr int kBK = 64;           // K elements per stage = one 128-byte swizzle span of bf16
+
+__device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  return make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+}
+
+// ---- fused epilogues: one warp finishes one token row r of a 128-feature tile; lane l holds
+//      features n0 + 4l .. 4l+3 in v.  What depends on the feature alone is worked out once per
+//      thread (LaneCtx); rows are finished without branches (`live` predicates the stores), so
+//      that the rows of a group interleave. ------------------------------------------------------
+struct LaneCtx {
+  int n;            // first of the lane's four features
+  bool in_range;    // n < N (N is a multiple of 8: then all four features are valid)
+  bool vec_out;     // EPI_PLAIN: the four results may be stored as one float4
+  // EPI_QKV
+  int kind;         // 0 = Q, 1 = K, 2 = V
+  int idx;          // offset of the feature inside its head
+  int shift;        // lanes between a feature and its rotation partner
+  float sg;         // sign of the partner's term
+  size_t kv_off;    // offset of (K or V, head, idx) inside a page
+  int rope_off;     // offset of the lane's first (cos, sin) pair inside a row of the table
+};
+
+template <int EPI>
+__device__ __forceinline__ LaneCtx make_lane_ctx(const GemmEpilogue& e, int n0, int lane, int N) {
+  LaneCtx c;
+  c.n = n0 + 4 * lane;
+  c.in_range = c.n < N;
+  c.vec_out = c.n + 3 < N && (e.ldo & 3) == 0;
+  c.kind = 0; c.idx = 0; c.shift = 0; c.sg = 0.f; c.kv_off = 0; c.rope_off = 0;
+  if (EPI == EPI_QKV) {
+    const int dh = e.dh, half = dh >> 1, dq = e.H * dh, dkv = e.Hkv * dh;
+    c.shift = dh >> 3;
+    c.kind = c.n < dq ? 0 : (c.n < dq + dkv ? 1 : 2);
+    c.idx = c.n % dh;          // four consecutive features stay inside one half of one head
+    c.sg = c.idx < half ? -1.f : 1.f;
+    c.rope_off = (c.idx % half) * 2;
+    if (c.kind) {
+      const int h = (c.n - dq - (c.kind - 1) * dkv) / dh;
+      c.kv_off = (size_t(c.kind - 1) * e.Hkv + h) * 16 * dh + c.idx;
+    }
+  }
+  return c;
+}
+
+__device__ __forceinline__ void epi_plain(const GemmEpilogue& e, const LaneCtx& c, int r, bool live, float4 v, float rstd, int N) {
+  if (!live || r >= e.R_store) return;
+  float* o = e.out + size_t(r) * e.ldo + c.n;
+  v.x *= rstd; v.y *= rstd; v.z *= rstd; v.w *= rstd;
+  if (c.vec_out) {
+    *reinterpret_cast<float4*>(o) = v;
+  } else {
+    if (c.n < N) o[0] = v.x;
+    if (c.n + 1 < N) o[1] = v.y;
+    if (c.n + 2 < N) o[2] = v.z;
+    if (c.n + 3 < N) o[3] = v.w;
+  }
+}
+
+// resid += acc; xb = bf16(resid * gain of the next norm); per-tile sum of squares for that norm
+__device__ __forceinline__ void epi_resid(const GemmEpilogue& e, const LaneCtx& c, int r, bool live, int lane, float4 v, int N,
+                                          int tile, float4 x, uint2 g2) {
+  float ss = 0.f;
+  x.x += v.x; x.y += v.y; x.z += v.z; x.w += v.w;
+  if (live && c.in_range) {
+    *reinterpret_cast<float4*>(e.resid + size_t(r) * N + c.n) = x;
+    const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&g2.x), g23 = *reinterpret_cast<const __nv_bfloat162*>(&g2.y);
+    *reinterpret_cast<uint2*>(e.xb + size_t(r) * N + c.n) =
+        pack4_bf16(x.x * __low2float(g01), x.y * __high2float(g01), x.z * __low2float(g23), x.w * __high2float(g23));
+    ss = x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+  }
+  for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if (live && lane == 0) e.sumsq_out[size_t(tile) * e.sumsq_ld + r] = ss;
+}
+
+// Tile rows 0..63 = gate features f0.., rows 64..127 = up features f0..: lanes 0-15 hold four
+// gate values each, lanes 16-31 the four up values of the same features.  Each pair of lanes
+// (l, l+16) trades two values, so that every lane finishes two features: act = silu(g) * u.
+__device__ __forceinline__ void epi_swiglu(const GemmEpilogue& e, int r, bool live, int f0, int lane, float4 v, float rstd) {
+  const bool lo = lane < 16;
+  const float t0 = __shfl_xor_sync(0xffffffffu, lo ? v.z : v.x, 16);
+  const float t1 = __shfl_xor_sync(0xffffffffu, lo ? v.w : v.y, 16);
+  const float g0 = (lo ? v.x : t0) * rstd, g1 = (lo ? v.y : t1) * rstd;
+  const float u0 = (lo ? t0 : v.z) * rstd, u1 = (lo ? t1 : v.w) * rstd;
+  const int fidx = f0 + 4 * (lane & 15) + (lo ? 0 : 2);
+  if (live && fidx < e.f) {  // f is a multiple of 8 (checked on the host)
+    const __nv_bfloat162 a = __floats2bfloat162_rn(__fdividef(g0, 1.f + __expf(-g0)) * u0, __fdividef(g1, 1.f + __expf(-g1)) * u1);
+    *reinterpret_cast<__nv_bfloat162*>(e.act + size_t(r) * e.f + fidx) = a;
+  }
+}
+
+// rotary embedding of Q and K (pair i, i + dh/2), bf16 rounding, Q store, K/V page write
+__device__ __forceinline__ void epi_qkv(const GemmEpilogue& e, const LaneCtx& c, int r, bool live, float4 v, float rstd,
+                                        int pos, int page, float4 cs01, float4 cs23) {
+  v.x *= rstd; v.y *= rstd; v.z *= rstd; v.w *= rstd;
+  float4 pv;
+  pv.x = __shfl_xor_sync(0xffffffffu, v.x, c.shift); pv.y = __shfl_xor_sync(0xffffffffu, v.y, c.shift);
+  pv.z = __shfl_xor_sync(0xffffffffu, v.z, c.shift); pv.w = __shfl_xor_sync(0xffffffffu, v.w, c.shift);
+  float4 y = v;
+  if (c.kind < 2) {
+    y.x = v.x * cs01.x + c.sg * pv.x * cs01.y;
+    y.y = v.y * cs01.z + c.sg * pv.y * cs01.w;
+    y.z = v.z * cs23.x + c.sg * pv.z * cs23.y;
+    y.w = v.w * cs23.z + c.sg * pv.w * cs23.w;
+  }
+  if (!live || !c.in_range) return;
+  if (c.kind == 0) {
+    if (pos < 0) y = make_float4(0.f, 0.f, 0.f, 0.f);
+    *reinterpret_cast<uint2*>(e.q + size_t(r) * (e.H * e.dh) + c.n) = pack4_bf16(y.x, y.y, y.z, y.w);
+  } else if (pos >= 0) {
+    bf16* dst = e.pages_layer + size_t(page) * e.page_elems + c.kv_off + size_t(pos & 15) * e.dh;
+    *reinterpret_cast<uint2*>(dst) = pack4_bf16(y.x, y.y, y.z, y.w);
+  }
+}
+
+}  // namespace laser

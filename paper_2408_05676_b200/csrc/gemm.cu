@@ -26,39 +26,18 @@
 #include <tuple>
 #include <type_traits>
 
-#include "model.cuh"
+#include "epilogue.cuh"
 #include "tma.cuh"
+#include "umma.cuh"
 
 namespace laser {
 namespace {
 
-using bf16 = __nv_bfloat16;
 constexpr int kTcThreads = 192;
-constexpr int kBM = 128;          // weight rows per tile (MMA M)
-constexpr int kBK = 64;           // K elements per stage = one 128-byte swizzle span of bf16
 constexpr int kMaxStages = 6;
 constexpr int kMaxNT = 192;       // token rows per tile: accumulator staging must fit shared memory
 constexpr int kSmemBudget = 110 * 1024;  // shared memory of one CTA: two CTAs per SM
 
-// Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows 128 B apart, groups
-// of 8 rows 1024 B apart.
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
-  uint64_t d = 0;
-  d |= uint64_t((smem_addr & 0x3FFFF) >> 4);        // start address
-  d |= uint64_t(1024 >> 4) << 32;                   // stride byte offset between 8-row groups
-  d |= uint64_t(1) << 46;                           // descriptor version of this architecture
-  d |= uint64_t(2) << 61;                           // 128-byte swizzle
-  return d;
-}
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
@@ -67,39 +46,6 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t ra
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
   return remote;
 }
-__device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v) {
-  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v));
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait on a barrier that peers of the cluster arrive on.
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_cluster(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_cluster(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; return false; }
-  }
-}
-// 16 consecutive fp32 columns of this thread's TMEM lane (no wait: pair with tmem_ld_wait)
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ float4 ld_cluster_f4(uint32_t cluster_addr) {
   float4 v;
   asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr));
@@ -108,129 +54,6 @@ __device__ __forceinline__ float4 ld_cluster_f4(uint32_t cluster_addr) {
 __device__ __forceinline__ void st_shared_f32(uint32_t addr, float v) {
   asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v));
 }
-// AND of a flag over the 128 epilogue threads (named barrier 1), so that they leave a loop together.
-__device__ __forceinline__ bool epilogue_all(bool ok) {
-  uint32_t r;
-  asm volatile(
-      "{\n.reg .pred p, q;\nsetp.ne.u32 q, %1, 0;\nbar.red.and.pred p, 1, 128, q;\nselp.u32 %0, 1, 0, p;\n}"
-      : "=r"(r) : "r"(uint32_t(ok)) : "memory");
-  return r != 0;
-}
-__device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
-  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
-  return make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
-}
-
-// ---- fused epilogues: one warp finishes one token row r of a 128-feature tile; lane l holds
-//      features n0 + 4l .. 4l+3 in v.  What depends on the feature alone is worked out once per
-//      thread (LaneCtx); rows are finished without branches (`live` predicates the stores), so
-//      that the rows of a group interleave. ------------------------------------------------------
-struct LaneCtx {
-  int n;            // first of the lane's four features
-  bool in_range;    // n < N (N is a multiple of 8: then all four features are valid)
-  bool vec_out;     // EPI_PLAIN: the four results may be stored as one float4
-  // EPI_QKV
-  int kind;         // 0 = Q, 1 = K, 2 = V
-  int idx;          // offset of the feature inside its head
-  int shift;        // lanes between a feature and its rotation partner
-  float sg;         // sign of the partner's term
-  size_t kv_off;    // offset of (K or V, head, idx) inside a page
-  int rope_off;     // offset of the lane's first (cos, sin) pair inside a row of the table
-};
-
-template <int EPI>
-__device__ __forceinline__ LaneCtx make_lane_ctx(const GemmEpilogue& e, int n0, int lane, int N) {
-  LaneCtx c;
-  c.n = n0 + 4 * lane;
-  c.in_range = c.n < N;
-  c.vec_out = c.n + 3 < N && (e.ldo & 3) == 0;
-  c.kind = 0; c.idx = 0; c.shift = 0; c.sg = 0.f; c.kv_off = 0; c.rope_off = 0;
-  if (EPI == EPI_QKV) {
-    const int dh = e.dh, half = dh >> 1, dq = e.H * dh, dkv = e.Hkv * dh;
-    c.shift = dh >> 3;
-    c.kind = c.n < dq ? 0 : (c.n < dq + dkv ? 1 : 2);
-    c.idx = c.n % dh;          // four consecutive features stay inside one half of one head
-    c.sg = c.idx < half ? -1.f : 1.f;
-    c.rope_off = (c.idx % half) * 2;
-    if (c.kind) {
-      const int h = (c.n - dq - (c.kind - 1) * dkv) / dh;
-      c.kv_off = (size_t(c.kind - 1) * e.Hkv + h) * 16 * dh + c.idx;
-    }
-  }
-  return c;
-}
-
-__device__ __forceinline__ void epi_plain(const GemmEpilogue& e, const LaneCtx& c, int r, bool live, float4 v, float rstd, int N) {
-  if (!live || r >= e.R_store) return;
-  float* o = e.out + size_t(r) * e.ldo + c.n;
-  v.x *= rstd; v.y *= rstd; v.z *= rstd; v.w *= rstd;
-  if (c.vec_out) {
-    *reinterpret_cast<float4*>(o) = v;
-  } else {
-    if (c.n < N) o[0] = v.x;
-    if (c.n + 1 < N) o[1] = v.y;
-    if (c.n + 2 < N) o[2] = v.z;
-    if (c.n + 3 < N) o[3] = v.w;
-  }
-}
-
-// resid += acc; xb = bf16(resid * gain of the next norm); per-tile sum of squares for that norm
-__device__ __forceinline__ void epi_resid(const GemmEpilogue& e, const LaneCtx& c, int r, bool live, int lane, float4 v, int N,
-                                          int tile, float4 x, uint2 g2) {
-  float ss = 0.f;
-  x.x += v.x; x.y += v.y; x.z += v.z; x.w += v.w;
-  if (live && c.in_range) {
-    *reinterpret_cast<float4*>(e.resid + size_t(r) * N + c.n) = x;
-    const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&g2.x), g23 = *reinterpret_cast<const __nv_bfloat162*>(&g2.y);
-    *reinterpret_cast<uint2*>(e.xb + size_t(r) * N + c.n) =
-        pack4_bf16(x.x * __low2float(g01), x.y * __high2float(g01), x.z * __low2float(g23), x.w * __high2float(g23));
-    ss = x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
-  }
-  for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-  if (live && lane == 0) e.sumsq_out[size_t(tile) * e.sumsq_ld + r] = ss;
-}
-
-// Tile rows 0..63 = gate features f0.., rows 64..127 = up features f0..: lanes 0-15 hold four
-// gate values each, lanes 16-31 the four up values of the same features.  Each pair of lanes
-// (l, l+16) trades two values, so that every lane finishes two features: act = silu(g) * u.
-__device__ __forceinline__ void epi_swiglu(const GemmEpilogue& e, int r, bool live, int f0, int lane, float4 v, float rstd) {
-  const bool lo = lane < 16;
-  const float t0 = __shfl_xor_sync(0xffffffffu, lo ? v.z : v.x, 16);
-  const float t1 = __shfl_xor_sync(0xffffffffu, lo ? v.w : v.y, 16);
-  const float g0 = (lo ? v.x : t0) * rstd, g1 = (lo ? v.y : t1) * rstd;
-  const float u0 = (lo ? t0 : v.z) * rstd, u1 = (lo ? t1 : v.w) * rstd;
-  const int fidx = f0 + 4 * (lane & 15) + (lo ? 0 : 2);
-  if (live && fidx < e.f) {  // f is a multiple of 8 (checked on the host)
-    const __nv_bfloat162 a = __floats2bfloat162_rn(__fdividef(g0, 1.f + __expf(-g0)) * u0, __fdividef(g1, 1.f + __expf(-g1)) * u1);
-    *reinterpret_cast<__nv_bfloat162*>(e.act + size_t(r) * e.f + fidx) = a;
-  }
-}
-
-// rotary embedding of Q and K (pair i, i + dh/2), bf16 rounding, Q store, K/V page write
-__device__ __forceinline__ void epi_qkv(const GemmEpilogue& e, const LaneCtx& c, int r, bool live, float4 v, float rstd,
-                                        int pos, int page, float4 cs01, float4 cs23) {
-  v.x *= rstd; v.y *= rstd; v.z *= rstd; v.w *= rstd;
-  float4 pv;
-  pv.x = __shfl_xor_sync(0xffffffffu, v.x, c.shift); pv.y = __shfl_xor_sync(0xffffffffu, v.y, c.shift);
-  pv.z = __shfl_xor_sync(0xffffffffu, v.z, c.shift); pv.w = __shfl_xor_sync(0xffffffffu, v.w, c.shift);
-  float4 y = v;
-  if (c.kind < 2) {
-    y.x = v.x * cs01.x + c.sg * pv.x * cs01.y;
-    y.y = v.y * cs01.z + c.sg * pv.y * cs01.w;
-    y.z = v.z * cs23.x + c.sg * pv.z * cs23.y;
-    y.w = v.w * cs23.z + c.sg * pv.w * cs23.w;
-  }
-  if (!live || !c.in_range) return;
-  if (c.kind == 0) {
-    if (pos < 0) y = make_float4(0.f, 0.f, 0.f, 0.f);
-    *reinterpret_cast<uint2*>(e.q + size_t(r) * (e.H * e.dh) + c.n) = pack4_bf16(y.x, y.y, y.z, y.w);
-  } else if (pos >= 0) {
-    bf16* dst = e.pages_layer + size_t(page) * e.page_elems + c.kv_off + size_t(pos & 15) * e.dh;
-    *reinterpret_cast<uint2*>(dst) = pack4_bf16(y.x, y.y, y.z, y.w);
-  }
-}
-
-
 template <int EPI>
 __global__ void __launch_bounds__(kTcThreads, 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, const GemmEpilogue e,
@@ -292,17 +115,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   if (warp == 0) {
     if (lane == 0) {  // ---- TMA producer ----
       const uint32_t full0 = smem_u32(&full_bar[0]);
-      auto load = [&](uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) { tma_load_2d(dst, tm, x, y, bar); };
+      // weights are read once per step: they must not push the activations, the residual stream and the
+      // cache pages of this step out of L2; every CTA of the launch reads the activations
+      const uint64_t w_policy = make_policy_evict_first(), a_policy = make_policy_evict_last();
+      auto load = [&](uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar, uint64_t pol) { tma_load_2d_hint(dst, tm, x, y, bar, pol); };
       auto expect = [&](int s) { mbar_expect_tx(smem_u32(&full_bar[s]), stage_bytes); };
       auto load_w = [&](int kb) {
         const int s = kb % stages, k = (kb0 + kb) * kBK;
         const uint32_t dst = tiles + uint32_t(s) * stage_bytes, bar = full0 + uint32_t(s) * 8;
-        load(dst, &tmW, k, EPI == EPI_SWIGLU ? wtile * 64 : n0, bar);
-        load(dst + w_bytes / 2, &tmW, k, EPI == EPI_SWIGLU ? e.f + wtile * 64 : n0 + 64, bar);
+        load(dst, &tmW, k, EPI == EPI_SWIGLU ? wtile * 64 : n0, bar, w_policy);
+        load(dst + w_bytes / 2, &tmW, k, EPI == EPI_SWIGLU ? e.f + wtile * 64 : n0 + 64, bar, w_policy);
       };
       auto load_a = [&](int kb) {
         const int s = kb % stages;
-        load(tiles + uint32_t(s) * stage_bytes + w_bytes, &tmA, (kb0 + kb) * kBK, r0, full0 + uint32_t(s) * 8);
+        load(tiles + uint32_t(s) * stage_bytes + w_bytes, &tmA, (kb0 + kb) * kBK, r0, full0 + uint32_t(s) * 8, a_policy);
       };
       // The weights do not depend on the kernel before this one: fill the ring with weight
       // tiles first, and only then wait for the previous kernel's results (the activations).
@@ -392,12 +218,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   __syncthreads();
   if (splits > 1) cluster_sync_all();  // every partial tile of the cluster is staged
 
-  if (warp == 0 && lane == 0 && !abort_flag) {
-    // Warm the L2 with the head of the next kernel's weights while the epilogue runs.
-    const unsigned worker = blockIdx.x + gridDim.x * blockIdx.y, n_workers = gridDim.x * gridDim.y;
-    prefetch_l2(e.next_w, e.next_bytes, worker, n_workers);
-    prefetch_l2(e.next_w2, e.next_bytes2, worker, n_workers);
-  }
   __syncwarp();
   if ((EPI == EPI_SWIGLU || EPI == EPI_PLAIN) && splits == 1) {
     // part 3 without partial tiles to sum or operands to prefetch: all six warps finish rows,

@@ -15,7 +15,6 @@ namespace {
 
 using bf16 = __nv_bfloat16;
 
-constexpr size_t kL2PrefetchBytes = size_t(8) << 20;   // more than this slows the epilogues it overlaps by more than it saves
 
 // ---- row bookkeeping -------------------------------------------------------------------
 // One block per row: position, cache slot, capacity check, rotary angles (fp64 -> fp32).
@@ -226,20 +225,6 @@ laser_status fuse_rows(laser_model* m, const void* const* pieces, const size_t* 
   *out = buf;
   return LASER_OK;
 }
-
-// Brackets one launch with events when profiling is on.
-struct ProfScope {
-  laser_model* m; int cls; cudaStream_t st; bool on;
-  ProfScope(laser_model* m_, int cls_, cudaStream_t st_) : m(m_), cls(cls_), st(st_), on(m_->profile) { mark(); }
-  ~ProfScope() { mark(); }
-  void mark() {
-    if (!on) return;
-    auto& ev = m->prof_events[cls];
-    size_t& used = m->prof_used[cls];
-    if (used == ev.size()) { cudaEvent_t e; if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; } ev.push_back(e); }
-    cudaEventRecord(ev[used++], st);
-  }
-};
 
 }  // namespace
 }  // namespace laser
@@ -498,8 +483,6 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
     LASER_CUDA(cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(attn_smem)));
   }
   const int d_tiles = ceil_div(d, 128);
-  // bytes of a following weight matrix worth prefetching into L2 while a kernel drains
-  auto head_bytes = [](size_t bytes) { return std::min<size_t>(bytes, kL2PrefetchBytes) & ~size_t(16383); };
   GemmEpilogue base;
   base.R_rows = m->R_pad;
   base.sumsq_ld = m->R_pad;
@@ -520,7 +503,7 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
     {
       ProfScope ps(m, 1, stream);
       if (use_tma_attn) {
-        LASER_TRY(attention_tma_launch(m, kv, l, seq_ids, B, tree, m->wo[l], head_bytes(size_t(d) * m->dq * 2), stream));
+        LASER_TRY(attention_tma_launch(m, kv, l, seq_ids, B, tree, stream));
       } else {
         attention_kernel<<<dim3(B, H), 128, attn_smem, stream>>>(m->q, seq_ids, m->row_ctx, m->row_n, Rs, H, Hkv, dh,
                                                                 kv->page_table, kv->pages_per_seq, pages_l,
@@ -531,8 +514,6 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
     {  // output projection; residual add; operand and statistics of the FFN norm
       GemmEpilogue e = base;
       e.resid = m->resid; e.xb = m->xn; e.gain_next = m->ffn_norm[l]; e.sumsq_out = m->sumsq;
-      e.next_w = m->wgu[l]; e.next_bytes = head_bytes(size_t(f) * d * 2) / 2;          // gate rows
-      e.next_w2 = m->wgu[l] + size_t(f) * d; e.next_bytes2 = e.next_bytes;             // up rows
       ProfScope ps(m, 0, stream);
       LASER_TRY(gemm_fused(m, m->attn, m->wo[l], Rp, d, m->dq, EPI_RESID, e, stream));
     }
@@ -540,7 +521,6 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
       GemmEpilogue e = base;
       e.sumsq_in = m->sumsq; e.sumsq_in_tiles = d_tiles;
       e.act = m->act; e.f = f;
-      e.next_w = m->wdown[l]; e.next_bytes = head_bytes(size_t(d) * f * 2);
       ProfScope ps(m, 0, stream);
       LASER_TRY(gemm_fused(m, m->xn, m->wgu[l], Rp, 2 * f, d, EPI_SWIGLU, e, stream));
     }
@@ -548,8 +528,6 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
       GemmEpilogue e = base;
       e.resid = m->resid; e.xb = m->xn; e.sumsq_out = m->sumsq;
       e.gain_next = l + 1 < c.n_layers ? m->attn_norm[l + 1] : m->final_norm;
-      e.next_w = l + 1 < c.n_layers ? m->wqkv[l + 1] : m->lm_head;
-      e.next_bytes = head_bytes(l + 1 < c.n_layers ? size_t(m->dqkv) * d * 2 : size_t(c.vocab) * d * 2);
       ProfScope ps(m, 0, stream);
       LASER_TRY(gemm_fused(m, m->act, m->wdown[l], Rp, d, f, EPI_RESID, e, stream));
     }

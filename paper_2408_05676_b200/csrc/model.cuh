@@ -41,12 +41,6 @@ enum { EPI_PLAIN = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_QKV = 3 };
 
 struct GemmEpilogue {
   int R_rows = 0;                    // rows the activation / output buffers really have
-  // weights of the kernel that follows (head of the matrix, multiple of 16 KB): prefetched
-  // into L2 once this kernel has issued its own loads; null = nothing
-  const void* next_w = nullptr;
-  size_t next_bytes = 0;
-  const void* next_w2 = nullptr;     // second region (the up half of a gate/up matrix)
-  size_t next_bytes2 = 0;
   // RMSNorm of the A operand, applied as a per-row scale of the result: the producer left
   // x * gain in bf16 and one sum of squares per (128-feature tile, row); null = no scale
   const float* sumsq_in = nullptr;
@@ -81,10 +75,25 @@ laser_status gemm_fused(laser_model* m, const __nv_bfloat16* A, const __nv_bfloa
                         const GemmEpilogue& e, cudaStream_t stream);
 void gemm_state_free(laser_model* m);
 
+// Brackets one launch with events when profiling is on.
+struct ProfScope {
+  laser_model* m; int cls; cudaStream_t st; bool on;
+  ProfScope(laser_model* m_, int cls_, cudaStream_t st_) : m(m_), cls(cls_), st(st_), on(m_->profile) { mark(); }
+  ~ProfScope() { mark(); }
+  void mark() {
+    if (!on) return;
+    auto& ev = m->prof_events[cls];
+    size_t& used = m->prof_used[cls];
+    if (used == ev.size()) { cudaEvent_t e; if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; } ev.push_back(e); }
+    cudaEventRecord(ev[used++], st);
+  }
+};
+
+
 // TMA-fed paged attention (head_dim 64 or 128 and a cache small enough for 32-bit row
 // coordinates); the verify forward falls back to a plain kernel otherwise.
 bool attention_tma_supported(const laser_model* m, const laser_kv* kv);
 laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const int32_t* seq_ids, int B, bool tree,
-                                  const void* next_w, size_t next_bytes, cudaStream_t stream);
+                                  cudaStream_t stream);
 
 }  // namespace laser
