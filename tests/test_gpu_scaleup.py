@@ -1,0 +1,139 @@
+"""The scale-up configuration: 13B shape (40 layers, d 5120, 40 heads of 128, FFN 13824, vocab 32000), 128
+sequences with prompts of 512-2048 tokens, 256 new tokens, drafts of 16, 64 groups of 4 M pool tokens.
+
+The cache of 128 such sequences (0.82 MB per token) does not fit beside the weights and the pool index,
+so the sequences run in waves sized from the free memory.  Where the configuration leaves the pools'
+source open they are a Zipf/template stream (4 M tokens per group); each group also holds two corrupted
+copies of what its test prompts generate (about 65 k generated tokens in all), so that drafts are found
+and are sometimes wrong.  Checked: strict speculative text == the library's plain greedy text (the
+lossless property, Section 2.1); acceptance and commit bit-exact against the oracle's rule on the
+library's logits of a full-depth step; drafts bit-exact against the oracle's scan on sampled queries.
+Logits of this layer shape are compared with the fp64 oracle at reduced depth in test_gpu_tree.py.
+Printed: tokens/s, accepted drafts per step, verify-step time and its share of the tensor roofline (with
+1088 rows per step the contractions are bound by the tensor cores, not by HBM)."""
+import json
+import os
+import time
+
+import numpy as np
+import pytest
+import torch
+
+from helpers import dev_i32, ensure_built
+from oracle import accept as A
+from oracle import retrieval as R
+from paper_2408_05676_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def L():
+    ensure_built()
+    from paper_2408_05676_b200 import binding
+    return binding
+
+
+def _peak_tflops():
+    try:
+        with open(os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured, sustained"
+    except (OSError, KeyError, ValueError):
+        return 1400.0, "fallback"
+
+
+def test_scale_up_13b_batch128(L):
+    B, K, NEW, G = 128, 16, 256, 64
+    pool_per_group = int(os.environ.get("LASER_C5_POOL_TOKENS", str(4_000_000)))
+    cfg = synth.model_cfg("13b", max_draft=K)
+    torch.cuda.empty_cache()
+    W = synth.make_weights(cfg, seed=0, device="cuda")
+    rng = np.random.default_rng(4000)
+    lens = rng.integers(512, 2049, size=B)
+    prompts = [synth.make_prompt(int(n), cfg["vocab"], 4000 + b) for b, n in enumerate(lens)]
+    gid = [b % G for b in range(B)]
+    # pools first (their index stays resident), then waves sized from what is left
+    t0 = time.time()
+    base, boffs = synth.make_zipf_pool(pool_per_group * G, G, vocab=cfg["vocab"], seed=46)
+    t_synth = time.time() - t0
+    pages = (2048 + NEW + K + 1 + 15) // 16 + 1
+    per_seq = pages * 16 * cfg["n_layers"] * 2 * cfg["n_kv_heads"] * cfg["head_dim"] * 2
+    index_bytes = int(170 * len(base))          # measured: about 160 bytes of index per pool token for n = 1..4
+    free, total = torch.cuda.mem_get_info()
+    wave_max = int(max(1, min(64, (free - index_bytes - (10 << 30)) // per_seq)))
+    wave = -(-B // -(-B // wave_max))           # waves of (nearly) equal size
+    model = L.model_create(cfg, W, max_batch=wave)
+    kv = L.kv_create(model, wave, wave * pages)
+    print("13B: %d sequences in waves of %d (cache %.1f GB per wave, weights 26 GB, %.0f M pool tokens, %.1f s to draw them)"
+          % (B, wave, wave * per_seq / 2 ** 30, len(base) / 1e6, t_synth))
+    # plain greedy text of every prompt (also the source of the generated part of the pools)
+    greedy, ms_greedy = [], 0.0
+    for w0 in range(0, B, wave):
+        r = L.generate(model, kv, None, prompts[w0:w0 + wave], [0] * len(prompts[w0:w0 + wave]), L.make_params(K=K, max_new=NEW))
+        greedy += r["out"]
+        ms_greedy += r["ms_total"] - r["ms_prefill"]
+    docs = [[] for _ in range(G)]
+    for b in range(B):
+        for rep in range(2):
+            d = list(greedy[b])
+            for i in range(3 + rep, len(d), 9 + 4 * rep):
+                d[i] = int(rng.integers(0, cfg["vocab"]))
+            docs[gid[b]].append(d)
+    parts, offs = [], [0]
+    for g in range(G):
+        seg = [base[boffs[g]:boffs[g + 1]]] + [np.asarray([synth.SENTINEL] + d, np.int32) for d in docs[g]]
+        seg = np.concatenate(seg)
+        parts.append(seg)
+        offs.append(offs[-1] + len(seg))
+    pool_np, offs = np.concatenate(parts), np.asarray(offs, np.int64)
+    del base, parts
+    t0 = time.time()
+    pool = L.pool_build(pool_np, offs, 1, 4)
+    torch.cuda.synchronize()
+    t_build = time.time() - t0
+    # strict speculative decoding, wave by wave
+    prm = L.make_params(K=K, n_min=1, n_max=4, max_occ=64, max_new=NEW)
+    tot = dict(steps=0, accepted=0, drafted=0, emitted=0, ms_decode=0.0, ms_prefill=0.0, ms_verify=0.0, verify_calls=0)
+    for w0 in range(0, B, wave):
+        ps, gs = prompts[w0:w0 + wave], gid[w0:w0 + wave]
+        r = L.generate(model, kv, pool, ps, gs, prm)
+        assert r["out"] == greedy[w0:w0 + wave]                       # lossless (same batch shape as the greedy run)
+        assert (L.kv_get_len(kv, list(range(len(ps)))) == lens[w0:w0 + wave] - 1 + NEW).all()
+        for k in ("steps", "accepted", "drafted", "emitted", "ms_prefill", "ms_verify", "verify_calls"):
+            tot[k] += r[k]
+        tot["ms_decode"] += r["ms_total"] - r["ms_prefill"]
+    assert tot["emitted"] == B * NEW
+    d, f, V, Lr = cfg["d_model"], cfg["d_ffn"], cfg["vocab"], cfg["n_layers"]
+    rows = wave * (K + 1)
+    flops = 2.0 * rows * (Lr * (4 * d * d + 3 * d * f) + d * V)
+    ms_step = tot["ms_verify"] / tot["verify_calls"]
+    peak, src = _peak_tflops()
+    print("speculative: decode %.0f tokens/s (greedy %.0f), accepted drafts/step %.2f, emitted/step %.2f, prefill %.0f tokens/s"
+          % (B * NEW / (tot["ms_decode"] * 1e-3), B * NEW / (ms_greedy * 1e-3), tot["accepted"] / tot["steps"],
+             tot["emitted"] / tot["steps"], float(lens.sum()) / (tot["ms_prefill"] * 1e-3)))
+    print("verify step of %d rows: %.2f ms, %.0f TFLOP/s in the contractions = %.2f of the bf16 tensor peak (%.0f TFLOP/s %s); "
+          "pool build %.1f s for %.0f M tokens" % (rows, ms_step, flops / ms_step * 1e-9, flops / ms_step * 1e-9 / peak, peak, src,
+                                                   t_build, len(pool_np) / 1e6))
+    # one full-depth step by hand: acceptance and commit against the oracle's rule on the library's logits
+    n = min(wave, 16)
+    ids = torch.arange(n, dtype=torch.int32, device="cuda")
+    hist = [np.concatenate([prompts[b], np.asarray(greedy[b][:40], np.int32)]) for b in range(n)]
+    L.generate(model, kv, None, hist, [0] * n, L.make_params(K=K, max_new=1))
+    L.kv_set_len(kv, list(range(n)), [len(h) - 1 for h in hist])
+    tails = np.asarray([h[-4:] for h in hist], np.int32)
+    dr, dl, _ = L.draft(pool, dev_i32(tails), dev_i32([4] * n), dev_i32(gid[:n]), prm)
+    for b in range(0, n, 5):                                            # drafts against the oracle's scan
+        want, _ = R.draft_one(pool_np, int(offs[gid[b]]), int(offs[gid[b] + 1]), tails[b], K, 1, 4, 1, 64)
+        assert int(dl[b]) == len(want) and dr[b, :len(want)].cpu().tolist() == want
+    tk, nr = L.make_rows(dev_i32([h[-1] for h in hist]), dr, dl, K)
+    logits = L.verify_step(model, kv, ids, tk, nr)
+    L.check(model)
+    lg, tkn, nrn = logits.cpu().numpy(), tk.cpu().numpy(), nr.cpu().numpy()
+    for mode, k, p in ((L.MODE_STRICT, 1, 0.0), (L.MODE_RELAXED, 2, 1e-3)):
+        L.kv_set_len(kv, list(range(n)), [len(h) - 1 for h in hist])
+        got = L.accept_commit(kv, ids, logits, tk, nr, L.make_params(K=K, mode=mode, topk=k, p=p))
+        ref = A.accept_batch(lg, tkn, nrn, mode, k, float(np.float32(p)))
+        for g_, w_ in zip(got, ref):
+            assert (g_.cpu().numpy() == w_).all()
+        assert (L.kv_get_len(kv, list(range(n))) == np.asarray([len(h) - 1 for h in hist]) + ref[2]).all()
+    assert tot["steps"] < B * NEW // 2
