@@ -48,7 +48,10 @@ enum {
   LASER_MODE_STRICT = 0,   /* Eq. 4: draft == arg max q_i                                  */
   LASER_MODE_RELAXED = 1,  /* Eq. 8: draft in TopK(q_i, k) and q_i(draft) > p              */
   LASER_MODE_TOPK = 2,     /* Eq. 7 alone                                                  */
-  LASER_MODE_TOPP = 3      /* draft == arg max q_i, or q_i(draft) > p                      */
+  LASER_MODE_TOPP = 3,     /* draft == arg max q_i, or q_i(draft) > p                      */
+  LASER_MODE_RELAXED_ARGMAX = 4  /* draft == arg max q_i, or Eq. 8: Eq. 8 with the arg-max always
+                              accepted ("highest probability or", Section 4.3.2); accepts whatever
+                              STRICT or RELAXED accepts                                    */
 };
 
 typedef struct laser_pool laser_pool;
@@ -343,6 +346,20 @@ laser_status laser_accept_commit_noalloc(laser_kv* kv, const int32_t* seq_ids, c
  *           producer role, [2] the producer saw its copy land, [3] cycles the wait took.
  * Asynchronous on `stream`.  Errors: INVALID_ARG. */
 laser_status laser_selftest_wait(laser_model* m, int64_t limit_cycles, int32_t* report, void* stream);
+
+/* ---- Grouping (Section 3.2, Collaborative-based Grouping) ------------------------------
+ * K-means over embeddings (Lloyd's iteration): the clustering by which the paper assigns users
+ * and items to the groups that each own a retrieval pool.  `iters` times: every point goes to its
+ * nearest centroid (squared Euclidean distance in fp32, ties to the smaller index), then every
+ * centroid becomes the mean of its points (a cluster without points keeps its centroid).
+ *   x dev fp32 [n, dim] row-major (dim <= 256); centroids dev fp32 [k, dim]: in = the starting
+ *   centroids, out = the final ones; assign dev int32[n] out: the assignment of the last
+ *   iteration (the group id of each point); counts dev int32[k] out: points per cluster in it.
+ * Assignments are identical from run to run for given centroids; the means are summed with
+ * atomics, so centroids agree between runs to fp32 summation accuracy.  Asynchronous on `stream`.
+ * Errors: INVALID_ARG (null pointer, sizes out of range, k * dim beyond shared memory), OOM. */
+laser_status laser_group_kmeans(const float* x, int64_t n, int32_t dim, int32_t k, int32_t iters,
+                                float* centroids, int32_t* assign, int32_t* counts, void* stream);
 
 /* ---- Generation loop (Section 2.1 / Section 3) ----------------------------------------
  * Prefills each prompt except its last token, then repeats draft -> verify -> accept ->

@@ -12,6 +12,9 @@ Modes
   RELAXED (1)  x_i in TopK(q_i, k)  and  q_i(x_i) > p              (Eq. 8)
   TOPK    (2)  x_i in TopK(q_i, k)                                 (Eq. 7)
   TOPP    (3)  x_i == argmax q_i  or  q_i(x_i) > p                 (Section 4.3.2, "top-p")
+  RELAXED_ARGMAX (4)  x_i == argmax q_i  or  Eq. 8                  (Eq. 8 read with the "highest probability
+               or" of Section 4.3.2: the arg-max is accepted whatever its probability, so this rule accepts
+               whatever STRICT or RELAXED accepts)
 
 Ties between equal logits rank the smaller token id first.  Probabilities are
 softmax at temperature 1, evaluated in fp64 from fp32 differences (l - max).
@@ -22,7 +25,7 @@ from typing import Tuple
 
 import numpy as np
 
-STRICT, RELAXED, TOPK, TOPP = 0, 1, 2, 3
+STRICT, RELAXED, TOPK, TOPP, RELAXED_ARGMAX = 0, 1, 2, 3, 4
 
 
 def argmax_row(row: np.ndarray) -> int:
@@ -51,6 +54,8 @@ def passes(row: np.ndarray, t: int, mode: int, k: int, p: float) -> bool:
         return rank_of(row, t) < k
     if mode == TOPP:
         return t == argmax_row(row) or prob_of(row, t) > p
+    if mode == RELAXED_ARGMAX:
+        return t == argmax_row(row) or (rank_of(row, t) < k and prob_of(row, t) > p)
     raise ValueError("mode")
 
 

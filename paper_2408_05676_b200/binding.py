@@ -20,7 +20,7 @@ if not os.path.exists(LIB_PATH):
 lib = C.CDLL(LIB_PATH)
 
 OK = 0
-MODE_STRICT, MODE_RELAXED, MODE_TOPK, MODE_TOPP = 0, 1, 2, 3
+MODE_STRICT, MODE_RELAXED, MODE_TOPK, MODE_TOPP, MODE_RELAXED_ARGMAX = 0, 1, 2, 3, 4
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "OOM", -3: "CUDA", -4: "CAPACITY", -5: "TIMEOUT", -6: "UNSUPPORTED"}
 
 
@@ -61,7 +61,7 @@ EXPORTS = ["laser_version", "laser_last_error", "laser_launch_count", "laser_poo
            "laser_kv_create", "laser_kv_free", "laser_kv_set_page_table", "laser_kv_set_len",
            "laser_kv_get_len", "laser_kv_set_len_dev", "laser_kv_import", "laser_kv_export",
            "laser_verify_step", "laser_verify_step_tree", "laser_check", "laser_profile_enable", "laser_profile_read", "laser_accept_commit", "laser_accept_commit_noalloc", "laser_accept_tree", "laser_kv_compact_path",
-           "laser_selftest_wait", "laser_generate"]
+           "laser_selftest_wait", "laser_group_kmeans", "laser_generate"]
 
 lib.laser_version.restype = C.c_char_p
 lib.laser_last_error.restype = C.c_char_p
@@ -414,6 +414,20 @@ def kv_compact_path(kv: KV, seq_ids, path_rows, n_accept, stream=None) -> None:
     _chk(lib.laser_kv_compact_path(kv.handle, _ptr(_dev(seq_ids, torch.int32)), _ptr(_dev(path_rows, torch.int32)),
                                    _ptr(_dev(n_accept, torch.int32)), C.c_int32(B), C.c_int32(path_rows.shape[1]),
                                    _stream(stream)))
+
+
+def group_kmeans(x: torch.Tensor, centroids: torch.Tensor, iters: int, stream=None):
+    """laser_group_kmeans: x fp32 [n, dim], centroids fp32 [k, dim] (updated in place).
+    Returns (assign int32[n], counts int32[k])."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous() and x.dim() == 2
+    assert centroids.is_cuda and centroids.dtype == torch.float32 and centroids.is_contiguous()
+    n, dim = x.shape
+    k = centroids.shape[0]
+    assign = torch.empty(n, dtype=torch.int32, device=x.device)
+    counts = torch.empty(k, dtype=torch.int32, device=x.device)
+    _chk(lib.laser_group_kmeans(_ptr(x), C.c_int64(n), C.c_int32(dim), C.c_int32(k), C.c_int32(iters),
+                                _ptr(centroids), _ptr(assign), _ptr(counts), _stream(stream)))
+    return assign, counts
 
 
 def generate(model: Model, kv: KV, pool: Optional[Pool], prompts: Sequence[np.ndarray], group_id: Sequence[int],

@@ -89,7 +89,7 @@ accept_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__
         pass = (t == arg);
       } else {
         const float lt = row[t];
-        const bool need_p = (mode == LASER_MODE_RELAXED || mode == LASER_MODE_TOPP);
+        const bool need_p = (mode == LASER_MODE_RELAXED || mode == LASER_MODE_TOPP || mode == LASER_MODE_RELAXED_ARGMAX);
         int ahead = 0;
         double sum = 0.0;
         auto visit = [&](float x, int j) {
@@ -117,6 +117,7 @@ accept_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__
           const bool above_p = need_p && (exp(double(lt - mx)) / sum > p);
           if (mode == LASER_MODE_RELAXED) pass = in_topk && above_p;
           else if (mode == LASER_MODE_TOPK) pass = in_topk;
+          else if (mode == LASER_MODE_RELAXED_ARGMAX) pass = (t == arg) || (in_topk && above_p);
           else pass = (t == arg) || above_p;
         }
       }
@@ -188,7 +189,7 @@ LASER_API laser_status laser_accept_commit_noalloc(laser_kv* kv, const int32_t* 
   using namespace laser;
   LASER_REQUIRE(p && logits && tokens && n_rows && n_accept && out_tokens && n_out, "null argument");
   LASER_REQUIRE(B >= 0 && V >= 1 && p->K >= 0, "B = %d, V = %d, K = %d", B, V, p->K);
-  LASER_REQUIRE(p->mode >= LASER_MODE_STRICT && p->mode <= LASER_MODE_TOPP, "mode = %d", p->mode);
+  LASER_REQUIRE(p->mode >= LASER_MODE_STRICT && p->mode <= LASER_MODE_RELAXED_ARGMAX, "mode = %d", p->mode);
   LASER_REQUIRE(p->mode == LASER_MODE_STRICT || p->mode == LASER_MODE_TOPP || p->topk >= 1, "topk = %d", p->topk);
   LASER_REQUIRE(kv == nullptr || seq_ids != nullptr, "seq_ids is required when committing");
   const int64_t rows = int64_t(B) * (int64_t(p->K) + 1);
@@ -223,7 +224,7 @@ LASER_API laser_status laser_accept_commit(laser_kv* kv, const int32_t* seq_ids,
   LASER_REQUIRE(B >= 0 && B <= kMaxAcceptSeqs, "B = %d outside [0, %d]", B, kMaxAcceptSeqs);
   LASER_REQUIRE(V >= 1, "V = %d", V);
   LASER_REQUIRE(p->K >= 0 && p->K <= 1023, "K = %d outside [0, 1023]", p->K);
-  LASER_REQUIRE(p->mode >= LASER_MODE_STRICT && p->mode <= LASER_MODE_TOPP, "mode = %d", p->mode);
+  LASER_REQUIRE(p->mode >= LASER_MODE_STRICT && p->mode <= LASER_MODE_RELAXED_ARGMAX, "mode = %d", p->mode);
   LASER_REQUIRE(p->mode == LASER_MODE_STRICT || p->mode == LASER_MODE_TOPP || p->topk >= 1,
                 "topk = %d", p->topk);
   LASER_REQUIRE(kv == nullptr || seq_ids != nullptr, "seq_ids is required when committing");

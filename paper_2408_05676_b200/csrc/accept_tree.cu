@@ -70,7 +70,7 @@ __device__ int cta_verdict(const float* __restrict__ row, int V, int t, float mx
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const bool vec = (V % 4 == 0) && ((reinterpret_cast<uintptr_t>(row) & 15) == 0);
   const float lt = row[t];
-  const bool need_p = (mode == LASER_MODE_RELAXED || mode == LASER_MODE_TOPP);
+  const bool need_p = (mode == LASER_MODE_RELAXED || mode == LASER_MODE_TOPP || mode == LASER_MODE_RELAXED_ARGMAX);
   int ahead = 0;
   double sum = 0.0;
   auto visit = [&](float x, int j) {
@@ -99,6 +99,7 @@ __device__ int cta_verdict(const float* __restrict__ row, int V, int t, float mx
     const bool above_p = need_p && (exp(double(lt - mx)) / sum > p);
     if (mode == LASER_MODE_RELAXED) pass = in_topk && above_p;
     else if (mode == LASER_MODE_TOPK) pass = in_topk;
+    else if (mode == LASER_MODE_RELAXED_ARGMAX) pass = (t == arg) || (in_topk && above_p);
     else pass = (t == arg) || above_p;
   }
   return pass;
@@ -238,7 +239,7 @@ LASER_API laser_status laser_accept_tree(laser_kv* kv, const int32_t* seq_ids, c
   LASER_REQUIRE(B >= 0 && B <= kMaxSeqs, "B = %d outside [0, %d]", B, kMaxSeqs);
   LASER_REQUIRE(V >= 1, "V = %d", V);
   LASER_REQUIRE(p->K >= 0 && p->K + 1 <= kMaxTreeRows, "a token tree has at most %d rows (K + 1 = %d)", kMaxTreeRows, p->K + 1);
-  LASER_REQUIRE(p->mode >= LASER_MODE_STRICT && p->mode <= LASER_MODE_TOPP, "mode = %d", p->mode);
+  LASER_REQUIRE(p->mode >= LASER_MODE_STRICT && p->mode <= LASER_MODE_RELAXED_ARGMAX, "mode = %d", p->mode);
   LASER_REQUIRE(p->mode == LASER_MODE_STRICT || p->mode == LASER_MODE_TOPP || p->topk >= 1, "topk = %d", p->topk);
   LASER_REQUIRE(kv == nullptr || seq_ids != nullptr, "seq_ids is required when committing");
   if (B == 0) return LASER_OK;

@@ -40,7 +40,7 @@ void set_error(const char* fmt, ...);
 // aligned, zero-filled when (re)allocated.  Grows by reallocation (synchronising the
 // device), so a pointer is only valid until the next call that asks for more.  Contents
 // persist between calls.
-enum { SCRATCH_ACCEPT = 0, SCRATCH_DRAFT = 1, SCRATCH_ACCEPT_TREE = 2, SCRATCH_SLOTS = 3 };
+enum { SCRATCH_ACCEPT = 0, SCRATCH_DRAFT = 1, SCRATCH_ACCEPT_TREE = 2, SCRATCH_GROUPING = 3, SCRATCH_SLOTS = 4 };
 laser_status scratch_get(int slot, size_t bytes, void** out);
 
 // Kernel launch counter (per process) for the statistics.

@@ -270,3 +270,16 @@ def make_accept_case(B: int, K: int, V: int, seed: int, tie_frac: float = 0.15
                 tokens[b, i] = order[2]
     n_rows = rng.integers(1, K + 2, size=B).astype(np.int32)
     return logits, tokens, n_rows
+
+
+def make_embeddings(n: int, dim: int, n_clusters: int, seed: int = 50, spread: float = 0.35
+                    ) -> Tuple[np.ndarray, np.ndarray]:
+    """Synthetic user / item embeddings for the grouping stand-in: a mixture of n_clusters Gaussians with
+    unit-scale centres and standard deviation `spread` per coordinate, cluster sizes log-normal.
+    Returns (fp32 [n, dim], the generating component int32[n])."""
+    rng = np.random.default_rng(seed)
+    centres = rng.standard_normal((n_clusters, dim))
+    w = rng.lognormal(0.0, 0.7, n_clusters)
+    comp = rng.choice(n_clusters, size=n, p=w / w.sum()).astype(np.int32)
+    x = centres[comp] + spread * rng.standard_normal((n, dim))
+    return x.astype(np.float32), comp

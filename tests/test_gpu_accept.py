@@ -31,7 +31,8 @@ def test_matches_oracle_all_modes(L, B, K, V, seed):
     n_rows[0] = 0 if B > 3 else n_rows[0]
     n_threshold_ties = 0
     for mode, k, p in [(A.STRICT, 1, 0.0), (A.RELAXED, 2, 0.1), (A.RELAXED, 3, 0.3), (A.RELAXED, 1, 0.0),
-                       (A.TOPK, 2, 0.0), (A.TOPP, 1, 0.1), (A.RELAXED, 2, 1.0)]:
+                       (A.TOPK, 2, 0.0), (A.TOPP, 1, 0.1), (A.RELAXED, 2, 1.0), (A.RELAXED_ARGMAX, 2, 0.1),
+                       (A.RELAXED_ARGMAX, 3, 0.3)]:
         got, p32 = _run(L, logits, tokens, n_rows, mode, k, p)
         want = A.accept_batch(logits, tokens, n_rows, mode, k, p32)
         for g, w, name in zip(got, want, ("n_accept", "out_tokens", "n_out")):

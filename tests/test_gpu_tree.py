@@ -110,7 +110,7 @@ def test_bad_parent_is_reported(L):
 
 
 @pytest.mark.parametrize("mode,topk,p", [(A.STRICT, 1, 0.0), (A.RELAXED, 2, 0.1), (A.RELAXED, 3, 0.02),
-                                         (A.TOPK, 2, 0.0), (A.TOPP, 1, 0.3)])
+                                         (A.TOPK, 2, 0.0), (A.TOPP, 1, 0.3), (A.RELAXED_ARGMAX, 2, 0.1)])
 def test_accept_tree_matches_oracle(L, mode, topk, p):
     """Bit-exact tree verification on synthesised logits that reach every branch of the rules (exact
     ties included): random trees whose tokens are the parent row's rank-1/2/3 or random tokens."""

@@ -8,7 +8,7 @@ from oracle import accept as A
 from paper_2408_05676_b200 import synth
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden", "accept_hand_examples.txt")
-MODES = dict(STRICT=A.STRICT, RELAXED=A.RELAXED, TOPK=A.TOPK, TOPP=A.TOPP)
+MODES = dict(STRICT=A.STRICT, RELAXED=A.RELAXED, TOPK=A.TOPK, TOPP=A.TOPP, RELAXED_ARGMAX=A.RELAXED_ARGMAX)
 
 
 def _cases():
@@ -67,7 +67,20 @@ def test_closed_forms():
     tp = A.accept_batch(logits, tokens, n_rows, A.TOPP, 2, 0.1)
     assert (tk[0] >= rv[0]).all() and (tp[0] >= s[0]).all()
     assert (rv[0] != s[0]).any() and (tk[0] != rv[0]).any()
-    for n_acc, out, n_out in (s, rv, tk, tp):
+    # RELAXED_ARGMAX passes a token exactly when STRICT or RELAXED does, row by row, so its prefix is at
+    # least as long as either; with k = 1 it is STRICT (the only top-1 token is the arg-max), and it is
+    # inside TOPP (arg-max or > p, without the top-k condition)
+    ra = A.accept_batch(logits, tokens, n_rows, A.RELAXED_ARGMAX, 2, 0.1)
+    assert (ra[0] >= np.maximum(s[0], rv[0])).all() and (ra[0] <= tp[0]).all()
+    for b in range(len(n_rows)):
+        for i in range(int(n_rows[b]) - 1):
+            t = int(tokens[b, i + 1])
+            assert A.passes(logits[b, i], t, A.RELAXED_ARGMAX, 2, 0.1) == (
+                A.passes(logits[b, i], t, A.STRICT, 2, 0.1) or A.passes(logits[b, i], t, A.RELAXED, 2, 0.1))
+    r1 = A.accept_batch(logits, tokens, n_rows, A.RELAXED_ARGMAX, 1, 0.1)
+    for x, y in zip(s, r1):
+        assert (x == y).all()
+    for n_acc, out, n_out in (s, rv, tk, tp, ra):
         assert (n_out == n_acc + 1).all() and (n_acc <= n_rows - 1).all()
         for b in range(len(n_rows)):
             a = n_acc[b]
