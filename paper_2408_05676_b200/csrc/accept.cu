@@ -10,18 +10,15 @@
 #include <mutex>
 
 #include "state.cuh"
+#include "verdict.cuh"
 
 namespace laser {
 namespace {
 
-constexpr int kAcceptThreads = 256;
+constexpr int kAcceptThreads = kVerdictThreads;
 constexpr int kMaxAcceptSeqs = 1 << 16;  // counters live at the start of the scratch
 
 struct RowVerdict { int32_t argmax; int32_t pass; };
-
-__device__ __forceinline__ void better(float& v, int& i, float ov, int oi) {
-  if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
-}
 
 __global__ void __launch_bounds__(kAcceptThreads)
 accept_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ tokens,
@@ -43,86 +40,13 @@ accept_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__
   if (i >= nr) return;
 
   const float* row = logits + (size_t(b) * R + i) * V;
-  const bool vec = (V % 4 == 0) && ((reinterpret_cast<uintptr_t>(row) & 15) == 0);
-  __shared__ float s_val[kAcceptThreads / 32];
-  __shared__ int s_idx[kAcceptThreads / 32];
-  __shared__ int s_cnt[kAcceptThreads / 32];
-  __shared__ double s_sum[kAcceptThreads / 32];
-  __shared__ float s_max;
-  __shared__ int s_arg;
-
-  // pass 1: max and arg max
-  float best = -INFINITY;
-  int besti = 0x7fffffff;
-  if (vec) {
-    const float4* r4 = reinterpret_cast<const float4*>(row);
-    for (int j = tid; j < V / 4; j += kAcceptThreads) {
-      float4 x = r4[j];
-      better(best, besti, x.x, 4 * j); better(best, besti, x.y, 4 * j + 1);
-      better(best, besti, x.z, 4 * j + 2); better(best, besti, x.w, 4 * j + 3);
-    }
-  } else {
-    for (int j = tid; j < V; j += kAcceptThreads) better(best, besti, row[j], j);
-  }
-  for (int o = 16; o; o >>= 1) {
-    float ov = __shfl_xor_sync(0xffffffffu, best, o);
-    int oi = __shfl_xor_sync(0xffffffffu, besti, o);
-    better(best, besti, ov, oi);
-  }
-  if (lane == 0) { s_val[warp] = best; s_idx[warp] = besti; }
-  __syncthreads();
-  if (tid == 0) {
-    for (int w = 1; w < kAcceptThreads / 32; ++w) better(best, besti, s_val[w], s_idx[w]);
-    s_max = best; s_arg = besti;
-  }
-  __syncthreads();
-  const float mx = s_max;
-  const int arg = s_arg;
-
-  // pass 2: verdict on the draft token verified by this row (if any); all branch
-  // conditions below are uniform across the CTA
+  // pass 1: max and arg max; pass 2 (the row is now in L1/L2): the verdict on the draft token this
+  // row verifies, if any.  The branch conditions are uniform across the CTA.
+  float mx;
+  int arg;
+  cta_argmax(row, V, &mx, &arg);
   int pass = 0;
-  if (i + 1 < nr) {
-    const int t = tokens[b * R + i + 1];
-    if (t >= 0 && t < V) {
-      if (mode == LASER_MODE_STRICT) {
-        pass = (t == arg);
-      } else {
-        const float lt = row[t];
-        const bool need_p = (mode == LASER_MODE_RELAXED || mode == LASER_MODE_TOPP || mode == LASER_MODE_RELAXED_ARGMAX);
-        int ahead = 0;
-        double sum = 0.0;
-        auto visit = [&](float x, int j) {
-          ahead += (x > lt) || (x == lt && j < t);
-          if (need_p) sum += exp(double(x - mx));
-        };
-        if (vec) {
-          const float4* r4 = reinterpret_cast<const float4*>(row);
-          for (int j = tid; j < V / 4; j += kAcceptThreads) {
-            float4 x = r4[j];
-            visit(x.x, 4 * j); visit(x.y, 4 * j + 1); visit(x.z, 4 * j + 2); visit(x.w, 4 * j + 3);
-          }
-        } else {
-          for (int j = tid; j < V; j += kAcceptThreads) visit(row[j], j);
-        }
-        for (int o = 16; o; o >>= 1) {
-          ahead += __shfl_xor_sync(0xffffffffu, ahead, o);
-          sum += __shfl_xor_sync(0xffffffffu, sum, o);
-        }
-        if (lane == 0) { s_cnt[warp] = ahead; s_sum[warp] = sum; }
-        __syncthreads();
-        if (tid == 0) {
-          for (int w = 1; w < kAcceptThreads / 32; ++w) { ahead += s_cnt[w]; sum += s_sum[w]; }
-          const bool in_topk = ahead < topk;
-          const bool above_p = need_p && (exp(double(lt - mx)) / sum > p);
-          if (mode == LASER_MODE_RELAXED) pass = in_topk && above_p;
-          else if (mode == LASER_MODE_TOPK) pass = in_topk;
-          else if (mode == LASER_MODE_RELAXED_ARGMAX) pass = (t == arg) || (in_topk && above_p);
-          else pass = (t == arg) || above_p;
-        }
-      }
-    }
-  }
+  if (i + 1 < nr) pass = cta_verdict(row, V, tokens[b * R + i + 1], mx, arg, mode, topk, p);
 
   // publish, then let the last CTA of this sequence scan the verdicts in order
   __shared__ int s_last;

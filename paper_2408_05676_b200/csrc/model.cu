@@ -273,6 +273,11 @@ LASER_API laser_status laser_model_create(const laser_model_cfg* cfg, const lase
   LASER_REQUIRE(cfg->page_size == 16, "page_size must be 16");
   LASER_REQUIRE(cfg->max_draft >= 0 && cfg->max_draft <= 63 && cfg->max_batch >= 1, "max_draft / max_batch");
   LASER_REQUIRE(w->tok_emb && w->lm_head && w->final_norm, "null weight");
+  // the epilogues read four norm gains at a time
+  LASER_REQUIRE((reinterpret_cast<uintptr_t>(w->final_norm) & 7) == 0, "final_norm must be 8-byte aligned");
+  for (int l = 0; l < cfg->n_layers; ++l)
+    LASER_REQUIRE(w->attn_norm[l] && w->ffn_norm[l] && (reinterpret_cast<uintptr_t>(w->attn_norm[l]) & 7) == 0 &&
+                  (reinterpret_cast<uintptr_t>(w->ffn_norm[l]) & 7) == 0, "norm gains of layer %d must be non-null and 8-byte aligned", l);
   laser_model* m = new laser_model();
   struct Guard { laser_model* p; ~Guard() { if (p) laser_model_free(p); } } guard{m};
   m->cfg = *cfg;
@@ -461,6 +466,8 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
   LASER_REQUIRE(B >= 1 && B <= m->cfg.max_batch, "B = %d outside [1, max_batch = %d]", B, m->cfg.max_batch);
   LASER_REQUIRE(kv->n_layers == m->cfg.n_layers && kv->n_kv_heads == m->cfg.n_kv_heads && kv->head_dim == m->cfg.head_dim,
                 "cache was created for another model shape");
+  // the LM head stores four logits at a time
+  LASER_REQUIRE((reinterpret_cast<uintptr_t>(logits) & 15) == 0, "logits must be 16-byte aligned");
   cudaStream_t stream = as_stream(stream_);
   const laser_model_cfg& c = m->cfg;
   const int Rs = m->rows_per_seq, R = B * Rs, Rp = ceil_div(R, 16) * 16;

@@ -228,28 +228,42 @@ draft_warp_kernel(PoolView pv, DraftArgs a) {
       const int64_t p1 = lane + 32 < n_occ ? int64_t(s_occ[warp][lane + 32]) : -1;
       bool al0 = p0 >= 0, al1 = p1 >= 0;
       int len = 0;
-      for (int j = 1; j <= a.K; ++j) {
-        const int32_t t0 = (al0 && p0 + j < hi) ? pv.tok[p0 + j] : -1;
-        const int32_t t1 = (al1 && p1 + j < hi) ? pv.tok[p1 + j] : -1;
-        al0 = t0 >= 0; al1 = t1 >= 0;
-        if (!__any_sync(0xffffffffu, al0 || al1)) break;
-        s_tok[warp][lane] = t0;
-        s_tok[warp][lane + 32] = t1;
-        __syncwarp();
-        uint32_t c0 = 0, c1 = 0;
-        for (int e = 0; e < n_occ; ++e) {
-          const int32_t x = s_tok[warp][e];
-          c0 += (x == t0); c1 += (x == t1);
+      bool go = true;
+      // The continuation of every occurrence is fetched eight depths at a time, all loads issued before
+      // the first vote: the walk then costs one memory round trip per eight tokens, not one per token.
+      for (int jb = 1; jb <= a.K && go; jb += 8) {
+        int32_t r0[8], r1[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int j = jb + u;
+          r0[u] = (al0 && j <= a.K && p0 + j < hi) ? pv.tok[p0 + j] : -1;
+          r1[u] = (al1 && j <= a.K && p1 + j < hi) ? pv.tok[p1 + j] : -1;
         }
-        unsigned long long cand = 0;
-        if (al0) cand = (uint64_t(c0) << 32) | uint32_t(0x7fffffff - t0);
-        if (al1) cand = max(cand, (unsigned long long)((uint64_t(c1) << 32) | uint32_t(0x7fffffff - t1)));
-        for (int o = 16; o; o >>= 1) cand = max(cand, __shfl_xor_sync(0xffffffffu, cand, o));
-        const int32_t pick = 0x7fffffff - int32_t(uint32_t(cand));
-        if (lane == 0) s_cur[warp][j - 1] = pick;
-        al0 = al0 && t0 == pick; al1 = al1 && t1 == pick;
-        len = j;
-        __syncwarp();
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int j = jb + u;
+          if (j > a.K) { go = false; break; }
+          const int32_t t0 = al0 ? r0[u] : -1, t1 = al1 ? r1[u] : -1;
+          al0 = t0 >= 0; al1 = t1 >= 0;
+          if (!__any_sync(0xffffffffu, al0 || al1)) { go = false; break; }
+          s_tok[warp][lane] = t0;
+          s_tok[warp][lane + 32] = t1;
+          __syncwarp();
+          uint32_t c0 = 0, c1 = 0;
+          for (int e = 0; e < n_occ; ++e) {
+            const int32_t x = s_tok[warp][e];
+            c0 += (x == t0); c1 += (x == t1);
+          }
+          unsigned long long cand = 0;
+          if (al0) cand = (uint64_t(c0) << 32) | uint32_t(0x7fffffff - t0);
+          if (al1) cand = max(cand, (unsigned long long)((uint64_t(c1) << 32) | uint32_t(0x7fffffff - t1)));
+          for (int o = 16; o; o >>= 1) cand = max(cand, __shfl_xor_sync(0xffffffffu, cand, o));
+          const int32_t pick = 0x7fffffff - int32_t(uint32_t(cand));
+          if (lane == 0) s_cur[warp][j - 1] = pick;
+          al0 = al0 && t0 == pick; al1 = al1 && t1 == pick;
+          len = j;
+          __syncwarp();
+        }
       }
       if (len > best_len) {
         for (int j = lane; j < len; j += 32) out[j] = s_cur[warp][j];
