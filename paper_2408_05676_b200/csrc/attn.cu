@@ -1,13 +1,14 @@
 // Causal attention of the verify forward (Eq. 3 / Eq. 6, chain form of the mask): the K+1
 // rows of a sequence against its paged bf16 KV cache, which already holds the rows' own K/V.
 //
-// One CTA per (sequence, head, 16-row tile).  A producer warp walks the sequence's page table
-// and streams each 16-token page of K and V through TMA (128-byte swizzle) into a ring of
-// shared-memory stages; four consumer warps take pages round-robin, compute S = Q K^T and
-// O += P V with warp-level MMA (the rows are 16 at most, far below a tensor-memory tile),
-// keep an online softmax with warp-shuffle row reductions, and merge their partial
-// (max, sum, O) through shared memory at the end.  A page is read from HBM exactly once and
-// used by exactly one warp.  Every mbarrier wait is bounded.
+// One CTA per (sequence, head, group of TPC 16-row tiles).  A producer warp walks the sequence's
+// page table and streams each 16-token page of K and V through TMA (128-byte swizzle) into a ring
+// of shared-memory stages; four consumer warps compute S = Q K^T and O += P V with warp-level MMA
+// (the rows are few, far below a tensor-memory tile), keep an online softmax with warp-shuffle row
+// reductions, and merge their partial (max, sum, O) through shared memory at the end.  With up to
+// 16 rows per sequence (TPC = 1) the four warps take pages round-robin; with more rows (K + 1 > 16
+// or a large token tree, TPC = 2) two warps serve each of two row tiles and both tiles use the same
+// staged page, so a page is still read from HBM once per 32 rows.  Every mbarrier wait is bounded.
 #include "model.cuh"
 #include "tma.cuh"
 
@@ -39,7 +40,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int DH>
+template <int DH, int TPC>
 __global__ void __launch_bounds__(kAttnThreads, kCtasPerSm)
 attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restrict__ q,
                   const int32_t* __restrict__ seq_ids, const int32_t* __restrict__ row_ctx,
@@ -65,13 +66,16 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
   const int hk = h / (H / Hkv);
   const int nr = row_n[b], ctx = row_ctx[b];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int row0 = mt * 16;
-  bf16* obase = out + (size_t(b) * Rs + row0) * H * DH + size_t(h) * DH;
-  if (row0 >= nr) {  // nothing active in this tile: zero its rows
+  constexpr int NPG = kConsumers / TPC;           // consumer warps that share a row tile (they split the pages)
+  const int cta_row0 = mt * 16 * TPC;              // first row of the CTA's tiles
+  const int tile = TPC == 1 ? 0 : (warp & (TPC - 1)), pgrp = TPC == 1 ? warp : (warp / TPC);
+  const int row0 = cta_row0 + tile * 16;           // first row of this warp's tile
+  bf16* obase = out + (size_t(b) * Rs + cta_row0) * H * DH + size_t(h) * DH;
+  if (cta_row0 >= nr) {  // nothing active in these tiles: zero their rows
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    for (int idx = tid; idx < 16 * DH; idx += kAttnThreads) {
+    for (int idx = tid; idx < 16 * TPC * DH; idx += kAttnThreads) {
       const int r = idx / DH, d = idx % DH;
-      if (row0 + r < Rs) obase[size_t(r) * H * DH + d] = __float2bfloat16(0.f);
+      if (cta_row0 + r < Rs) obase[size_t(r) * H * DH + d] = __float2bfloat16(0.f);
     }
     return;
   }
@@ -85,7 +89,7 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
 
   if (tid == 0) {
     abort_flag = 0;
-    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), TPC); }
     mbar_fence_init();
     tma_prefetch_map(&kvmap);
   }
@@ -124,11 +128,11 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
 
   // ---- consumers ----
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  // Q tile: rows of this sequence, zero beyond the active ones
-  for (int idx = tid; idx < 16 * (DH / 8); idx += kConsumers * 32) {
+  // Q tiles: rows of this sequence, zero beyond the active ones
+  for (int idx = tid; idx < 16 * TPC * (DH / 8); idx += kConsumers * 32) {
     const int r = idx / (DH / 8), c = idx % (DH / 8);
     uint4 v = make_uint4(0, 0, 0, 0);
-    if (row0 + r < nr) v = *reinterpret_cast<const uint4*>(q + (size_t(b) * Rs + row0 + r) * H * DH + size_t(h) * DH + c * 8);
+    if (cta_row0 + r < nr) v = *reinterpret_cast<const uint4*>(q + (size_t(b) * Rs + cta_row0 + r) * H * DH + size_t(h) * DH + c * 8);
     *reinterpret_cast<uint4*>(q_ptr + r * QLD + c * 8) = v;
   }
   asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -136,7 +140,7 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
   const float sl2 = rsqrtf(float(DH)) * 1.4426950408889634f;
   // Q fragments are re-read from shared memory for every page: keeping them in registers
   // would cost 32 registers per thread and one resident CTA per SM
-  const uint32_t q_frag = q_smem + uint32_t(((lane & 7) + ((lane >> 3) & 1) * 8) * QLD + (lane >> 4) * 8) * 2;
+  const uint32_t q_frag = q_smem + uint32_t((tile * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * QLD + (lane >> 4) * 8) * 2;
   float o[DH / 8][4];
 #pragma unroll
   for (int t = 0; t < DH / 8; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
@@ -147,7 +151,7 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
   const unsigned long long vis0 = row_mask ? row_mask[size_t(b) * Rs + min(row0 + g, nr - 1)] : 0ull;
   const unsigned long long vis1 = row_mask ? row_mask[size_t(b) * Rs + min(row0 + g + 8, nr - 1)] : 0ull;
 
-  for (int p = warp; p < n_pg; p += kConsumers) {
+  for (int p = pgrp; p < n_pg; p += NPG) {
     const int s = p % kStages;
     if (!mbar_wait(smem_u32(&full_bar[s]), (p / kStages) & 1, &abort_flag)) break;
     const uint32_t kbase = tiles + uint32_t(s) * STAGE, vbase = kbase + HALVES * SUB;
@@ -238,33 +242,37 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
   asm volatile("bar.sync 1, 128;" ::: "memory");
   // weight of each warp's partial result per row, normalisation included: e_w / sum_w e_w l_w
   if (tid < 16 * kConsumers) {
-    const int r = tid % 16, wsel = tid / 16;
+    const int r = tid % 16, wsel = tid / 16, tsel = TPC == 1 ? 0 : (wsel & (TPC - 1));
     float mt_ = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < kConsumers; ++w) mt_ = fmaxf(mt_, s_m[w][r]);
+    for (int w = 0; w < kConsumers; ++w)
+      if (TPC == 1 || (w & (TPC - 1)) == tsel) mt_ = fmaxf(mt_, s_m[w][r]);
     float den = 0.f, mine = 0.f;
 #pragma unroll
     for (int w = 0; w < kConsumers; ++w) {
+      if (TPC != 1 && (w & (TPC - 1)) != tsel) continue;
       const float e = s_m[w][r] == -INFINITY ? 0.f : exp2f((s_m[w][r] - mt_) * sl2);
       den += e * s_l[w][r];
       if (w == wsel) mine = e;
     }
-    const bool live = row0 + r < nr && den > 0.f && !abort_flag;
+    const bool live = cta_row0 + tsel * 16 + r < nr && den > 0.f && !abort_flag;
     s_wgt[wsel][r] = live ? mine / den : 0.f;
   }
   asm volatile("bar.sync 1, 128;" ::: "memory");
-  for (int idx = tid; idx < 16 * (DH / 4); idx += kConsumers * 32) {   // four features per thread
-    const int r = idx / (DH / 4), d = (idx % (DH / 4)) * 4;
-    if (row0 + r >= Rs) continue;
+  for (int idx = tid; idx < 16 * TPC * (DH / 4); idx += kConsumers * 32) {   // four features per thread
+    const int rr = idx / (DH / 4), d = (idx % (DH / 4)) * 4;      // rr: row within the CTA's tiles
+    const int tsel = rr / 16, r = rr % 16;
+    if (cta_row0 + rr >= Rs) continue;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int w = 0; w < kConsumers; ++w) {
+      if (TPC != 1 && (w & (TPC - 1)) != tsel) continue;
       const float e = s_wgt[w][r];
       const float4 x = *reinterpret_cast<const float4*>(s_o + (w * 16 + r) * DH + d);
       acc.x += e * x.x; acc.y += e * x.y; acc.z += e * x.z; acc.w += e * x.w;
     }
     const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
-    *reinterpret_cast<uint2*>(obase + size_t(r) * H * DH + d) =
+    *reinterpret_cast<uint2*>(obase + size_t(rr) * H * DH + d) =
         make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
   }
   if (tid == 0 && abort_flag) atomicCAS(status, 0, LASER_ERR_TIMEOUT);
@@ -281,9 +289,10 @@ laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const
   const int dh = m->cfg.head_dim, H = m->cfg.n_heads, Hkv = m->cfg.n_kv_heads, Rs = m->rows_per_seq;
   const int64_t rows_per_layer = int64_t(kv->n_pages) * 2 * Hkv * 16;
   const int layer_row0 = int(rows_per_layer * layer);
-  const size_t smem = 1024 + size_t(kStages) * (2 * (dh / 64) * 16 * 128) + size_t(16) * (dh + 8) * 2;
+  const int tiles = ceil_div(Rs, 16), tpc = tiles > 1 ? 2 : 1;   // row tiles of a sequence; tiles per CTA
+  const size_t smem = 1024 + size_t(kStages) * (2 * (dh / 64) * 16 * 128) + size_t(16) * tpc * (dh + 8) * 2;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(unsigned(B), unsigned(H), unsigned(ceil_div(Rs, 16)));
+  cfg.gridDim = dim3(unsigned(B), unsigned(H), unsigned(ceil_div(tiles, tpc)));
   cfg.blockDim = dim3(kAttnThreads, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
@@ -295,15 +304,17 @@ laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const
   const __nv_bfloat16* q = m->q;
   const int32_t *rc = m->row_ctx, *rn = m->row_n, *pt = kv->page_table;
   const unsigned long long* mask = tree ? m->row_mask : nullptr;
-  if (dh == 128) {
-    LASER_CUDA(cudaFuncSetAttribute(attn_paged_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-    LASER_CUDA(cudaLaunchKernelEx(&cfg, attn_paged_kernel<128>, kv->pages_map, q, seq_ids, rc, rn, Rs, H, Hkv, pt,
-                                  kv->pages_per_seq, layer_row0, m->attn, m->status, mask));
-  } else {
-    LASER_CUDA(cudaFuncSetAttribute(attn_paged_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-    LASER_CUDA(cudaLaunchKernelEx(&cfg, attn_paged_kernel<64>, kv->pages_map, q, seq_ids, rc, rn, Rs, H, Hkv, pt,
-                                  kv->pages_per_seq, layer_row0, m->attn, m->status, mask));
-  }
+#define LASER_ATTN_LAUNCH(DH_, TPC_)                                                                                     \
+  do {                                                                                                                   \
+    LASER_CUDA(cudaFuncSetAttribute(attn_paged_kernel<DH_, TPC_>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))); \
+    LASER_CUDA(cudaLaunchKernelEx(&cfg, attn_paged_kernel<DH_, TPC_>, kv->pages_map, q, seq_ids, rc, rn, Rs, H, Hkv, pt, \
+                                  kv->pages_per_seq, layer_row0, m->attn, m->status, mask));                              \
+  } while (0)
+  if (dh == 128 && tpc == 1) LASER_ATTN_LAUNCH(128, 1);
+  else if (dh == 128) LASER_ATTN_LAUNCH(128, 2);
+  else if (tpc == 1) LASER_ATTN_LAUNCH(64, 1);
+  else LASER_ATTN_LAUNCH(64, 2);
+#undef LASER_ATTN_LAUNCH
   count_launch();
   LASER_CUDA(cudaGetLastError());
   return LASER_OK;

@@ -111,8 +111,8 @@ def test_scale_up_13b_batch128(L):
     print("speculative: decode %.0f tokens/s (greedy %.0f), accepted drafts/step %.2f, emitted/step %.2f, prefill %.0f tokens/s"
           % (B * NEW / (tot["ms_decode"] * 1e-3), B * NEW / (ms_greedy * 1e-3), tot["accepted"] / tot["steps"],
              tot["emitted"] / tot["steps"], float(lens.sum()) / (tot["ms_prefill"] * 1e-3)))
-    print("verify step of %d rows: %.2f ms, %.0f TFLOP/s in the contractions = %.2f of the bf16 tensor peak (%.0f TFLOP/s %s); "
-          "pool build %.1f s for %.0f M tokens" % (rows, ms_step, flops / ms_step * 1e-9, flops / ms_step * 1e-9 / peak, peak, src,
+    print("verify step of %d rows: %.2f ms on average; the contractions' flops over the whole step (attention included) "
+          "%.0f TFLOP/s = %.2f of the bf16 tensor peak (%.0f TFLOP/s %s); pool build %.1f s for %.0f M tokens" % (rows, ms_step, flops / ms_step * 1e-9, flops / ms_step * 1e-9 / peak, peak, src,
                                                    t_build, len(pool_np) / 1e6))
     # one full-depth step by hand: acceptance and commit against the oracle's rule on the library's logits
     n = min(wave, 16)
@@ -128,6 +128,25 @@ def test_scale_up_13b_batch128(L):
     tk, nr = L.make_rows(dev_i32([h[-1] for h in hist]), dr, dl, K)
     logits = L.verify_step(model, kv, ids, tk, nr)
     L.check(model)
+    # where a step's time goes at this size: dense contractions against attention (event brackets per launch)
+    full_ids = torch.arange(wave, dtype=torch.int32, device="cuda")
+    full_tok = torch.randint(0, V, (wave, K + 1), dtype=torch.int32, device="cuda")
+    full_nr = torch.full((wave,), K + 1, dtype=torch.int32, device="cuda")
+    big = torch.empty(wave, K + 1, V, dtype=torch.float32, device="cuda")
+    ctx_w = [int(lens[b]) for b in range(wave)]
+    L.profile_enable(model, True)
+    for _ in range(2):
+        L.kv_set_len(kv, list(range(wave)), ctx_w)
+        L.verify_step(model, kv, full_ids, full_tok, full_nr, big)
+    gemm_ms, n_gemm = L.profile_read(model, 0)
+    attn_ms, _ = L.profile_read(model, 1)
+    L.profile_enable(model, False)
+    L.check(model)
+    kv_gb = sum(ctx_w) * Lr * 2 * cfg["n_kv_heads"] * cfg["head_dim"] * 2 / 1e9
+    print("one step of %d rows, launches bracketed by events: contractions %.2f ms = %.0f TFLOP/s = %.2f of the tensor peak; "
+          "attention %.2f ms for %.1f GB of cached K/V (%.0f GB/s)"
+          % (rows, gemm_ms / 2, flops / (gemm_ms / 2) * 1e-9, flops / (gemm_ms / 2) * 1e-9 / peak, attn_ms / 2, kv_gb,
+             kv_gb / (attn_ms / 2) * 1e3))
     lg, tkn, nrn = logits.cpu().numpy(), tk.cpu().numpy(), nr.cpu().numpy()
     for mode, k, p in ((L.MODE_STRICT, 1, 0.0), (L.MODE_RELAXED, 2, 1e-3)):
         L.kv_set_len(kv, list(range(n)), [len(h) - 1 for h in hist])
