@@ -33,7 +33,7 @@ WORKLOAD = "verify-step-7b: batch 16, ctx 512 (16-token pages), 1+8 rows/seq, dr
 B, K, CTX, N_MAX = 16, 8, 512, 4
 POOL_TOKENS, POOL_GROUPS = 5_000_000, 1000
 # read + write MB of the QKV, O, gate/up and down launches of a layer x 32 + the LM head, from the ncu capture
-GEMM_DRAM_TRAFFIC_PER_STEP = int((105.7 + 45.6 + 193.5 + 108.8) * 32e6 + 268.0e6)
+GEMM_DRAM_TRAFFIC_PER_STEP = int((105.3 + 37.2 + 187.1 + 99.8) * 32e6 + 269.1e6)
 
 
 def measured_peaks():
@@ -373,7 +373,7 @@ def run_ours(args):
         "roofline": {"kernel": "gemm_tc_kernel (all dense contractions of one verify step)", "bound": "hbm",
                      "achieved": gemm_gbs, "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
                      "frac": gemm_gbs / peaks["hbm_gbs"], "traffic": GEMM_DRAM_TRAFFIC_PER_STEP if args.layers == 32 else None,
-                     "traffic_note": "ncu dram read+write summed over the 129 launches of a step (per-launch figures in profiles/gemm_tc_kernel_7b_rows144.md, scaled from a 2-layer capture); includes up to 8 MB of next-kernel L2 prefetch per launch, counted twice under ncu's serialised replay",
+                     "traffic_note": "ncu dram read+write summed over the 129 launches of a step (per-launch figures in profiles/gemm_tc_kernel_7b_rows144.md, scaled from a 2-layer capture: per-launch traffic does not depend on the layer count)",
                      "algorithmic_bytes_per_step": ab["weights"], "ms_per_step": gemm_ms, "launches_per_step": gemm_n // args.steps},
         "tree_drafting": tree_res,
         "verify_step": {"ms": verify_ms, "algorithmic_bytes": ab["total"],
