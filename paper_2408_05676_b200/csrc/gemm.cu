@@ -324,11 +324,6 @@ laser_status tensor_map(GemmState* st, const void* ptr, int rows, int cols, int 
 }
 
 struct TcShape { int n_ttiles, NT, stages, tmem_cols; size_t smem; };
-}  // namespace
-// Tuning aids: non-zero values override the modelled split count / the stage count.
-int g_force_splits = 0;
-int g_force_stages = 0;
-namespace {
 
 TcShape tc_shape(int R_pad) {
   TcShape s;
@@ -336,7 +331,6 @@ TcShape tc_shape(int R_pad) {
   s.NT = ceil_div(ceil_div(R_pad, s.n_ttiles), 16) * 16;
   const int stage_bytes = kBM * 128 + s.NT * 128;
   s.stages = std::max(2, std::min(kMaxStages, kSmemBudget / stage_bytes));
-  if (g_force_stages) s.stages = std::max(2, std::min(s.stages, g_force_stages));
   s.tmem_cols = 32;
   while (s.tmem_cols < s.NT) s.tmem_cols <<= 1;
   s.smem = std::max(size_t(s.stages) * stage_bytes, size_t(s.NT) * kBM * 4) + 1024;
@@ -385,7 +379,7 @@ laser_status prepare(GemmState* st) {
 int pick_splits(int R_pad, int N, int K, int epi) {
   const int n_wtiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
   const int tiles = n_wtiles * tc_shape(R_pad).n_ttiles, total_kb = ceil_div(K, kBK);
-  int s = g_force_splits ? g_force_splits : int(208.0 / tiles + 0.5);
+  int s = int(208.0 / tiles + 0.5);
   s = std::max(1, std::min(s, std::min(total_kb, 8)));   // portable cluster size
   while (s > 1 && ceil_div(total_kb, s) * (s - 1) >= total_kb) --s;   // no rank without K blocks
   return s;
