@@ -257,6 +257,23 @@ def run_ours(args):
 
     res = {name: timed(prm, args.steps, args.warmup, sample_clocks=(name == "strict")) for name, prm in modes.items()}
     main = res["strict"]
+    step(strict)        # the rows of the headline step
+
+    def verify_alone():
+        """laser_verify_step alone, back to back on the step's rows (it leaves the committed lengths as
+        they are, so every call does the same work): one pair of events around all of them."""
+        L.kv_set_len_dev(kv, lens)
+        for _ in range(3):
+            L.verify_step(model, kv, seq_ids, tokens, n_rows, logits)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            L.verify_step(model, kv, seq_ids, tokens, n_rows, logits)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / args.steps
+
+    verify_ms = verify_alone()
 
     # tree-based drafting (Section 3.3) against chain drafting, both on the pool with three variants per
     # continuation: same verify forward (tree attention), tree verification, cache compaction
@@ -322,21 +339,6 @@ def run_ours(args):
         v_ms = sum(ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(args.steps)) / args.steps
         return v_ms, g_ms / args.steps, a_ms / args.steps, g_n
 
-    def verify_alone():
-        """laser_verify_step alone, back to back on the step's rows (it leaves the committed lengths as
-        they are, so every call does the same work): one pair of events around all of them."""
-        L.kv_set_len_dev(kv, lens)
-        for _ in range(3):
-            L.verify_step(model, kv, seq_ids, tokens, n_rows, logits)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(args.steps):
-            L.verify_step(model, kv, seq_ids, tokens, n_rows, logits)
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / args.steps
-
-    verify_ms = verify_alone()
     verify_in_step_ms, _, _, _ = verify_pass(False)
     verify_prof_ms, gemm_ms, attn_ms, gemm_n = verify_pass(True)
 

@@ -284,9 +284,9 @@ bool attention_tma_supported(const laser_model* m, const laser_kv* kv) {
   return kv->has_pages_map && (m->cfg.head_dim == 64 || m->cfg.head_dim == 128);
 }
 
-laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const int32_t* seq_ids, int B, bool tree,
+laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const int32_t* seq_ids, int B, int Rs, bool tree,
                                   cudaStream_t stream) {
-  const int dh = m->cfg.head_dim, H = m->cfg.n_heads, Hkv = m->cfg.n_kv_heads, Rs = m->rows_per_seq;
+  const int dh = m->cfg.head_dim, H = m->cfg.n_heads, Hkv = m->cfg.n_kv_heads;
   const int64_t rows_per_layer = int64_t(kv->n_pages) * 2 * Hkv * 16;
   const int layer_row0 = int(rows_per_layer * layer);
   const int tiles = ceil_div(Rs, 16), tpc = tiles > 1 ? 2 : 1;   // row tiles of a sequence; tiles per CTA

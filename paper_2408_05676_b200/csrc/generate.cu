@@ -21,21 +21,22 @@ struct GenState {
   int max_total;
 };
 
-// Prompt chunk for the prefill: up to Rs of the not yet cached prompt tokens (all but the last).
-__global__ void prefill_rows_kernel(GenState g, int B, int Rs, int32_t* __restrict__ tokens, int32_t* __restrict__ n_rows) {
-  const int b = blockIdx.x;
+// Prompt chunk for the prefill of sequences b0 .. b0 + nb - 1: up to Rs of the not yet cached prompt
+// tokens (all but the last) of each.
+__global__ void prefill_rows_kernel(GenState g, int b0, int Rs, int32_t* __restrict__ tokens, int32_t* __restrict__ n_rows) {
+  const int i = blockIdx.x, b = b0 + i;
   const int remaining = g.prompt_len[b] - 1 - g.cursor[b];
   const int n = max(0, min(Rs, remaining));
   for (int j = threadIdx.x; j < Rs; j += blockDim.x)
-    tokens[b * Rs + j] = j < n ? g.seq_tok[size_t(b) * g.max_total + g.cursor[b] + j] : -1;
-  if (threadIdx.x == 0) n_rows[b] = n;
+    tokens[i * Rs + j] = j < n ? g.seq_tok[size_t(b) * g.max_total + g.cursor[b] + j] : -1;
+  if (threadIdx.x == 0) n_rows[i] = n;
 }
 
-__global__ void prefill_advance_kernel(GenState g, int B, const int32_t* __restrict__ n_rows, int32_t* __restrict__ kv_len) {
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b >= B) return;
-  g.cursor[b] += n_rows[b];
-  kv_len[b] += n_rows[b];
+__global__ void prefill_advance_kernel(GenState g, int b0, int nb, const int32_t* __restrict__ n_rows, int32_t* __restrict__ kv_len) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= nb) return;
+  g.cursor[b0 + i] += n_rows[i];
+  kv_len[b0 + i] += n_rows[i];
 }
 
 // Tail (last n_max tokens, right-aligned) and pending token of every active sequence.
@@ -146,7 +147,7 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
   LASER_TRY(buf.get(&g.cursor, size_t(B)));
   LASER_TRY(buf.get(&g.counters, size_t(4)));
   LASER_TRY(buf.get(&g.n_active, size_t(1)));
-  LASER_TRY(buf.get(&tokens, size_t(B) * Rs));
+  LASER_TRY(buf.get(&tokens, std::max(size_t(B) * Rs, size_t(m->R_pad))));
   LASER_TRY(buf.get(&n_rows, size_t(B)));
   LASER_TRY(buf.get(&tails, size_t(B) * n_max));
   LASER_TRY(buf.get(&tail_len, size_t(B)));
@@ -187,14 +188,23 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
   float ms_prefill = 0, ms_draft = 0, ms_verify = 0, ms_accept = 0, ms;
   LASER_CUDA(cudaEventRecord(ev.e[0], stream));
 
-  // prefill: every prompt token but the last, Rs rows per sequence per pass
-  const int passes = ceil_div(std::max(max_prompt - 1, 0), Rs);
-  for (int it = 0; it < passes; ++it) {
-    prefill_rows_kernel<<<B, 32, 0, stream>>>(g, B, Rs, tokens, n_rows);
-    LASER_TRY(laser_verify_step(m, kv, seq_ids, tokens, n_rows, B, logits, stream));
-    prefill_advance_kernel<<<ceil_div(B, 128), 128, 0, stream>>>(g, B, n_rows, kv->seq_len);
-    count_launch(2);
-    if ((it & 15) == 15) LASER_TRY(laser_check(m, stream));   // do not keep launching after a device-side error
+  // prefill: every prompt token but the last.  A pass of Rs rows per sequence would read a sequence's
+  // whole cached prefix once per Rs prompt tokens; instead the model's row workspace is given to few
+  // sequences at a time, up to 128 rows each, and the LM head is left out.
+  const int chunk = std::max(Rs, std::min(128, m->R_pad / 16 * 16));
+  const int group = std::max(1, std::min(B, m->R_pad / chunk));
+  int n_pass = 0;
+  for (int b0 = 0; b0 < B; b0 += group) {
+    const int nb = std::min(group, B - b0);
+    int longest = 0;
+    for (int b = b0; b < b0 + nb; ++b) longest = std::max(longest, h_len[b] - 1);
+    for (int it = 0; it < ceil_div(longest, chunk); ++it, ++n_pass) {
+      prefill_rows_kernel<<<nb, 32, 0, stream>>>(g, b0, chunk, tokens, n_rows);
+      LASER_TRY(prefill_rows(m, kv, seq_ids + b0, tokens, n_rows, nb, chunk, stream));
+      prefill_advance_kernel<<<ceil_div(nb, 128), 128, 0, stream>>>(g, b0, nb, n_rows, kv->seq_len);
+      count_launch(2);
+      if ((n_pass & 15) == 15) LASER_TRY(laser_check(m, stream));   // do not keep launching after a device-side error
+    }
   }
   LASER_CUDA(cudaEventRecord(ev.e[1], stream));
   LASER_CUDA(cudaStreamSynchronize(stream));

@@ -445,11 +445,12 @@ LASER_API laser_status laser_check(laser_model* m, void* stream) {
 }
 
 static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
-                                const int32_t* parents, const int32_t* n_rows, int32_t B, float* logits, void* stream_);
+                                const int32_t* parents, const int32_t* n_rows, int32_t B, int32_t Rs, float* logits, void* stream_);
 
 LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
                                          const int32_t* n_rows, int32_t B, float* logits, void* stream) {
-  return verify_impl(m, kv, seq_ids, tokens, nullptr, n_rows, B, logits, stream);
+  LASER_REQUIRE(m && logits, "null argument");
+  return verify_impl(m, kv, seq_ids, tokens, nullptr, n_rows, B, m->rows_per_seq, logits, stream);
 }
 
 LASER_API laser_status laser_verify_step_tree(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
@@ -457,20 +458,32 @@ LASER_API laser_status laser_verify_step_tree(laser_model* m, laser_kv* kv, cons
                                               void* stream) {
   LASER_REQUIRE(parents, "null argument");
   LASER_REQUIRE(m && m->rows_per_seq <= 64, "a token tree has at most 64 rows (K + 1 = %d)", m ? m->rows_per_seq : 0);
-  return verify_impl(m, kv, seq_ids, tokens, parents, n_rows, B, logits, stream);
+  LASER_REQUIRE(logits, "null argument");
+  return verify_impl(m, kv, seq_ids, tokens, parents, n_rows, B, m->rows_per_seq, logits, stream);
 }
 
+namespace laser {
+// Prompt processing (the x_<=t of Eq. 3): the same forward over B sequences with Rs rows each, any Rs
+// with B * Rs inside the model's row workspace; only K and V are wanted, so the LM head is left out.
+laser_status prefill_rows(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
+                          const int32_t* n_rows, int32_t B, int32_t Rs, cudaStream_t stream) {
+  return verify_impl(m, kv, seq_ids, tokens, nullptr, n_rows, B, Rs, nullptr, stream);
+}
+}  // namespace laser
+
+// The forward over B sequences of Rs rows each; logits == nullptr: no LM head (prompt processing).
 static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
-                                const int32_t* parents, const int32_t* n_rows, int32_t B, float* logits, void* stream_) {
-  LASER_REQUIRE(m && kv && seq_ids && tokens && n_rows && logits, "null argument");
-  LASER_REQUIRE(B >= 1 && B <= m->cfg.max_batch, "B = %d outside [1, max_batch = %d]", B, m->cfg.max_batch);
+                                const int32_t* parents, const int32_t* n_rows, int32_t B, int32_t Rs, float* logits, void* stream_) {
+  LASER_REQUIRE(m && kv && seq_ids && tokens && n_rows, "null argument");
+  LASER_REQUIRE(B >= 1 && Rs >= 1 && B <= m->cfg.max_batch && int64_t(B) * Rs <= m->R_pad,
+                "B = %d sequences of %d rows outside the model's %d rows (max_batch = %d)", B, Rs, m->R_pad, m->cfg.max_batch);
   LASER_REQUIRE(kv->n_layers == m->cfg.n_layers && kv->n_kv_heads == m->cfg.n_kv_heads && kv->head_dim == m->cfg.head_dim,
                 "cache was created for another model shape");
   // the LM head stores four logits at a time
   LASER_REQUIRE((reinterpret_cast<uintptr_t>(logits) & 15) == 0, "logits must be 16-byte aligned");
   cudaStream_t stream = as_stream(stream_);
   const laser_model_cfg& c = m->cfg;
-  const int Rs = m->rows_per_seq, R = B * Rs, Rp = ceil_div(R, 16) * 16;
+  const int R = B * Rs, Rp = ceil_div(R, 16) * 16;
   const int d = c.d_model, f = c.d_ffn, dh = c.head_dim, H = c.n_heads, Hkv = c.n_kv_heads;
   const int capacity = int(std::min<int64_t>(kv->capacity_tokens(), INT32_MAX));
 
@@ -510,7 +523,7 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
     {
       ProfScope ps(m, 1, stream);
       if (use_tma_attn) {
-        LASER_TRY(attention_tma_launch(m, kv, l, seq_ids, B, tree, stream));
+        LASER_TRY(attention_tma_launch(m, kv, l, seq_ids, B, Rs, tree, stream));
       } else {
         attention_kernel<<<dim3(B, H), 128, attn_smem, stream>>>(m->q, seq_ids, m->row_ctx, m->row_n, Rs, H, Hkv, dh,
                                                                 kv->page_table, kv->pages_per_seq, pages_l,
@@ -540,7 +553,7 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
     }
     norm_tiles = d_tiles;
   }
-  {  // final norm (as a row scale) and LM head straight into the caller's logits
+  if (logits) {  // final norm (as a row scale) and LM head straight into the caller's logits
     GemmEpilogue e = base;
     e.sumsq_in = m->sumsq; e.sumsq_in_tiles = norm_tiles;
     e.out = logits; e.ldo = c.vocab; e.R_store = R;

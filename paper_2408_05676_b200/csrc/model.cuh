@@ -93,7 +93,12 @@ struct ProfScope {
 // TMA-fed paged attention (head_dim 64 or 128 and a cache small enough for 32-bit row
 // coordinates); the verify forward falls back to a plain kernel otherwise.
 bool attention_tma_supported(const laser_model* m, const laser_kv* kv);
-laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const int32_t* seq_ids, int B, bool tree,
+laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const int32_t* seq_ids, int B, int Rs, bool tree,
                                   cudaStream_t stream);
+
+// Prompt processing: the verify forward without the LM head over B sequences of Rs rows each (any Rs with
+// B * Rs inside the model's row workspace); K and V of the rows go to the cache, lengths are not changed.
+laser_status prefill_rows(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
+                          const int32_t* n_rows, int32_t B, int32_t Rs, cudaStream_t stream);
 
 }  // namespace laser

