@@ -226,6 +226,9 @@ laser_status laser_kv_set_len(laser_kv* kv, const int32_t* seq_ids, const int32_
                               int32_t n, void* stream);
 laser_status laser_kv_get_len(const laser_kv* kv, const int32_t* seq_ids, int32_t* lens,
                               int32_t n, void* stream);
+/* Forgets every sequence of the cache: all committed lengths become 0 (the pages keep their
+ * contents, which are no longer valid).  Asynchronous on `stream`. */
+laser_status laser_kv_reset(laser_kv* kv, void* stream);
 /* Same as laser_kv_set_len for slots 0..n-1 with a dev int32[n] source; asynchronous. */
 laser_status laser_kv_set_len_dev(laser_kv* kv, const int32_t* lens_dev, int32_t n, void* stream);
 /* Copy K and V of one layer for token positions [pos0, pos0+n) of one sequence between the

@@ -59,7 +59,7 @@ class Stats(C.Structure):
 EXPORTS = ["laser_version", "laser_last_error", "laser_launch_count", "laser_pool_build", "laser_pool_free",
            "laser_pool_info", "laser_draft", "laser_draft_temp", "laser_draft_tree", "laser_make_rows", "laser_make_rows_tree", "laser_model_create", "laser_model_free",
            "laser_kv_create", "laser_kv_free", "laser_kv_set_page_table", "laser_kv_set_len",
-           "laser_kv_get_len", "laser_kv_set_len_dev", "laser_kv_import", "laser_kv_export",
+           "laser_kv_get_len", "laser_kv_reset", "laser_kv_set_len_dev", "laser_kv_import", "laser_kv_export",
            "laser_verify_step", "laser_verify_step_tree", "laser_check", "laser_profile_enable", "laser_profile_read", "laser_accept_commit", "laser_accept_commit_noalloc", "laser_accept_tree", "laser_kv_compact_path",
            "laser_selftest_wait", "laser_group_kmeans", "laser_generate"]
 
@@ -284,6 +284,10 @@ def kv_set_len(kv: KV, seq_ids: Sequence[int], lens: Sequence[int], stream=None)
     s = np.ascontiguousarray(seq_ids, dtype=np.int32)
     l = np.ascontiguousarray(lens, dtype=np.int32)
     _chk(lib.laser_kv_set_len(kv.handle, _ptr(s), _ptr(l), C.c_int32(len(s)), _stream(stream)))
+
+
+def kv_reset(kv: KV, stream=None) -> None:
+    _chk(lib.laser_kv_reset(kv.handle, _stream(stream)))
 
 
 def kv_set_len_dev(kv: KV, lens_dev: torch.Tensor, stream=None) -> None:

@@ -87,14 +87,33 @@ __global__ void step_append_kernel(GenState g, int B, int Rs, int max_new, int e
   }
 }
 
+// Work buffers of one laser_generate call, carved out of one allocation that the model keeps and only
+// ever grows: requests are collected first, then placed (256-byte aligned) and cleared together.
 struct DevBuf {
-  std::vector<void*> ptrs;
-  ~DevBuf() { for (void* p : ptrs) cudaFree(p); }
+  struct Req { void** p; size_t bytes; };
+  std::vector<Req> reqs;
   template <typename T>
   laser_status get(T** p, size_t count) {
-    LASER_CUDA(cudaMalloc(reinterpret_cast<void**>(p), std::max<size_t>(count, 1) * sizeof(T)));
-    LASER_CUDA(cudaMemset(*p, 0, std::max<size_t>(count, 1) * sizeof(T)));
-    ptrs.push_back(*p);
+    reqs.push_back(Req{reinterpret_cast<void**>(p), std::max<size_t>(count, 1) * sizeof(T)});
+    return LASER_OK;
+  }
+  laser_status commit(laser_model* m, cudaStream_t stream) {
+    size_t total = 0;
+    for (const Req& r : reqs) total += (r.bytes + 255) & ~size_t(255);
+    if (total > m->gen_bytes) {
+      LASER_CUDA(cudaStreamSynchronize(stream));
+      if (m->gen_buf) {
+        LASER_CUDA(cudaFree(m->gen_buf));
+        m->owned.erase(std::remove(m->owned.begin(), m->owned.end(), m->gen_buf), m->owned.end());
+      }
+      m->gen_buf = nullptr; m->gen_bytes = 0;
+      LASER_CUDA(cudaMalloc(&m->gen_buf, total));
+      m->owned.push_back(m->gen_buf);
+      m->gen_bytes = total;
+    }
+    LASER_CUDA(cudaMemsetAsync(m->gen_buf, 0, total, stream));
+    size_t off = 0;
+    for (const Req& r : reqs) { *r.p = static_cast<char*>(m->gen_buf) + off; off += (r.bytes + 255) & ~size_t(255); }
     return LASER_OK;
   }
 };
@@ -165,6 +184,7 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
   LASER_TRY(buf.get(&n_out, size_t(B)));
   LASER_TRY(buf.get(&d_out, size_t(B) * p->max_new));
   LASER_TRY(buf.get(&logits, size_t(B) * Rs * m->cfg.vocab));
+  LASER_TRY(buf.commit(m, stream));
 
   // host -> device: prompts, lengths, ids
   std::vector<int32_t> h_len(B), h_ids(B);

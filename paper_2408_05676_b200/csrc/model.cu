@@ -388,6 +388,12 @@ LASER_API laser_status laser_kv_set_len(laser_kv* kv, const int32_t* seq_ids, co
   return LASER_OK;
 }
 
+LASER_API laser_status laser_kv_reset(laser_kv* kv, void* stream) {
+  LASER_REQUIRE(kv, "null argument");
+  LASER_CUDA(cudaMemsetAsync(kv->seq_len, 0, size_t(kv->max_seqs) * 4, as_stream(stream)));
+  return LASER_OK;
+}
+
 LASER_API laser_status laser_kv_set_len_dev(laser_kv* kv, const int32_t* lens_dev, int32_t n, void* stream) {
   LASER_REQUIRE(kv && lens_dev && n >= 0 && n <= kv->max_seqs, "bad argument");
   if (n == 0) return LASER_OK;

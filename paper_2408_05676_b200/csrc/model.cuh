@@ -28,6 +28,8 @@ struct laser_model {
   unsigned long long* row_mask = nullptr;  // [R_pad] token tree: rows of its sequence a row attends to (bit j = row j)
   int32_t* status = nullptr;       // first device-side error of the stream, 0 = none
   void* gemm_state = nullptr;      // tensor-map cache of the tensor-core GEMM
+  void* gen_buf = nullptr;         // work buffers of laser_generate, kept between calls (in `owned`)
+  size_t gen_bytes = 0;
   // optional per-class kernel timing (class 0 = GEMM, 1 = attention)
   bool profile = false;
   std::vector<cudaEvent_t> prof_events[2];  // begin/end pairs

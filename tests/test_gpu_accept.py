@@ -70,6 +70,8 @@ def test_commit_advances_cache_length_and_calls_repeat(L):
     exp = np.asarray([10, 11, 12, 13, 14, 15, 16, 17])
     exp[seq_ids] += 3 * want[2]
     assert (lens == exp).all()
+    L.kv_reset(kv)                      # every committed length back to zero
+    assert (L.kv_get_len(kv, list(range(8))) == 0).all()
 
 
 def test_rejects_bad_arguments(L):
