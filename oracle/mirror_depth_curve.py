@@ -8,7 +8,7 @@ logits the two give when the model is cut after L = 1, 2, 4, 8, 16, 32 layers (f
 applied to the residual stream leaving layer L).  The table answers: how far can ANY implementation
 that feeds bf16 activations to its matrix products be from the exact forward at this width and depth.
 
-    python -m oracle.mirror_depth_curve [--layers 32] [--rows 9] [--write the benchmark spec]
+    python -m oracle.mirror_depth_curve [--layers 32] [--rows 9] [--write FILE]
 
 With --write the table replaces the block between the markers
 `<!-- mirror-depth-curve:begin -->` and `<!-- mirror-depth-curve:end -->` of that file.
@@ -68,7 +68,7 @@ def curve(n_layers: int, rows: int, ctx: int, depths, seed_w: int = 0, seed_kv: 
 def table(rows_out, rows, ctx) -> str:
     lines = ["Yardstick: fp64 forward with bf16-rounded matrix-product operands against the exact fp64 forward,",
              "7B width, one sequence, %d cached tokens, %d rows x 32000 logits (written by" % (ctx, rows),
-             "`python -m oracle.mirror_depth_curve --write BASELINE.md`; CPU only, oracle only).", "",
+             "`python -m oracle.mirror_depth_curve --write <this file>`; CPU only, oracle only).", "",
              "| layers L | max-abs | rms | logit std | arg-max agreement |", "|---|---|---|---|---|"]
     for r in rows_out:
         lines.append("| %d | %.4f | %.5f | %.3f | %.2f |" % (r["L"], r["max_abs"], r["rms"], r["logit_std"], r["argmax_agree"]))
