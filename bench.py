@@ -391,7 +391,12 @@ def run_ours(args):
                      "achieved": gemm_gbs, "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
                      "frac": gemm_gbs / peaks["hbm_gbs"], "traffic": GEMM_DRAM_TRAFFIC_PER_STEP if args.layers == 32 else None,
                      "traffic_note": "ncu dram read+write summed over the 129 launches of a step (per-launch figures in profiles/gemm_tc_kernel_7b_rows144.md, scaled from a 2-layer capture: per-launch traffic does not depend on the layer count)",
-                     "algorithmic_bytes_per_step": ab["weights"], "ms_per_step": gemm_ms, "launches_per_step": gemm_n // args.steps},
+                     "algorithmic_bytes_per_step": ab["weights"], "ms_per_step": gemm_ms, "launches_per_step": gemm_n // args.steps,
+                     "in_pipeline_estimate": {
+                         "note": "the event brackets stop consecutive launches from overlapping; scaling the bracketed "
+                                 "share of the contractions to the unbracketed verify step gives their time inside the pipeline",
+                         "ms_per_step": verify_ms * gemm_ms / verify_prof_ms,
+                         "frac": ab["weights"] / (verify_ms * gemm_ms / verify_prof_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}},
         "tree_drafting": tree_res,
         "verify_step": {"ms": verify_ms, "how": "laser_verify_step back to back, one pair of events around %d calls" % args.steps,
                         "ms_bracketed_inside_the_step": verify_in_step_ms, "algorithmic_bytes": ab["total"],
