@@ -83,7 +83,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     for (int s = 0; s < stages; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
     mbar_init(smem_u32(&acc_bar), 1);
     mbar_fence_init();
-    tma_prefetch_map(&tmW);
+    // The first weight stages are requested here, before tensor memory is allocated and the CTA's
+    // threads meet: they depend on nothing, and a CTA that starts late (once an earlier kernel's CTA
+    // has left its slot) has its first bytes on the way that much sooner.
+    const uint64_t w_policy0 = make_policy_evict_first();
+    for (int kb = 0; kb < min(stages, nkb); ++kb) {
+      const uint32_t bar = smem_u32(&full_bar[kb]), dst = tiles + uint32_t(kb) * stage_bytes;
+      mbar_expect_tx(bar, stage_bytes);
+      tma_load_2d_hint(dst, &tmW, (kb0 + kb) * kBK, EPI == EPI_SWIGLU ? wtile * 64 : n0, bar, w_policy0);
+      tma_load_2d_hint(dst + w_bytes / 2, &tmW, (kb0 + kb) * kBK, EPI == EPI_SWIGLU ? e.f + wtile * 64 : n0 + 64, bar, w_policy0);
+    }
     tma_prefetch_map(&tmA);
   }
   if (warp == 1) {
@@ -130,10 +139,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const int s = kb % stages;
         load(tiles + uint32_t(s) * stage_bytes + w_bytes, &tmA, (kb0 + kb) * kBK, r0, full0 + uint32_t(s) * 8, a_policy);
       };
-      // The weights do not depend on the kernel before this one: fill the ring with weight
-      // tiles first, and only then wait for the previous kernel's results (the activations).
+      // The ring was filled with weight tiles at the start of the kernel (they do not depend on the
+      // kernel before this one); only now wait for that kernel's results (the activations).
       const int pre = min(stages, nkb);
-      for (int kb = 0; kb < pre; ++kb) { expect(kb % stages); load_w(kb); }
       asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int kb = 0; kb < pre; ++kb) load_a(kb);
       bool ok = true;
