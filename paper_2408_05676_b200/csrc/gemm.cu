@@ -37,6 +37,8 @@ constexpr int kTcThreads = 192;
 constexpr int kMaxStages = 6;
 constexpr int kMaxNT = 192;       // token rows per tile: accumulator staging must fit shared memory
 constexpr int kSmemBudget = 110 * 1024;  // shared memory of one CTA: two CTAs per SM
+constexpr int kSmemBudgetWide = 200 * 1024;  // with two weight tiles per CTA: one CTA per SM
+constexpr int kAccCols = 256;     // tensor-memory columns between the accumulators of a CTA's weight tiles
 
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -54,8 +56,12 @@ __device__ __forceinline__ float4 ld_cluster_f4(uint32_t cluster_addr) {
 __device__ __forceinline__ void st_shared_f32(uint32_t addr, float v) {
   asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v));
 }
-template <int EPI>
-__global__ void __launch_bounds__(kTcThreads, 2)
+// MT = weight tiles per CTA.  1: the form for few token rows (the step is bound by the weight stream;
+// two CTAs per SM).  2: for several token tiles, where the launches are bound by L2->SM traffic: a CTA
+// multiplies two 128-row weight tiles with the same staged activation tile (two accumulators), so the
+// activation bytes per flop halve; one CTA per SM, no K split.
+template <int EPI, int MT>
+__global__ void __launch_bounds__(kTcThreads, MT == 1 ? 2 : 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, const GemmEpilogue e,
                int N, int NT, int total_kb, int kb_per_split, int splits, int stages, int tmem_cols,
                int32_t* __restrict__ status) {
@@ -68,11 +74,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its prologue
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
-  const uint32_t w_bytes = kBM * 128, a_bytes = uint32_t(NT) * 128, stage_bytes = w_bytes + a_bytes;
+  const uint32_t w_bytes = kBM * 128, a_bytes = uint32_t(NT) * 128, stage_bytes = MT * w_bytes + a_bytes;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int krank = blockIdx.x % splits, ttile = blockIdx.x / splits;   // cluster rank = K range
   const int wtile = blockIdx.y;
-  const int r0 = ttile * NT, n0 = wtile * kBM;
+  const int r0 = ttile * NT, n0 = wtile * kBM * MT;           // wtile counts groups of MT weight tiles
   const int kb0 = krank * kb_per_split;
   const int nkb = max(0, min(kb_per_split, total_kb - kb0));
   const int slice = (NT + splits - 1) / splits;            // token columns finished by one CTA of the cluster
@@ -90,8 +96,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     for (int kb = 0; kb < min(stages, nkb); ++kb) {
       const uint32_t bar = smem_u32(&full_bar[kb]), dst = tiles + uint32_t(kb) * stage_bytes;
       mbar_expect_tx(bar, stage_bytes);
-      tma_load_2d_hint(dst, &tmW, (kb0 + kb) * kBK, EPI == EPI_SWIGLU ? wtile * 64 : n0, bar, w_policy0);
-      tma_load_2d_hint(dst + w_bytes / 2, &tmW, (kb0 + kb) * kBK, EPI == EPI_SWIGLU ? e.f + wtile * 64 : n0 + 64, bar, w_policy0);
+#pragma unroll
+      for (int t = 0; t < MT; ++t) {
+        const int T = wtile * MT + t;
+        tma_load_2d_hint(dst + t * w_bytes, &tmW, (kb0 + kb) * kBK, EPI == EPI_SWIGLU ? T * 64 : T * kBM, bar, w_policy0);
+        tma_load_2d_hint(dst + t * w_bytes + w_bytes / 2, &tmW, (kb0 + kb) * kBK, EPI == EPI_SWIGLU ? e.f + T * 64 : T * kBM + 64, bar, w_policy0);
+      }
     }
     tma_prefetch_map(&tmA);
   }
@@ -104,19 +114,34 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = tmem_slot;
 
-  const int nfeat = n0 + 4 * lane;
-  const LaneCtx lc = make_lane_ctx<EPI>(e, n0, lane, N);
-  uint2 gain4 = make_uint2(0u, 0u);   // gains of the next norm: a weight, not a result of the kernel before
-  if (EPI == EPI_RESID && nfeat < N) gain4 = *reinterpret_cast<const uint2*>(e.gain_next + nfeat);
-  auto fetch_operands = [&](int jj, float4& g0, float4& g1) {
-    g0 = make_float4(0.f, 0.f, 0.f, 0.f); g1 = g0;
-    const int r = r0 + krank * slice + jj;
-    if (jj < own && r < e.R_rows && nfeat < N) {
-      if (EPI == EPI_RESID) g0 = *reinterpret_cast<const float4*>(e.resid + size_t(r) * N + nfeat);
-      if (EPI == EPI_QKV && lc.kind < 2) {
-        const float* cs = e.rope + size_t(r) * e.dh + lc.rope_off;
-        g0 = *reinterpret_cast<const float4*>(cs);       // c0 s0 c1 s1
-        g1 = *reinterpret_cast<const float4*>(cs + 4);   // c2 s2 c3 s3
+  // gains of the next norm for the first weight tile: a weight, not a result of the kernel before, so
+  // requested now, long before the epilogue uses it
+  uint2 gain4_first = make_uint2(0u, 0u);
+  if (EPI == EPI_RESID && n0 + 4 * lane < N) gain4_first = *reinterpret_cast<const uint2*>(e.gain_next + n0 + 4 * lane);
+  bool acc_ok = true;
+  // accumulator t from tensor memory to shared memory, token-major [NT][128] (epilogue warps; a warp may
+  // only touch its own 32 TMEM lanes)
+  auto drain = [&](int t) {
+    const int quarter = warp & 3;
+    const uint32_t src = tmem_acc + uint32_t(t) * kAccCols + (uint32_t(quarter * 32) << 16);
+    const uint32_t dst0 = tiles + uint32_t((quarter * 32 + lane) * 4);
+    for (int c = 0; c < NT; c += 48) {   // three loads in flight, one wait; reads past NT stay inside the allocation
+      uint32_t v0[16], v1[16], v2[16];
+      if (acc_ok && nkb > 0) {
+        tmem_ld16(src + uint32_t(c), v0);
+        if (c + 16 < NT) tmem_ld16(src + uint32_t(c + 16), v1);
+        if (c + 32 < NT) tmem_ld16(src + uint32_t(c + 32), v2);
+        tmem_ld_wait();
+      } else {
+#pragma unroll
+        for (int x = 0; x < 16; ++x) v0[x] = v1[x] = v2[x] = 0u;
+      }
+      const uint32_t dst = dst0 + uint32_t(c) * (kBM * 4);
+#pragma unroll
+      for (int x = 0; x < 16; ++x) {
+        if (c + x < NT) st_shared_f32(dst + x * (kBM * 4), __uint_as_float(v0[x]));
+        if (c + 16 + x < NT) st_shared_f32(dst + (16 + x) * (kBM * 4), __uint_as_float(v1[x]));
+        if (c + 32 + x < NT) st_shared_f32(dst + (32 + x) * (kBM * 4), __uint_as_float(v2[x]));
       }
     }
   };
@@ -132,12 +157,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       auto load_w = [&](int kb) {
         const int s = kb % stages, k = (kb0 + kb) * kBK;
         const uint32_t dst = tiles + uint32_t(s) * stage_bytes, bar = full0 + uint32_t(s) * 8;
-        load(dst, &tmW, k, EPI == EPI_SWIGLU ? wtile * 64 : n0, bar, w_policy);
-        load(dst + w_bytes / 2, &tmW, k, EPI == EPI_SWIGLU ? e.f + wtile * 64 : n0 + 64, bar, w_policy);
+#pragma unroll
+        for (int t = 0; t < MT; ++t) {
+          const int T = wtile * MT + t;
+          load(dst + t * w_bytes, &tmW, k, EPI == EPI_SWIGLU ? T * 64 : T * kBM, bar, w_policy);
+          load(dst + t * w_bytes + w_bytes / 2, &tmW, k, EPI == EPI_SWIGLU ? e.f + T * 64 : T * kBM + 64, bar, w_policy);
+        }
       };
       auto load_a = [&](int kb) {
         const int s = kb % stages;
-        load(tiles + uint32_t(s) * stage_bytes + w_bytes, &tmA, (kb0 + kb) * kBK, r0, full0 + uint32_t(s) * 8, a_policy);
+        load(tiles + uint32_t(s) * stage_bytes + MT * w_bytes, &tmA, (kb0 + kb) * kBK, r0, full0 + uint32_t(s) * 8, a_policy);
       };
       // The ring was filled with weight tiles at the start of the kernel (they do not depend on the
       // kernel before this one); only now wait for that kernel's results (the activations).
@@ -167,10 +196,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t w_addr = tiles + uint32_t(s) * stage_bytes;
-        const uint64_t wdesc = umma_desc(w_addr), adesc = umma_desc(w_addr + w_bytes);
+        const uint64_t adesc = umma_desc(w_addr + MT * w_bytes);
 #pragma unroll
-        for (int k = 0; k < kBK / 16; ++k)  // 16 bf16 = 32 bytes further along K inside the swizzle span
-          umma_bf16(tmem_acc, wdesc + uint64_t(k * 2), adesc + uint64_t(k * 2), idesc, (kb | k) != 0);
+        for (int t = 0; t < MT; ++t) {
+          const uint64_t wdesc = umma_desc(w_addr + t * w_bytes);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k)  // 16 bf16 = 32 bytes further along K inside the swizzle span
+            umma_bf16(tmem_acc + uint32_t(t) * kAccCols, wdesc + uint64_t(k * 2), adesc + uint64_t(k * 2), idesc, (kb | k) != 0);
+        }
         umma_commit(smem_u32(&empty_bar[s]));
       }
       // arrives when every MMA issued so far has finished
@@ -196,38 +229,43 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       }
       s_rstd[j] = rstd; s_pos[j] = pos; s_page[j] = page;
     }
-    // part 2: accumulator from tensor memory to shared memory, token-major [NT][128]
-    const int quarter = warp & 3;  // a warp may only touch its own 32 TMEM lanes
-    const bool ok = mbar_wait(smem_u32(&acc_bar), 0, &abort_flag);
+    // part 2: the first accumulator to shared memory
+    acc_ok = mbar_wait(smem_u32(&acc_bar), 0, &abort_flag);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t src = tmem_acc + (uint32_t(quarter * 32) << 16);
-    const uint32_t dst0 = tiles + uint32_t((quarter * 32 + lane) * 4);
-    for (int c = 0; c < NT; c += 48) {   // three loads in flight, one wait; reads past NT stay inside the allocation
-      uint32_t v0[16], v1[16], v2[16];
-      if (ok && nkb > 0) {
-        tmem_ld16(src + uint32_t(c), v0);
-        if (c + 16 < NT) tmem_ld16(src + uint32_t(c + 16), v1);
-        if (c + 32 < NT) tmem_ld16(src + uint32_t(c + 32), v2);
-        tmem_ld_wait();
-      } else {
+    drain(0);
+  }
 #pragma unroll
-        for (int x = 0; x < 16; ++x) v0[x] = v1[x] = v2[x] = 0u;
-      }
-      const uint32_t dst = dst0 + uint32_t(c) * (kBM * 4);
-#pragma unroll
-      for (int x = 0; x < 16; ++x) {
-        if (c + x < NT) st_shared_f32(dst + x * (kBM * 4), __uint_as_float(v0[x]));
-        if (c + 16 + x < NT) st_shared_f32(dst + (16 + x) * (kBM * 4), __uint_as_float(v1[x]));
-        if (c + 32 + x < NT) st_shared_f32(dst + (32 + x) * (kBM * 4), __uint_as_float(v2[x]));
-      }
-    }
+  for (int t = 0; t < MT; ++t) {   // the CTA's weight tiles, one after the other through the same staging buffer
+  if (t > 0) {
+    __syncthreads();               // the staged tile before this one has been finished
+    if (warp >= 2) drain(t);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (splits > 1) cluster_sync_all();  // every partial tile of the cluster is staged
+  const int wt = wtile * MT + t, n0t = wt * kBM;
+  const int nfeat = n0t + 4 * lane;
+  const LaneCtx lc = make_lane_ctx<EPI>(e, n0t, lane, N);
+  uint2 gain4 = gain4_first;
+  if (EPI == EPI_RESID && t > 0 && nfeat < N) gain4 = *reinterpret_cast<const uint2*>(e.gain_next + nfeat);
+  auto fetch_operands = [&](int jj, float4& g0, float4& g1) {
+    g0 = make_float4(0.f, 0.f, 0.f, 0.f); g1 = g0;
+    const int r = r0 + krank * slice + jj;
+    if (jj < own && r < e.R_rows && nfeat < N) {
+      if (EPI == EPI_RESID) g0 = *reinterpret_cast<const float4*>(e.resid + size_t(r) * N + nfeat);
+      if (EPI == EPI_QKV && lc.kind < 2) {
+        const float* cs = e.rope + size_t(r) * e.dh + lc.rope_off;
+        g0 = *reinterpret_cast<const float4*>(cs);       // c0 s0 c1 s1
+        g1 = *reinterpret_cast<const float4*>(cs + 4);   // c2 s2 c3 s3
+      }
+    }
+  };
 
   __syncwarp();
-  if ((EPI == EPI_SWIGLU || EPI == EPI_PLAIN) && splits == 1) {
+  // (an odd tile count leaves the last group's second tile beyond the matrix: nothing to finish)
+  const bool tile_valid = EPI == EPI_SWIGLU ? wt * 64 < e.f : n0t < N;
+  if (!tile_valid) {
+  } else if ((EPI == EPI_SWIGLU || EPI == EPI_PLAIN) && splits == 1) {
     // part 3 without partial tiles to sum or operands to prefetch: all six warps finish rows,
     // in wide groups whose loads are issued first.
     constexpr int kWide = 12;
@@ -245,7 +283,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const bool live = jb + b < NT && r < e.R_rows && !(abort_flag);
         const float rstd = s_rstd[j];
         if (EPI == EPI_PLAIN) epi_plain(e, lc, r, live, acc[b], rstd, N);
-        else epi_swiglu(e, r, live, wtile * 64, lane, acc[b], rstd);
+        else epi_swiglu(e, r, live, wt * 64, lane, acc[b], rstd);
       }
     }
   } else {
@@ -280,8 +318,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           const bool live = jj < own && r < e.R_rows && !abort_flag;   // the last token tile may overhang the buffers
           const float rstd = s_rstd[j];
           if (EPI == EPI_PLAIN) epi_plain(e, lc, r, live, acc, rstd, N);
-          else if (EPI == EPI_RESID) epi_resid(e, lc, r, live, lane, acc, N, wtile, g0[b], gain4);
-          else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, live, wtile * 64, lane, acc, rstd);
+          else if (EPI == EPI_RESID) epi_resid(e, lc, r, live, lane, acc, N, wt, g0[b], gain4);
+          else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, live, wt * 64, lane, acc, rstd);
           else epi_qkv(e, lc, r, live, acc, rstd, s_pos[j], s_page[j], g0[b], g1[b]);
         }
       }
@@ -299,6 +337,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
   }
   __syncwarp();
+  }  // weight tiles of the CTA
   if (splits > 1) cluster_sync_all();  // peers may still be reading this CTA's staged tile or tensor memory
   __syncthreads();
   if (warp == 1) {
@@ -333,19 +372,21 @@ laser_status tensor_map(GemmState* st, const void* ptr, int rows, int cols, int 
 
 struct TcShape { int n_ttiles, NT, stages, tmem_cols; size_t smem; };
 
-TcShape tc_shape(int R_pad) {
+// mt = weight tiles per CTA (1 or 2)
+TcShape tc_shape(int R_pad, int mt = 1) {
   TcShape s;
   s.n_ttiles = ceil_div(R_pad, kMaxNT);
   s.NT = ceil_div(ceil_div(R_pad, s.n_ttiles), 16) * 16;
-  const int stage_bytes = kBM * 128 + s.NT * 128;
-  s.stages = std::max(2, std::min(kMaxStages, kSmemBudget / stage_bytes));
+  const int stage_bytes = mt * kBM * 128 + s.NT * 128;
+  s.stages = std::max(2, std::min(kMaxStages, (mt == 1 ? kSmemBudget : kSmemBudgetWide) / stage_bytes));
   s.tmem_cols = 32;
   while (s.tmem_cols < s.NT) s.tmem_cols <<= 1;
+  if (mt == 2) s.tmem_cols = 2 * kAccCols;
   s.smem = std::max(size_t(s.stages) * stage_bytes, size_t(s.NT) * kBM * 4) + 1024;
   return s;
 }
 
-template <int EPI>
+template <int EPI, int MT>
 laser_status launch_epi(const CUtensorMap& tw, const CUtensorMap& ta, const GemmEpilogue& e, int N, const TcShape& sh,
                         int n_wtiles, int total_kb, int kbps, int splits, int32_t* status, cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
@@ -364,18 +405,22 @@ laser_status launch_epi(const CUtensorMap& tw, const CUtensorMap& ta, const Gemm
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  LASER_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI>, tw, ta, e, N, sh.NT, total_kb, kbps, splits, sh.stages,
+  LASER_CUDA(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI, MT>, tw, ta, e, N, sh.NT, total_kb, kbps, splits, sh.stages,
                                 sh.tmem_cols, status));
   return LASER_OK;
 }
 
 laser_status prepare(GemmState* st) {
   if (st->ready) return LASER_OK;
-  const int bytes = kSmemBudget + 2048;
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  const int bytes = kSmemBudget + 2048, wide = kSmemBudgetWide + 2048;
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, wide));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, wide));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, wide));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, wide));
   st->ready = true;
   return LASER_OK;
 }
@@ -405,12 +450,21 @@ laser_status gemm_fused(laser_model* m, const __nv_bfloat16* A, const __nv_bfloa
   LASER_TRY(prepare(st));
   const int n_wtiles = epi == EPI_SWIGLU ? ceil_div(N / 2, 64) : ceil_div(N, kBM);
   const int splits = pick_splits(R_pad, N, K, epi);
-  const TcShape sh = tc_shape(R_pad);
+  // several token tiles and no K split: two weight tiles per CTA share every staged activation tile
+  // (where the halved CTA count still gives every SM one)
+  const int n_tt = tc_shape(R_pad).n_ttiles;
+  const int mt = (n_tt > 1 && splits == 1 && ceil_div(n_wtiles, 2) * n_tt >= 148) ? 2 : 1;
+  const TcShape sh = tc_shape(R_pad, mt);
   const CUtensorMap *tw = nullptr, *ta = nullptr;
   LASER_TRY(tensor_map(st, W, N, K, 64, &tw));
   LASER_TRY(tensor_map(st, A, m->R_pad, K, sh.NT, &ta));
   const int total_kb = ceil_div(K, kBK), kbps = ceil_div(total_kb, splits);
-#define LASER_GEMM_LAUNCH(E) LASER_TRY((launch_epi<E>(*tw, *ta, e, N, sh, n_wtiles, total_kb, kbps, splits, m->status, stream)));
+  const int n_groups = ceil_div(n_wtiles, mt);     // grid rows: groups of mt weight tiles
+#define LASER_GEMM_LAUNCH(E)                                                                                            \
+  do {                                                                                                                  \
+    if (mt == 1) LASER_TRY((launch_epi<E, 1>(*tw, *ta, e, N, sh, n_groups, total_kb, kbps, splits, m->status, stream))); \
+    else LASER_TRY((launch_epi<E, 2>(*tw, *ta, e, N, sh, n_groups, total_kb, kbps, splits, m->status, stream)));         \
+  } while (0);
   switch (epi) {
     case EPI_PLAIN: LASER_GEMM_LAUNCH(EPI_PLAIN) break;
     case EPI_RESID: LASER_GEMM_LAUNCH(EPI_RESID) break;
