@@ -65,14 +65,21 @@ MIRROR_SITES_PER_LAYER = 5
 MIRROR_SITES_FINAL = 1
 
 
-def _r(x: torch.Tensor, mirror: bool) -> torch.Tensor:
-    """Yardstick mode: round an activation to bf16 (nearest-even) where a bf16-operand
-    implementation would hand it to a matrix product; identity otherwise."""
-    return x.to(torch.bfloat16).to(F64) if mirror else x
+def _r(x: torch.Tensor, mirror) -> torch.Tensor:
+    """Yardstick mode: round an activation where a bf16-operand implementation would hand it to a matrix
+    product.  mirror = True: to bf16 (nearest-even).  mirror = 2: to a sum of two bf16 values, hi = bf16(x)
+    and lo = bf16(x - hi), which is what an implementation gets that feeds the operand as two bf16
+    matrices (about 16 significant bits).  False: identity."""
+    if not mirror:
+        return x
+    hi = x.to(torch.bfloat16).to(F64)
+    if mirror == 2:
+        return hi + (x - hi).to(torch.bfloat16).to(F64)
+    return hi
 
 
 def forward(W: Dict, cfg: Dict, kv: KVCache, seq_ids: Sequence[int],
-            tokens: Sequence[np.ndarray], mirror_bf16: bool = False,
+            tokens: Sequence[np.ndarray], mirror_bf16=False,
             parents: Optional[Sequence[Sequence[int]]] = None,
             hidden_out: Optional[List[torch.Tensor]] = None) -> List[torch.Tensor]:
     """One forward over the new rows of each listed sequence.

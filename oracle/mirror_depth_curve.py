@@ -44,7 +44,7 @@ def curve(n_layers: int, rows: int, ctx: int, depths, seed_w: int = 0, seed_kv: 
     kv.ctx[:] = ctx
     tokens = np.random.default_rng(seed_tok).integers(0, cfg["vocab"], size=rows).astype(np.int32)
     hid = {}
-    for mirror in (False, True):
+    for mirror in (False, True, 2):
         t0 = time.time()
         hs = []
         O.forward(W, cfg, kv.clone(), [0], [tokens], mirror_bf16=mirror, hidden_out=hs)
@@ -57,10 +57,12 @@ def curve(n_layers: int, rows: int, ctx: int, depths, seed_w: int = 0, seed_kv: 
             continue
         exact = O.rmsnorm(hid[False][L], gain, cfg["rms_eps"]) @ head.T
         mirr = O._r(O.rmsnorm(hid[True][L], gain, cfg["rms_eps"]), True) @ head.T
+        split = O._r(O.rmsnorm(hid[2][L], gain, cfg["rms_eps"]), 2) @ head.T
         diff = mirr - exact
         out.append(dict(L=L, max_abs=float(diff.abs().max()), rms=float(diff.pow(2).mean().sqrt()),
                         logit_std=float(exact.std()),
-                        argmax_agree=float((mirr.argmax(-1) == exact.argmax(-1)).double().mean())))
+                        argmax_agree=float((mirr.argmax(-1) == exact.argmax(-1)).double().mean()),
+                        split_max_abs=float((split - exact).abs().max())))
         print(out[-1], flush=True)
     return out
 
@@ -69,9 +71,11 @@ def table(rows_out, rows, ctx) -> str:
     lines = ["Yardstick: fp64 forward with bf16-rounded matrix-product operands against the exact fp64 forward,",
              "7B width, one sequence, %d cached tokens, %d rows x 32000 logits (written by" % (ctx, rows),
              "`python -m oracle.mirror_depth_curve --write <this file>`; CPU only, oracle only).", "",
-             "| layers L | max-abs | rms | logit std | arg-max agreement |", "|---|---|---|---|---|"]
+             "| layers L | max-abs | rms | logit std | arg-max agreement | max-abs with operands as hi + lo bf16 pairs |",
+             "|---|---|---|---|---|---|"]
     for r in rows_out:
-        lines.append("| %d | %.4f | %.5f | %.3f | %.2f |" % (r["L"], r["max_abs"], r["rms"], r["logit_std"], r["argmax_agree"]))
+        lines.append("| %d | %.4f | %.5f | %.3f | %.2f | %.2e |" % (r["L"], r["max_abs"], r["rms"], r["logit_std"], r["argmax_agree"],
+                                                                   r["split_max_abs"]))
     return "\n".join(lines)
 
 

@@ -257,3 +257,15 @@ def test_hidden_out_observes_the_residual_stream_without_changing_the_result():
     assert torch.equal(hs[0], W["tok_emb"].double()[torch.as_tensor(toks, dtype=torch.long)])
     last = O.rmsnorm(hs[-1], W["final_norm"].double(), CFG["rms_eps"]) @ W["lm_head"].double().T
     assert (last - a).abs().max() < 1e-12
+
+
+def test_split_rounding_keeps_sixteen_bits():
+    """The hi + lo form of the yardstick's rounding: exact on bf16 values, within 2^-16 relative elsewhere,
+    and never worse than the plain bf16 rounding."""
+    g = torch.Generator().manual_seed(3)
+    x = torch.randn(10000, generator=g, dtype=torch.float64) * 37.0
+    r1, r2 = O._r(x, True), O._r(x, 2)
+    assert ((r2 - x).abs() <= 2.0 ** -16 * x.abs()).all()
+    assert ((r2 - x).abs() <= (r1 - x).abs()).all() and ((r1 - x).abs() <= 2.0 ** -8 * x.abs()).all()
+    b = x.to(torch.bfloat16).to(torch.float64)
+    assert torch.equal(O._r(b, 2), b) and torch.equal(O._r(b, True), b) and torch.equal(O._r(x, False), x)
