@@ -103,6 +103,8 @@ typedef struct {
                             generated tokens (temporary branch, Section 3.2; needs max_occ in 1..64) */
   int32_t tree;          /* laser_generate: non-zero = draft a token tree and verify it with tree
                             attention (Section 3.3; needs K <= 32 and max_occ in 1..64)            */
+  int32_t fused_accept;  /* laser_generate: non-zero = chain steps run laser_verify_accept (no logits
+                            are stored); ignored for token trees                                  */
 } laser_params;
 
 typedef struct {
@@ -337,6 +339,27 @@ laser_status laser_accept_commit_noalloc(laser_kv* kv, const int32_t* seq_ids, c
                                          const int32_t* tokens, const int32_t* n_rows, int32_t B,
                                          int32_t V, const laser_params* p, int32_t* n_accept,
                                          int32_t* out_tokens, int32_t* n_out, void* stream);
+
+/* ---- Verify forward with fused acceptance (Section 3.4; Eq. 4, Eq. 7, Eq. 8) -------------
+ * laser_verify_step followed by laser_accept_commit as one call in which the [B, K+1, vocab]
+ * logits are never stored: the LM head's epilogue keeps, per row and 128-token vocabulary tile,
+ * the tile's largest logits with their ids, the tile's sum of exp(l - tile max) and the logit
+ * of the row's draft token, and a small second kernel finishes the rule from those.
+ *   Arguments as for the two calls (p->K must equal the model's max_draft); commit != 0 advances
+ *   the cache lengths by n_out as laser_accept_commit does with a cache.
+ *   logits  dev fp32 [B, K+1, vocab] or NULL.  When given (16-byte aligned), the same launch also
+ *           stores the logits it decided on, so that the verdicts can be checked against the rule
+ *           applied to stored logits; NULL is the form meant for decoding.
+ *   The arg max, the rank test (Eq. 7) and so STRICT and TOPK are exact: identical to
+ *   laser_accept_commit on the stored logits.  Probabilities are combined in fp64 from per-tile
+ *   fp32 sums and agree with the two-pass rule to about 1e-6 relative, so a RELAXED / TOPP /
+ *   RELAXED_ARGMAX verdict can differ only where the draft's probability lies within that distance
+ *   of p.  Rules that rank need topk <= 4 (four logits are kept per tile): UNSUPPORTED otherwise.
+ * Asynchronous on `stream`.  Errors: as laser_verify_step, and INVALID_ARG / UNSUPPORTED above. */
+laser_status laser_verify_accept(laser_model* m, laser_kv* kv, const int32_t* seq_ids,
+                                 const int32_t* tokens, const int32_t* n_rows, int32_t B,
+                                 const laser_params* p, int32_t commit, float* logits,
+                                 int32_t* n_accept, int32_t* out_tokens, int32_t* n_out, void* stream);
 
 /* Self-test of the library's failure path (the paper has no counterpart).  Every wait inside the
  * TMA-fed kernels is bounded; when one runs out the kernel stops waiting, lets its copies in flight

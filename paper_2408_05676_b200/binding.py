@@ -45,7 +45,8 @@ class Weights(C.Structure):
 
 class Params(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("K", "n_min", "n_max", "min_draft", "max_occ", "mode", "topk")] + \
-               [("p", C.c_float), ("max_new", C.c_int32), ("eos_id", C.c_int32), ("temp_branches", C.c_int32), ("tree", C.c_int32)]
+               [("p", C.c_float), ("max_new", C.c_int32), ("eos_id", C.c_int32), ("temp_branches", C.c_int32), ("tree", C.c_int32),
+                ("fused_accept", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -61,6 +62,7 @@ EXPORTS = ["laser_version", "laser_last_error", "laser_launch_count", "laser_poo
            "laser_kv_create", "laser_kv_free", "laser_kv_set_page_table", "laser_kv_set_len",
            "laser_kv_get_len", "laser_kv_reset", "laser_kv_set_len_dev", "laser_kv_import", "laser_kv_export",
            "laser_verify_step", "laser_verify_step_tree", "laser_check", "laser_profile_enable", "laser_profile_read", "laser_accept_commit", "laser_accept_commit_noalloc", "laser_accept_tree", "laser_kv_compact_path",
+           "laser_verify_accept",
            "laser_selftest_wait", "laser_group_kmeans", "laser_generate"]
 
 lib.laser_version.restype = C.c_char_p
@@ -99,8 +101,8 @@ def _stream(stream) -> C.c_void_p:
 
 
 def make_params(K=8, n_min=1, n_max=4, min_draft=1, max_occ=64, mode=MODE_STRICT, topk=2, p=0.1,
-                max_new=0, eos_id=-1, temp_branches=0, tree=0) -> Params:
-    return Params(K, n_min, n_max, min_draft, max_occ, mode, topk, p, max_new, eos_id, temp_branches, tree)
+                max_new=0, eos_id=-1, temp_branches=0, tree=0, fused_accept=0) -> Params:
+    return Params(K, n_min, n_max, min_draft, max_occ, mode, topk, p, max_new, eos_id, temp_branches, tree, fused_accept)
 
 
 def version() -> str:
@@ -391,6 +393,25 @@ def accept_commit(kv: Optional[KV], seq_ids, logits, tokens, n_rows, params: Par
                                  _ptr(seq_ids) if seq_ids is not None else C.c_void_p(0),
                                  _ptr(_dev(logits, torch.float32)), _ptr(_dev(tokens, torch.int32)),
                                  _ptr(_dev(n_rows, torch.int32)), C.c_int32(B), C.c_int32(V), C.byref(params),
+                                 _ptr(n_accept), _ptr(out_tokens), _ptr(n_out), _stream(stream)))
+    return n_accept, out_tokens, n_out
+
+
+def verify_accept(model: Model, kv: KV, seq_ids, tokens, n_rows, params: Params, commit: bool = True, logits=None, out=None,
+                  stream=None):
+    """laser_verify_accept: the verify forward with acceptance fused into the LM head; logits (optional, fp32
+    [B, K+1, vocab]) are stored only when given.  Returns n_accept, out_tokens, n_out (device tensors)."""
+    B = seq_ids.shape[0]
+    R = model.cfg["max_draft"] + 1
+    assert tokens.shape == (B, R), (tokens.shape, B, R)
+    if out is None:
+        dev = tokens.device
+        out = (torch.empty(B, dtype=torch.int32, device=dev), torch.empty(B, R, dtype=torch.int32, device=dev),
+               torch.empty(B, dtype=torch.int32, device=dev))
+    n_accept, out_tokens, n_out = out
+    _chk(lib.laser_verify_accept(model.handle, kv.handle, _ptr(_dev(seq_ids, torch.int32)), _ptr(_dev(tokens, torch.int32)),
+                                 _ptr(_dev(n_rows, torch.int32)), C.c_int32(B), C.byref(params), C.c_int32(1 if commit else 0),
+                                 _ptr(_dev(logits, torch.float32)) if logits is not None else C.c_void_p(0),
                                  _ptr(n_accept), _ptr(out_tokens), _ptr(n_out), _stream(stream)))
     return n_accept, out_tokens, n_out
 

@@ -69,6 +69,73 @@ __device__ __forceinline__ void epi_plain(const GemmEpilogue& e, const LaneCtx& 
   }
 }
 
+// Order-preserving map of finite floats (and infinities) onto unsigned integers, and back
+__device__ __forceinline__ uint32_t f32_to_ordered(float x) {
+  const uint32_t u = __float_as_uint(x);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float ordered_to_f32(uint32_t o) {
+  return __uint_as_float((o & 0x80000000u) ? (o & 0x7fffffffu) : ~o);
+}
+
+// Acceptance fused into the LM head (Eq. 4, Eq. 7, Eq. 8): the warp holds the 128 logits of (row r, vocabulary
+// tile wt).  It leaves the tile's top_n largest logits with their token ids (equal logits: smaller id first), the
+// tile's sum of exp(l - tile max) where the rule needs a probability, and - from the tile that holds it - the logit
+// of the row's draft token.  From these a second, small kernel takes the row's arg max, the draft's rank among the
+// first top_n and its softmax probability without a row of logits ever being stored.  The reductions are warp-wide
+// integer max / min over order-preserving keys: exact, the same from run to run.
+__device__ __forceinline__ void epi_verdict(const GemmEpilogue& e, const LaneCtx& c, int r, bool live, int lane, float4 v,
+                                            float rstd, int N, int wt) {
+  float x[4] = {v.x * rstd, v.y * rstd, v.z * rstd, v.w * rstd};
+  live = live && r < e.R_store;
+  if (e.out && live) {
+    float* o = e.out + size_t(r) * e.ldo + c.n;
+    if (c.vec_out) {
+      *reinterpret_cast<float4*>(o) = make_float4(x[0], x[1], x[2], x[3]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) if (c.n + i < N) o[i] = x[i];
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    if (x[i] == 0.f) x[i] = 0.f;                 // -0 and +0 are one value and must map to one key
+    if (c.n + i >= N) x[i] = -INFINITY;          // beyond the vocabulary
+  }
+  const int off = (live ? e.row_draft[r] : -1) - c.n;
+  if (off >= 0 && off < 4 && c.n + off < N) e.draft_logit[r] = off == 0 ? x[0] : off == 1 ? x[1] : off == 2 ? x[2] : x[3];
+  float tv[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+  int ti[4] = {0x7fffffff, 0x7fffffff, 0x7fffffff, 0x7fffffff};
+  uint32_t taken = 0;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    if (q < e.top_n) {   // uniform over the launch
+      float bv = -INFINITY;
+      int bi = 0x7fffffff, bslot = -1;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)   // ids ascend with i: a strict comparison keeps the smaller id on ties
+        if (!((taken >> i) & 1u) && c.n + i < N && (bslot < 0 || x[i] > bv)) { bv = x[i]; bi = c.n + i; bslot = i; }
+      const uint32_t key = bslot < 0 ? 0u : f32_to_ordered(bv);
+      const uint32_t best = __reduce_max_sync(0xffffffffu, key);
+      const int who = __reduce_min_sync(0xffffffffu, (key == best && bslot >= 0) ? bi : 0x7fffffff);
+      if (bslot >= 0 && bi == who) taken |= 1u << bslot;
+      if (who != 0x7fffffff) { tv[q] = ordered_to_f32(best); ti[q] = who; }
+    }
+  }
+  float s = 0.f;
+  if (e.tile_sum) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) if (c.n + i < N) s += expf(x[i] - tv[0]);
+    for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  }
+  if (live && lane == 0) {
+    const size_t at = size_t(r) * e.n_vtiles + wt;
+    e.top_val[at] = make_float4(tv[0], tv[1], tv[2], tv[3]);
+    e.top_idx[at] = make_int4(ti[0], ti[1], ti[2], ti[3]);
+    if (e.tile_sum) e.tile_sum[at] = s;
+  }
+}
+
 // resid += acc; xb = bf16(resid * gain of the next norm); per-tile sum of squares for that norm
 __device__ __forceinline__ void epi_resid(const GemmEpilogue& e, const LaneCtx& c, int r, bool live, int lane, float4 v, int N,
                                           int tile, float4 x, uint2 g2) {

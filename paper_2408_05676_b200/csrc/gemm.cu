@@ -265,7 +265,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   // (an odd tile count leaves the last group's second tile beyond the matrix: nothing to finish)
   const bool tile_valid = EPI == EPI_SWIGLU ? wt * 64 < e.f : n0t < N;
   if (!tile_valid) {
-  } else if ((EPI == EPI_SWIGLU || EPI == EPI_PLAIN) && splits == 1) {
+  } else if ((EPI == EPI_SWIGLU || EPI == EPI_PLAIN || EPI == EPI_VERDICT) && splits == 1) {
     // part 3 without partial tiles to sum or operands to prefetch: all six warps finish rows,
     // in wide groups whose loads are issued first.
     constexpr int kWide = 12;
@@ -283,6 +283,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const bool live = jb + b < NT && r < e.R_rows && !(abort_flag);
         const float rstd = s_rstd[j];
         if (EPI == EPI_PLAIN) epi_plain(e, lc, r, live, acc[b], rstd, N);
+        else if (EPI == EPI_VERDICT) epi_verdict(e, lc, r, live, lane, acc[b], rstd, N, wt);
         else epi_swiglu(e, r, live, wt * 64, lane, acc[b], rstd);
       }
     }
@@ -318,6 +319,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           const bool live = jj < own && r < e.R_rows && !abort_flag;   // the last token tile may overhang the buffers
           const float rstd = s_rstd[j];
           if (EPI == EPI_PLAIN) epi_plain(e, lc, r, live, acc, rstd, N);
+          else if (EPI == EPI_VERDICT) epi_verdict(e, lc, r, live, lane, acc, rstd, N, wt);
           else if (EPI == EPI_RESID) epi_resid(e, lc, r, live, lane, acc, N, wt, g0[b], gain4);
           else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, live, wt * 64, lane, acc, rstd);
           else epi_qkv(e, lc, r, live, acc, rstd, s_pos[j], s_page[j], g0[b], g1[b]);
@@ -421,6 +423,8 @@ laser_status prepare(GemmState* st) {
   LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_RESID, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, wide));
   LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, wide));
   LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, wide));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_VERDICT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  LASER_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<EPI_VERDICT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, wide));
   st->ready = true;
   return LASER_OK;
 }
@@ -469,6 +473,7 @@ laser_status gemm_fused(laser_model* m, const __nv_bfloat16* A, const __nv_bfloa
     case EPI_PLAIN: LASER_GEMM_LAUNCH(EPI_PLAIN) break;
     case EPI_RESID: LASER_GEMM_LAUNCH(EPI_RESID) break;
     case EPI_SWIGLU: LASER_GEMM_LAUNCH(EPI_SWIGLU) break;
+    case EPI_VERDICT: LASER_GEMM_LAUNCH(EPI_VERDICT) break;
     default: LASER_GEMM_LAUNCH(EPI_QKV) break;
   }
 #undef LASER_GEMM_LAUNCH

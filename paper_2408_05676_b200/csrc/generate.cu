@@ -183,7 +183,8 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
   LASER_TRY(buf.get(&out_tokens, size_t(B) * Rs));
   LASER_TRY(buf.get(&n_out, size_t(B)));
   LASER_TRY(buf.get(&d_out, size_t(B) * p->max_new));
-  LASER_TRY(buf.get(&logits, size_t(B) * Rs * m->cfg.vocab));
+  const bool fused = p->fused_accept && !(pool && p->tree);   // chain steps without stored logits
+  LASER_TRY(buf.get(&logits, fused ? size_t(4) : size_t(B) * Rs * m->cfg.vocab));
   LASER_TRY(buf.commit(m, stream));
 
   // host -> device: prompts, lengths, ids
@@ -258,10 +259,13 @@ LASER_API laser_status laser_generate(laser_model* m, laser_kv* kv, const laser_
     else LASER_TRY(laser_make_rows(last, draft, draft_len, B, K, tokens, n_rows, stream));
     LASER_CUDA(cudaEventRecord(ev.e[1], stream));
     if (tree) LASER_TRY(laser_verify_step_tree(m, kv, seq_ids, tokens, parents, n_rows, B, logits, stream));
+    else if (fused) LASER_TRY(laser_verify_accept(m, kv, seq_ids, tokens, n_rows, B, &acc, 0, nullptr, n_accept, out_tokens, n_out, stream));
     else LASER_TRY(laser_verify_step(m, kv, seq_ids, tokens, n_rows, B, logits, stream));
     ++verify_calls;
     LASER_CUDA(cudaEventRecord(ev.e[2], stream));
-    if (tree) {
+    if (fused && !tree) {
+      // the verdict came with the forward
+    } else if (tree) {
       // verdict, then the accepted path's K/V to consecutive slots (the lengths advance in step_append)
       LASER_TRY(laser_accept_tree(nullptr, nullptr, logits, tokens, parents, n_rows, B, m->cfg.vocab, &acc, n_accept,
                                   out_tokens, n_out, path_rows, stream));

@@ -91,10 +91,15 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 __global__ void __launch_bounds__(256)
 embed_kernel(const int32_t* __restrict__ tokens, int R, int d, int vocab, const bf16* __restrict__ emb,
              const bf16* __restrict__ gain, float* __restrict__ resid, bf16* __restrict__ xb,
-             float* __restrict__ sumsq) {
+             float* __restrict__ sumsq, const int32_t* __restrict__ n_rows, int Rs, int32_t* __restrict__ row_draft) {
   __shared__ float red[8];
   const int r = blockIdx.x;
   const int tok = r < R ? tokens[r] : -1;
+  if (row_draft && threadIdx.x == 0) {   // fused acceptance: the draft token that this row's distribution verifies
+    int dt = -1;
+    if (r < R && (r % Rs) + 1 < min(n_rows[r / Rs], Rs)) dt = tokens[r + 1];
+    row_draft[r] = dt;
+  }
   const bool ok = tok >= 0 && tok < vocab;
   float ss = 0.f;
   for (int j = threadIdx.x; j < d; j += blockDim.x) {
@@ -321,6 +326,12 @@ LASER_API laser_status laser_model_create(const laser_model_cfg* cfg, const lase
   LASER_TRY(model_alloc(m, &m->row_ctx, size_t(cfg->max_batch)));
   LASER_TRY(model_alloc(m, &m->row_n, size_t(cfg->max_batch)));
   LASER_TRY(model_alloc(m, &m->row_mask, size_t(m->R_pad)));
+  const size_t v_tiles = size_t(ceil_div(cfg->vocab, 128));
+  LASER_TRY(model_alloc(m, &m->row_draft, Rp));
+  LASER_TRY(model_alloc(m, &m->draft_logit, Rp));
+  LASER_TRY(model_alloc(m, &m->top_val, Rp * v_tiles));
+  LASER_TRY(model_alloc(m, &m->top_idx, Rp * v_tiles));
+  LASER_TRY(model_alloc(m, &m->tile_sum, Rp * v_tiles));
   LASER_TRY(model_alloc(m, &m->status, size_t(1)));
   guard.p = nullptr;
   *out = m;
@@ -450,8 +461,11 @@ LASER_API laser_status laser_check(laser_model* m, void* stream) {
   return LASER_OK;
 }
 
+// fused: 0 = LM head stores logits (none at all if logits is null); otherwise acceptance is fused into the LM head:
+// the number of largest logits kept per vocabulary tile (1..4), negative when the tile sums of exp are wanted too
 static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
-                                const int32_t* parents, const int32_t* n_rows, int32_t B, int32_t Rs, float* logits, void* stream_);
+                                const int32_t* parents, const int32_t* n_rows, int32_t B, int32_t Rs, float* logits, void* stream_,
+                                int fused = 0);
 
 LASER_API laser_status laser_verify_step(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
                                          const int32_t* n_rows, int32_t B, float* logits, void* stream) {
@@ -475,11 +489,18 @@ laser_status prefill_rows(laser_model* m, laser_kv* kv, const int32_t* seq_ids, 
                           const int32_t* n_rows, int32_t B, int32_t Rs, cudaStream_t stream) {
   return verify_impl(m, kv, seq_ids, tokens, nullptr, n_rows, B, Rs, nullptr, stream);
 }
+// The verify forward whose LM head leaves, per (row, vocabulary tile), what the acceptance rule needs
+// (see GemmEpilogue) in the model's buffers; logits may be null.
+laser_status verify_fused(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
+                          const int32_t* n_rows, int32_t B, float* logits, int top_n, bool sums, cudaStream_t stream) {
+  return verify_impl(m, kv, seq_ids, tokens, nullptr, n_rows, B, m->rows_per_seq, logits, stream, sums ? -top_n : top_n);
+}
 }  // namespace laser
 
 // The forward over B sequences of Rs rows each; logits == nullptr: no LM head (prompt processing).
 static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
-                                const int32_t* parents, const int32_t* n_rows, int32_t B, int32_t Rs, float* logits, void* stream_) {
+                                const int32_t* parents, const int32_t* n_rows, int32_t B, int32_t Rs, float* logits, void* stream_,
+                                int fused) {
   LASER_REQUIRE(m && kv && seq_ids && tokens && n_rows, "null argument");
   LASER_REQUIRE(B >= 1 && Rs >= 1 && B <= m->cfg.max_batch && int64_t(B) * Rs <= m->R_pad,
                 "B = %d sequences of %d rows outside the model's %d rows (max_batch = %d)", B, Rs, m->R_pad, m->cfg.max_batch);
@@ -500,7 +521,8 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
                                           double(c.rope_theta), dh, m->row_pos, m->row_seq, m->row_ctx, m->row_n,
                                           m->rope, m->status);
   const __nv_bfloat16* first_gain = c.n_layers > 0 ? m->attn_norm[0] : m->final_norm;
-  embed_kernel<<<m->R_pad, 256, 0, stream>>>(tokens, R, d, c.vocab, m->tok_emb, first_gain, m->resid, m->xn, m->sumsq);
+  embed_kernel<<<m->R_pad, 256, 0, stream>>>(tokens, R, d, c.vocab, m->tok_emb, first_gain, m->resid, m->xn, m->sumsq, n_rows, Rs,
+                                             fused ? m->row_draft : nullptr);
   count_launch(2);
   const bool use_tma_attn = attention_tma_supported(m, kv);
   const size_t attn_smem = (size_t(dh) + size_t(capacity) + 8) * sizeof(float);
@@ -559,12 +581,17 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
     }
     norm_tiles = d_tiles;
   }
-  if (logits) {  // final norm (as a row scale) and LM head straight into the caller's logits
+  if (logits || fused) {  // final norm (as a row scale) and LM head straight into the caller's logits
     GemmEpilogue e = base;
     e.sumsq_in = m->sumsq; e.sumsq_in_tiles = norm_tiles;
     e.out = logits; e.ldo = c.vocab; e.R_store = R;
+    if (fused) {   // ... or into what the acceptance rule needs of every (row, vocabulary tile)
+      e.row_draft = m->row_draft; e.draft_logit = m->draft_logit; e.top_val = m->top_val; e.top_idx = m->top_idx;
+      e.tile_sum = fused < 0 ? m->tile_sum : nullptr;
+      e.top_n = fused < 0 ? -fused : fused; e.n_vtiles = ceil_div(c.vocab, 128);
+    }
     ProfScope ps(m, 0, stream);
-    LASER_TRY(gemm_fused(m, m->xn, m->lm_head, Rp, c.vocab, d, EPI_PLAIN, e, stream));
+    LASER_TRY(gemm_fused(m, m->xn, m->lm_head, Rp, c.vocab, d, fused ? EPI_VERDICT : EPI_PLAIN, e, stream));
   }
   LASER_CUDA(cudaGetLastError());
   return LASER_OK;

@@ -26,6 +26,12 @@ struct laser_model {
   int32_t* row_ctx = nullptr;      // [max_batch] committed length of each sequence of the step
   int32_t* row_n = nullptr;        // [max_batch] effective rows of each sequence
   unsigned long long* row_mask = nullptr;  // [R_pad] token tree: rows of its sequence a row attends to (bit j = row j)
+  // acceptance fused into the LM head: what its epilogue leaves per (row, 128-token vocabulary tile)
+  int32_t* row_draft = nullptr;    // [R_pad] token whose verdict the row gives, -1 = none
+  float* draft_logit = nullptr;    // [R_pad] logit of that token
+  float4* top_val = nullptr;       // [R_pad][vocab tiles] the tile's four largest logits, in order
+  int4* top_idx = nullptr;         // [R_pad][vocab tiles] their token ids
+  float* tile_sum = nullptr;       // [R_pad][vocab tiles] sum over the tile of exp(l - tile max)
   int32_t* status = nullptr;       // first device-side error of the stream, 0 = none
   void* gemm_state = nullptr;      // tensor-map cache of the tensor-core GEMM
   void* gen_buf = nullptr;         // work buffers of laser_generate, kept between calls (in `owned`)
@@ -39,7 +45,7 @@ struct laser_model {
 namespace laser {
 
 // What the GEMM does with a finished 128-feature x NT-row accumulator tile.
-enum { EPI_PLAIN = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_QKV = 3 };
+enum { EPI_PLAIN = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_QKV = 3, EPI_VERDICT = 4 };
 
 struct GemmEpilogue {
   int R_rows = 0;                    // rows the activation / output buffers really have
@@ -51,6 +57,15 @@ struct GemmEpilogue {
   // EPI_PLAIN: out[r][n] = scale * acc (fp32), rows < R_store
   float* out = nullptr;
   int ldo = 0, R_store = 0;
+  // EPI_VERDICT: the scaled row is a row of logits; per (row, weight tile) the tile's top_n largest of them with
+  // their ids (ties: smaller id first), the sum of exp(l - tile max) when tile_sum is given, and the logit of the
+  // row's draft token from the tile that holds it; `out` may be null (logits never stored)
+  const int32_t* row_draft = nullptr;
+  float* draft_logit = nullptr;
+  float4* top_val = nullptr;
+  int4* top_idx = nullptr;
+  float* tile_sum = nullptr;
+  int top_n = 0, n_vtiles = 0;
   // EPI_RESID: resid[r][n] += acc; xb = bf16(resid * gain_next); sumsq_out[tile][r]
   float* resid = nullptr;
   __nv_bfloat16* xb = nullptr;
@@ -102,5 +117,12 @@ laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const
 // B * Rs inside the model's row workspace); K and V of the rows go to the cache, lengths are not changed.
 laser_status prefill_rows(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
                           const int32_t* n_rows, int32_t B, int32_t Rs, cudaStream_t stream);
+
+
+// The verify forward with acceptance fused into the LM head: per (row, 128-token vocabulary tile) the tile's
+// top_n (1..4) largest logits and ids, with `sums` the tile's sum of exp(l - tile max), and per row the logit of
+// its draft token, all in the model's buffers; logits (may be null) are stored only when given.
+laser_status verify_fused(laser_model* m, laser_kv* kv, const int32_t* seq_ids, const int32_t* tokens,
+                          const int32_t* n_rows, int32_t B, float* logits, int top_n, bool sums, cudaStream_t stream);
 
 }  // namespace laser

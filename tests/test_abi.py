@@ -24,7 +24,7 @@ def test_binding_structs_match_header_and_names():
     ensure_built()
     from paper_2408_05676_b200 import binding as L
     assert ctypes.sizeof(L.ModelCfg) == 12 * 4
-    assert ctypes.sizeof(L.Params) == 12 * 4
+    assert ctypes.sizeof(L.Params) == 13 * 4
     assert ctypes.sizeof(L.Weights) == 12 * 8
     assert ctypes.sizeof(L.Stats) == 6 * 8 + 5 * 4 + 4
     header = open(os.path.join(ROOT, "include", "laser.h")).read()
