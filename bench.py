@@ -218,6 +218,12 @@ def run_ours(args):
         L.verify_step(model, kv, seq_ids, tokens, n_rows, logits)
         L.accept_commit(kv, seq_ids, logits, tokens, n_rows, prm, out=outs)
 
+    def step_fused(prm):     # the same step with acceptance fused into the LM head: no logits are stored
+        L.kv_set_len_dev(kv, lens)
+        L.draft(pool, d_tails, d_tl, d_gid, prm, draft, dlen, mn)
+        L.make_rows(d_last, draft, dlen, K, tokens, n_rows)
+        L.verify_accept(model, kv, seq_ids, tokens, n_rows, prm, commit=True, out=outs)
+
     strict = L.make_params(K=K, n_min=1, n_max=N_MAX, max_occ=64, mode=L.MODE_STRICT)
     step(strict)
     torch.cuda.synchronize()
@@ -233,7 +239,7 @@ def run_ours(args):
     def barrier():
         replicas.barrier(dist, torch.device(dev))
 
-    def timed(prm, steps, warmup, sample_clocks=False):
+    def timed(prm, steps, warmup, sample_clocks=False, step=step):
         for _ in range(warmup):
             step(prm)
         barrier()
@@ -257,6 +263,10 @@ def run_ours(args):
 
     res = {name: timed(prm, args.steps, args.warmup, sample_clocks=(name == "strict")) for name, prm in modes.items()}
     main = res["strict"]
+    step(strict)
+    unfused_out = [t.clone() for t in outs]
+    res["strict_fused_lm_head"] = timed(strict, args.steps, args.warmup, step=step_fused)
+    assert all(bool((a == b).all()) for a, b in zip(unfused_out, outs)), "fused acceptance differs from the two-kernel path"
     step(strict)        # the rows of the headline step
 
     def verify_alone():

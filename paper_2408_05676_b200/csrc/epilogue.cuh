@@ -10,6 +10,7 @@ namespace laser {
 using bf16 = __nv_bfloat16;
 constexpr int kBM = 128;          // weight rows per tile (MMA M)
 constexpr int kBK = 64;           // K elements per stage = one 128-byte swizzle span of bf16
+constexpr int kVerdictRow = 132;  // floats per staged token row where one lane reads one row (16-byte reads of 8 lanes hit 8 bank groups)
 
 __device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
   __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
@@ -85,7 +86,7 @@ __device__ __forceinline__ float ordered_to_f32(uint32_t o) {
 // first top_n and its softmax probability without a row of logits ever being stored.  The reductions are warp-wide
 // integer max / min over order-preserving keys: exact, the same from run to run.
 __device__ __forceinline__ void epi_verdict(const GemmEpilogue& e, const LaneCtx& c, int r, bool live, int lane, float4 v,
-                                            float rstd, int N, int wt) {
+                                            float rstd, int N, int wt, int draft) {
   float x[4] = {v.x * rstd, v.y * rstd, v.z * rstd, v.w * rstd};
   live = live && r < e.R_store;
   if (e.out && live) {
@@ -102,8 +103,8 @@ __device__ __forceinline__ void epi_verdict(const GemmEpilogue& e, const LaneCtx
     if (x[i] == 0.f) x[i] = 0.f;                 // -0 and +0 are one value and must map to one key
     if (c.n + i >= N) x[i] = -INFINITY;          // beyond the vocabulary
   }
-  const int off = (live ? e.row_draft[r] : -1) - c.n;
-  if (off >= 0 && off < 4 && c.n + off < N) e.draft_logit[r] = off == 0 ? x[0] : off == 1 ? x[1] : off == 2 ? x[2] : x[3];
+  const int off = draft - c.n;          // `draft` is the row's draft token (-1: none), read before the tile was ready
+  if (live && draft >= 0 && off >= 0 && off < 4 && c.n + off < N) e.draft_logit[r] = off == 0 ? x[0] : off == 1 ? x[1] : off == 2 ? x[2] : x[3];
   float tv[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
   int ti[4] = {0x7fffffff, 0x7fffffff, 0x7fffffff, 0x7fffffff};
   uint32_t taken = 0;
@@ -132,6 +133,67 @@ __device__ __forceinline__ void epi_verdict(const GemmEpilogue& e, const LaneCtx
     const size_t at = size_t(r) * e.n_vtiles + wt;
     e.top_val[at] = make_float4(tv[0], tv[1], tv[2], tv[3]);
     e.top_idx[at] = make_int4(ti[0], ti[1], ti[2], ti[3]);
+    if (e.tile_sum) e.tile_sum[at] = s;
+  }
+}
+
+// The same per (row, vocabulary tile) record as epi_verdict, for a tile staged whole in this CTA's shared memory
+// (rows of kVerdictRow floats): one lane per token row walks the row's 128 logits in ascending token id, keeping
+// the TOPN largest in registers (a later equal logit never displaces an earlier one: smaller id first), then sums
+// exp(l - tile max) in a second walk where the rule has a probability.
+template <int TOPN>
+__device__ __forceinline__ void verdict_rows(const GemmEpilogue& e, uint32_t tile_smem, int NT, int r0, int n0t, int wt, int N,
+                                             int warp, int lane, const float* s_rstd, const int* s_draft, bool ok) {
+  const int nch = min(32, (N - n0t) >> 2);       // 16-byte chunks of the tile inside the vocabulary (N % 8 == 0)
+  for (int jb = warp * 32; jb < NT; jb += 6 * 32) {
+    const int j = jb + lane, r = r0 + j;
+    if (j >= NT) continue;
+    const bool live = ok && r < e.R_store;
+    const float rstd = s_rstd[j];
+    const uint32_t row = tile_smem + uint32_t(j) * (kVerdictRow * 4);
+    float tv[TOPN];
+    int ti[TOPN];
+#pragma unroll
+    for (int q = 0; q < TOPN; ++q) { tv[q] = -INFINITY; ti[q] = 0x7fffffff; }
+#pragma unroll 4
+    for (int c = 0; c < nch; ++c) {
+      float4 a;
+      asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w) : "r"(row + uint32_t(c) * 16));
+      const float x[4] = {a.x * rstd, a.y * rstd, a.z * rstd, a.w * rstd};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (x[i] > tv[TOPN - 1]) {
+          tv[TOPN - 1] = x[i]; ti[TOPN - 1] = n0t + 4 * c + i;
+#pragma unroll
+          for (int q = TOPN - 1; q > 0; --q)
+            if (tv[q] > tv[q - 1]) {
+              const float fv = tv[q]; tv[q] = tv[q - 1]; tv[q - 1] = fv;
+              const int fi = ti[q]; ti[q] = ti[q - 1]; ti[q - 1] = fi;
+            }
+        }
+      }
+    }
+    float s = 0.f;
+    if (e.tile_sum) {
+#pragma unroll 4
+      for (int c = 0; c < nch; ++c) {
+        float4 a;
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w) : "r"(row + uint32_t(c) * 16));
+        s += (__expf(a.x * rstd - tv[0]) + __expf(a.y * rstd - tv[0])) + (__expf(a.z * rstd - tv[0]) + __expf(a.w * rstd - tv[0]));
+      }
+    }
+    if (!live) continue;
+    const int off = s_draft[j] - n0t;
+    if (off >= 0 && off < 4 * nch) {
+      float dl;
+      asm volatile("ld.shared.f32 %0, [%1];" : "=f"(dl) : "r"(row + uint32_t(off) * 4));
+      e.draft_logit[r] = dl * rstd;
+    }
+    const size_t at = size_t(r) * e.n_vtiles + wt;
+    e.top_val[at] = make_float4(tv[0], TOPN > 1 ? tv[TOPN > 1 ? 1 : 0] : -INFINITY, TOPN > 2 ? tv[TOPN > 2 ? 2 : 0] : -INFINITY,
+                                TOPN > 3 ? tv[TOPN > 3 ? 3 : 0] : -INFINITY);
+    e.top_idx[at] = make_int4(ti[0], TOPN > 1 ? ti[TOPN > 1 ? 1 : 0] : 0x7fffffff, TOPN > 2 ? ti[TOPN > 2 ? 2 : 0] : 0x7fffffff,
+                              TOPN > 3 ? ti[TOPN > 3 ? 3 : 0] : 0x7fffffff);
     if (e.tile_sum) e.tile_sum[at] = s;
   }
 }

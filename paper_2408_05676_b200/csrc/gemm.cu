@@ -113,6 +113,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = tmem_slot;
+  // floats between consecutive token rows of the staged accumulator; the verdict epilogue reads one row per lane
+  // and pads the rows so that those reads spread over the banks
+  constexpr int kRow = EPI == EPI_VERDICT ? kVerdictRow : kBM;
 
   // gains of the next norm for the first weight tile: a weight, not a result of the kernel before, so
   // requested now, long before the epilogue uses it
@@ -136,12 +139,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 #pragma unroll
         for (int x = 0; x < 16; ++x) v0[x] = v1[x] = v2[x] = 0u;
       }
-      const uint32_t dst = dst0 + uint32_t(c) * (kBM * 4);
+      const uint32_t dst = dst0 + uint32_t(c) * (kRow * 4);
 #pragma unroll
       for (int x = 0; x < 16; ++x) {
-        if (c + x < NT) st_shared_f32(dst + x * (kBM * 4), __uint_as_float(v0[x]));
-        if (c + 16 + x < NT) st_shared_f32(dst + (16 + x) * (kBM * 4), __uint_as_float(v1[x]));
-        if (c + 32 + x < NT) st_shared_f32(dst + (32 + x) * (kBM * 4), __uint_as_float(v2[x]));
+        if (c + x < NT) st_shared_f32(dst + x * (kRow * 4), __uint_as_float(v0[x]));
+        if (c + 16 + x < NT) st_shared_f32(dst + (16 + x) * (kRow * 4), __uint_as_float(v1[x]));
+        if (c + 32 + x < NT) st_shared_f32(dst + (32 + x) * (kRow * 4), __uint_as_float(v2[x]));
       }
     }
   };
@@ -222,6 +225,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           for (int tt = 0; tt < e.sumsq_in_tiles; ++tt) ss += e.sumsq_in[size_t(tt) * e.sumsq_ld + r];
           rstd = rsqrtf(ss * e.inv_d + e.eps);
         }
+        if (EPI == EPI_VERDICT) pos = r < e.R_store ? e.row_draft[r] : -1;   // the row's draft token, in the slot of the position
         if (EPI == EPI_QKV) {
           pos = e.row_pos[r];
           if (pos >= 0) page = e.page_table[size_t(e.row_seq[r]) * e.pages_per_seq + (pos >> 4)];
@@ -265,7 +269,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   // (an odd tile count leaves the last group's second tile beyond the matrix: nothing to finish)
   const bool tile_valid = EPI == EPI_SWIGLU ? wt * 64 < e.f : n0t < N;
   if (!tile_valid) {
-  } else if ((EPI == EPI_SWIGLU || EPI == EPI_PLAIN || EPI == EPI_VERDICT) && splits == 1) {
+  } else if (EPI == EPI_VERDICT && splits == 1) {
+    // part 3, acceptance fused into the LM head: one lane per token row scans the row's 128 staged logits
+    if (e.out) {   // on request the logits are stored as well (the plain epilogue's stores)
+      for (int j = warp; j < NT; j += kTcThreads / 32) {
+        float4 a;
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w) : "r"(tiles + uint32_t((j * kRow + 4 * lane) * 4)));
+        epi_plain(e, lc, r0 + j, r0 + j < e.R_rows && !abort_flag, a, s_rstd[j], N);
+      }
+    }
+    const bool ok = !abort_flag;
+    if (e.top_n <= 1) verdict_rows<1>(e, tiles, NT, r0, n0t, wt, N, warp, lane, s_rstd, s_pos, ok);
+    else if (e.top_n == 2) verdict_rows<2>(e, tiles, NT, r0, n0t, wt, N, warp, lane, s_rstd, s_pos, ok);
+    else verdict_rows<4>(e, tiles, NT, r0, n0t, wt, N, warp, lane, s_rstd, s_pos, ok);
+  } else if ((EPI == EPI_SWIGLU || EPI == EPI_PLAIN) && splits == 1) {
     // part 3 without partial tiles to sum or operands to prefetch: all six warps finish rows,
     // in wide groups whose loads are issued first.
     constexpr int kWide = 12;
@@ -275,7 +292,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       for (int b = 0; b < kWide; ++b) {
         const int j = min(jb + b, NT - 1);
         asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
-                     : "=f"(acc[b].x), "=f"(acc[b].y), "=f"(acc[b].z), "=f"(acc[b].w) : "r"(tiles + uint32_t((j * kBM + 4 * lane) * 4)));
+                     : "=f"(acc[b].x), "=f"(acc[b].y), "=f"(acc[b].z), "=f"(acc[b].w) : "r"(tiles + uint32_t((j * kRow + 4 * lane) * 4)));
       }
 #pragma unroll
       for (int b = 0; b < kWide; ++b) {
@@ -283,7 +300,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const bool live = jb + b < NT && r < e.R_rows && !(abort_flag);
         const float rstd = s_rstd[j];
         if (EPI == EPI_PLAIN) epi_plain(e, lc, r, live, acc[b], rstd, N);
-        else if (EPI == EPI_VERDICT) epi_verdict(e, lc, r, live, lane, acc[b], rstd, N, wt);
         else epi_swiglu(e, r, live, wt * 64, lane, acc[b], rstd);
       }
     }
@@ -305,7 +321,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           const int jj = min(jb + b, own - 1);
 #pragma unroll
           for (int q = 0; q < S; ++q)
-            part[b][q] = ld_cluster_f4(rank_base[q] + uint32_t(((krank * slice + jj) * kBM + 4 * lane) * 4));
+            part[b][q] = ld_cluster_f4(rank_base[q] + uint32_t(((krank * slice + jj) * kRow + 4 * lane) * 4));
         }
 #pragma unroll
         for (int b = 0; b < RB; ++b) fetch_operands(jb + b, g0[b], g1[b]);
@@ -319,7 +335,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           const bool live = jj < own && r < e.R_rows && !abort_flag;   // the last token tile may overhang the buffers
           const float rstd = s_rstd[j];
           if (EPI == EPI_PLAIN) epi_plain(e, lc, r, live, acc, rstd, N);
-          else if (EPI == EPI_VERDICT) epi_verdict(e, lc, r, live, lane, acc, rstd, N, wt);
+          else if (EPI == EPI_VERDICT) epi_verdict(e, lc, r, live, lane, acc, rstd, N, wt, s_pos[j]);
           else if (EPI == EPI_RESID) epi_resid(e, lc, r, live, lane, acc, N, wt, g0[b], gain4);
           else if (EPI == EPI_SWIGLU) epi_swiglu(e, r, live, wt * 64, lane, acc, rstd);
           else epi_qkv(e, lc, r, live, acc, rstd, s_pos[j], s_page[j], g0[b], g1[b]);
@@ -384,7 +400,7 @@ TcShape tc_shape(int R_pad, int mt = 1) {
   s.tmem_cols = 32;
   while (s.tmem_cols < s.NT) s.tmem_cols <<= 1;
   if (mt == 2) s.tmem_cols = 2 * kAccCols;
-  s.smem = std::max(size_t(s.stages) * stage_bytes, size_t(s.NT) * kBM * 4) + 1024;
+  s.smem = std::max(size_t(s.stages) * stage_bytes, size_t(s.NT) * kVerdictRow * 4) + 1024;
   return s;
 }
 

@@ -1,5 +1,6 @@
 """Device time of laser_verify_step alone for a model shape and step size, with the split into dense
-contractions and attention (the library's per-launch event brackets).
+contractions and attention (the library's per-launch event brackets), and of the step with acceptance after
+the forward against acceptance fused into the LM head.
 
     python -m paper_2408_05676_b200.step_probe [--shape 7b|13b|tiny] [--layers L] [--batch B] [--draft K]
                                                [--ctx N] [--steps S]
@@ -49,6 +50,31 @@ def run(shape: str, layers: int, batch: int, draft: int, ctx: int, steps: int) -
         L.verify_step(model, kv, ids, tokens, n_rows, logits)
     e1.record()
     torch.cuda.synchronize()
+    # acceptance after the forward (logits stored, two more passes over them) against acceptance fused into the
+    # LM head (no logits), strict rule, alternating so that clock drift hits both alike
+    prm = L.make_params(K=draft, mode=L.MODE_STRICT)
+    outs = (torch.empty(batch, dtype=torch.int32, device=dev), torch.empty(batch, draft + 1, dtype=torch.int32, device=dev),
+            torch.empty(batch, dtype=torch.int32, device=dev))
+
+    def two_kernels():
+        L.verify_step(model, kv, ids, tokens, n_rows, logits)
+        L.accept_commit(None, None, logits, tokens, n_rows, prm, out=outs)
+
+    def fused():
+        L.verify_accept(model, kv, ids, tokens, n_rows, prm, commit=False, out=outs)
+
+    ab = {"two": 0.0, "fused": 0.0}
+    for rnd in range(4):
+        for name, fn in (("two", two_kernels), ("fused", fused)) if rnd % 2 == 0 else (("fused", fused), ("two", two_kernels)):
+            fn()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record()
+            for _ in range(steps):
+                fn()
+            a1.record()
+            torch.cuda.synchronize()
+            ab[name] += a0.elapsed_time(a1) / steps / 4
+    L.check(model)
     L.profile_enable(model, True)
     for _ in range(2):
         L.verify_step(model, kv, ids, tokens, n_rows, logits)
@@ -63,6 +89,7 @@ def run(shape: str, layers: int, batch: int, draft: int, ctx: int, steps: int) -
     flops = float(rows) * weight_bytes
     kv_bytes = batch * ctx * layers * 2 * dkv * 2
     return dict(shape=shape, layers=layers, batch=batch, rows=rows, ctx=ctx, ms_per_step=e0.elapsed_time(e1) / steps,
+                verify_then_accept_ms=ab["two"], verify_accept_fused_ms=ab["fused"],
                 contractions_ms=gemm_ms / 2, contraction_launches=n_gemm // 2, attention_ms=attn_ms / 2,
                 attention_launches=n_attn // 2, weight_gb=weight_bytes / 1e9, kv_gb=kv_bytes / 1e9,
                 contraction_tflops=flops / (gemm_ms / 2) * 1e-9, weight_gbs=weight_bytes / (gemm_ms / 2) * 1e-6,
