@@ -1,7 +1,7 @@
 // Fused epilogues of the dense contractions of the verify forward: what happens to a finished
-// 128-feature x token-row accumulator tile.  Shared by the per-matrix kernel and the persistent
-// whole-step kernel.  Values that another SM may have written during the running kernel (the
-// residual stream) are read past L1.
+// 128-feature x token-row accumulator tile (RMSNorm scale, rotary embedding + cache write, residual
+// add + next norm's operand, SwiGLU, logits, or the acceptance rule's per-tile record).  Values that
+// another SM may have written during the running kernel (the residual stream) are read past L1.
 #pragma once
 #include "model.cuh"
 

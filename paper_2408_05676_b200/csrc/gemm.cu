@@ -36,6 +36,10 @@ namespace {
 constexpr int kTcThreads = 192;
 constexpr int kMaxStages = 6;
 constexpr int kMaxNT = 192;       // token rows per tile: accumulator staging must fit shared memory
+#ifndef LASER_WIDE_NT
+#define LASER_WIDE_NT 256
+#endif
+constexpr int kMaxNTWide = LASER_WIDE_NT;   // ... with two weight tiles per CTA (one CTA per SM); 256 = the largest MMA N
 constexpr int kSmemBudget = 110 * 1024;  // shared memory of one CTA: two CTAs per SM
 constexpr int kSmemBudgetWide = 200 * 1024;  // with two weight tiles per CTA: one CTA per SM
 constexpr int kAccCols = 256;     // tensor-memory columns between the accumulators of a CTA's weight tiles
@@ -69,8 +73,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_bar;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  __shared__ float s_rstd[kMaxNT];
-  __shared__ int s_pos[kMaxNT], s_page[kMaxNT];
+  __shared__ float s_rstd[MT == 1 ? kMaxNT : kMaxNTWide];
+  __shared__ int s_pos[MT == 1 ? kMaxNT : kMaxNTWide], s_page[MT == 1 ? kMaxNT : kMaxNTWide];
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its prologue
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
@@ -390,10 +394,10 @@ laser_status tensor_map(GemmState* st, const void* ptr, int rows, int cols, int 
 
 struct TcShape { int n_ttiles, NT, stages, tmem_cols; size_t smem; };
 
-// mt = weight tiles per CTA (1 or 2)
-TcShape tc_shape(int R_pad, int mt = 1) {
+// mt = weight tiles per CTA (1 or 2); max_nt = most token rows per tile
+TcShape tc_shape(int R_pad, int mt = 1, int max_nt = kMaxNT) {
   TcShape s;
-  s.n_ttiles = ceil_div(R_pad, kMaxNT);
+  s.n_ttiles = ceil_div(R_pad, max_nt);
   s.NT = ceil_div(ceil_div(R_pad, s.n_ttiles), 16) * 16;
   const int stage_bytes = mt * kBM * 128 + s.NT * 128;
   s.stages = std::max(2, std::min(kMaxStages, (mt == 1 ? kSmemBudget : kSmemBudgetWide) / stage_bytes));
@@ -474,7 +478,15 @@ laser_status gemm_fused(laser_model* m, const __nv_bfloat16* A, const __nv_bfloa
   // (where the halved CTA count still gives every SM one)
   const int n_tt = tc_shape(R_pad).n_ttiles;
   const int mt = (n_tt > 1 && splits == 1 && ceil_div(n_wtiles, 2) * n_tt >= 148) ? 2 : 1;
-  const TcShape sh = tc_shape(R_pad, mt);
+  TcShape sh = tc_shape(R_pad, mt);
+  if (mt == 2) {
+    // Token tiles of up to 256 rows (the largest MMA N) re-read the weights from L2 fewer times, but make fewer,
+    // longer CTAs: taken where they do not cost more in whole waves of CTAs over the SMs (a CTA's time goes with
+    // the bytes it stages per K block: 256 weight rows + NT token rows).
+    const TcShape wide = tc_shape(R_pad, 2, kMaxNTWide);
+    auto cost = [&](const TcShape& t) { return ceil_div(ceil_div(n_wtiles, 2) * t.n_ttiles, 148) * (256 + t.NT); };
+    if (cost(wide) < cost(sh)) sh = wide;
+  }
   const CUtensorMap *tw = nullptr, *ta = nullptr;
   LASER_TRY(tensor_map(st, W, N, K, 64, &tw));
   LASER_TRY(tensor_map(st, A, m->R_pad, K, sh.NT, &ta));
