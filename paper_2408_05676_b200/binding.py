@@ -34,7 +34,7 @@ class ModelCfg(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "n_kv_heads", "head_dim",
                                           "d_ffn", "vocab")] + \
                [("rms_eps", C.c_float), ("rope_theta", C.c_float)] + \
-               [(n, C.c_int32) for n in ("page_size", "max_draft", "max_batch")]
+               [(n, C.c_int32) for n in ("page_size", "max_draft", "max_batch", "precise")]
 
 
 class Weights(C.Structure):
@@ -236,7 +236,7 @@ def model_create(cfg: Dict, W: Dict, max_batch: int) -> Model:
     """cfg: dict as synth.model_cfg; W: dict of CUDA bf16 tensors as synth.make_weights."""
     c = ModelCfg(cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["n_kv_heads"], cfg["head_dim"],
                  cfg["d_ffn"], cfg["vocab"], cfg["rms_eps"], cfg["rope_theta"], cfg["page_size"],
-                 cfg["max_draft"], max_batch)
+                 cfg["max_draft"], max_batch, int(cfg.get("precise", 0)))
     L = cfg["n_layers"]
 
     def arr(name):

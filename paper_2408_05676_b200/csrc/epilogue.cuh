@@ -17,6 +17,15 @@ __device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) 
   return make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
 }
 
+// hi = bf16(x), lo = bf16(x - hi): the pair carries about 16 significant bits of x
+__device__ __forceinline__ void split4_bf16(float a, float b, float c, float d, uint2& hi, uint2& lo) {
+  const __nv_bfloat162 h01 = __floats2bfloat162_rn(a, b), h23 = __floats2bfloat162_rn(c, d);
+  const __nv_bfloat162 l01 = __floats2bfloat162_rn(a - __low2float(h01), b - __high2float(h01));
+  const __nv_bfloat162 l23 = __floats2bfloat162_rn(c - __low2float(h23), d - __high2float(h23));
+  hi = make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
+  lo = make_uint2(*reinterpret_cast<const uint32_t*>(&l01), *reinterpret_cast<const uint32_t*>(&l23));
+}
+
 // ---- fused epilogues: one warp finishes one token row r of a 128-feature tile; lane l holds
 //      features n0 + 4l .. 4l+3 in v.  What depends on the feature alone is worked out once per
 //      thread (LaneCtx); rows are finished without branches (`live` predicates the stores), so
@@ -206,8 +215,15 @@ __device__ __forceinline__ void epi_resid(const GemmEpilogue& e, const LaneCtx& 
   if (live && c.in_range) {
     *reinterpret_cast<float4*>(e.resid + size_t(r) * N + c.n) = x;
     const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&g2.x), g23 = *reinterpret_cast<const __nv_bfloat162*>(&g2.y);
-    *reinterpret_cast<uint2*>(e.xb + size_t(r) * N + c.n) =
-        pack4_bf16(x.x * __low2float(g01), x.y * __high2float(g01), x.z * __low2float(g23), x.w * __high2float(g23));
+    const float y0 = x.x * __low2float(g01), y1 = x.y * __high2float(g01), y2 = x.z * __low2float(g23), y3 = x.w * __high2float(g23);
+    if (e.out_split) {
+      uint2 hi, lo;
+      split4_bf16(y0, y1, y2, y3, hi, lo);
+      *reinterpret_cast<uint2*>(e.xb + size_t(r) * (2 * N) + c.n) = hi;
+      *reinterpret_cast<uint2*>(e.xb + size_t(r) * (2 * N) + N + c.n) = lo;
+    } else {
+      *reinterpret_cast<uint2*>(e.xb + size_t(r) * N + c.n) = pack4_bf16(y0, y1, y2, y3);
+    }
     ss = x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
   }
   for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
@@ -225,8 +241,15 @@ __device__ __forceinline__ void epi_swiglu(const GemmEpilogue& e, int r, bool li
   const float u0 = (lo ? t0 : v.z) * rstd, u1 = (lo ? t1 : v.w) * rstd;
   const int fidx = f0 + 4 * (lane & 15) + (lo ? 0 : 2);
   if (live && fidx < e.f) {  // f is a multiple of 8 (checked on the host)
-    const __nv_bfloat162 a = __floats2bfloat162_rn(__fdividef(g0, 1.f + __expf(-g0)) * u0, __fdividef(g1, 1.f + __expf(-g1)) * u1);
-    *reinterpret_cast<__nv_bfloat162*>(e.act + size_t(r) * e.f + fidx) = a;
+    const float a0 = __fdividef(g0, 1.f + __expf(-g0)) * u0, a1 = __fdividef(g1, 1.f + __expf(-g1)) * u1;
+    const __nv_bfloat162 a = __floats2bfloat162_rn(a0, a1);
+    if (e.out_split) {
+      *reinterpret_cast<__nv_bfloat162*>(e.act + size_t(r) * (2 * e.f) + fidx) = a;
+      *reinterpret_cast<__nv_bfloat162*>(e.act + size_t(r) * (2 * e.f) + e.f + fidx) =
+          __floats2bfloat162_rn(a0 - __low2float(a), a1 - __high2float(a));
+    } else {
+      *reinterpret_cast<__nv_bfloat162*>(e.act + size_t(r) * e.f + fidx) = a;
+    }
   }
 }
 
@@ -247,7 +270,8 @@ __device__ __forceinline__ void epi_qkv(const GemmEpilogue& e, const LaneCtx& c,
   if (!live || !c.in_range) return;
   if (c.kind == 0) {
     if (pos < 0) y = make_float4(0.f, 0.f, 0.f, 0.f);
-    *reinterpret_cast<uint2*>(e.q + size_t(r) * (e.H * e.dh) + c.n) = pack4_bf16(y.x, y.y, y.z, y.w);
+    if (e.qf) *reinterpret_cast<float4*>(e.qf + size_t(r) * (e.H * e.dh) + c.n) = y;
+    else *reinterpret_cast<uint2*>(e.q + size_t(r) * (e.H * e.dh) + c.n) = pack4_bf16(y.x, y.y, y.z, y.w);
   } else if (pos >= 0) {
     bf16* dst = e.pages_layer + size_t(page) * e.page_elems + c.kv_off + size_t(pos & 15) * e.dh;
     *reinterpret_cast<uint2*>(dst) = pack4_bf16(y.x, y.y, y.z, y.w);

@@ -85,6 +85,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const int r0 = ttile * NT, n0 = wtile * kBM * MT;           // wtile counts groups of MT weight tiles
   const int kb0 = krank * kb_per_split;
   const int nkb = max(0, min(kb_per_split, total_kb - kb0));
+  // Activations given as hi + lo bf16 pairs ([hi | lo] side by side in a row, lo starting at column a_lo_off): K
+  // block g multiplies weight block g / 2 with the hi (g even) or lo (g odd) part, into the same accumulator.
+  const int wshift = e.a_lo_off ? 1 : 0;
   const int slice = (NT + splits - 1) / splits;            // token columns finished by one CTA of the cluster
   const int own = max(0, min(slice, NT - krank * slice));
 
@@ -99,12 +102,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const uint64_t w_policy0 = make_policy_evict_first();
     for (int kb = 0; kb < min(stages, nkb); ++kb) {
       const uint32_t bar = smem_u32(&full_bar[kb]), dst = tiles + uint32_t(kb) * stage_bytes;
+      const int wk = ((kb0 + kb) >> wshift) * kBK;
       mbar_expect_tx(bar, stage_bytes);
 #pragma unroll
       for (int t = 0; t < MT; ++t) {
         const int T = wtile * MT + t;
-        tma_load_2d_hint(dst + t * w_bytes, &tmW, (kb0 + kb) * kBK, EPI == EPI_SWIGLU ? T * 64 : T * kBM, bar, w_policy0);
-        tma_load_2d_hint(dst + t * w_bytes + w_bytes / 2, &tmW, (kb0 + kb) * kBK, EPI == EPI_SWIGLU ? e.f + T * 64 : T * kBM + 64, bar, w_policy0);
+        tma_load_2d_hint(dst + t * w_bytes, &tmW, wk, EPI == EPI_SWIGLU ? T * 64 : T * kBM, bar, w_policy0);
+        tma_load_2d_hint(dst + t * w_bytes + w_bytes / 2, &tmW, wk, EPI == EPI_SWIGLU ? e.f + T * 64 : T * kBM + 64, bar, w_policy0);
       }
     }
     tma_prefetch_map(&tmA);
@@ -162,7 +166,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       auto load = [&](uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar, uint64_t pol) { tma_load_2d_hint(dst, tm, x, y, bar, pol); };
       auto expect = [&](int s) { mbar_expect_tx(smem_u32(&full_bar[s]), stage_bytes); };
       auto load_w = [&](int kb) {
-        const int s = kb % stages, k = (kb0 + kb) * kBK;
+        const int s = kb % stages, k = ((kb0 + kb) >> wshift) * kBK;
         const uint32_t dst = tiles + uint32_t(s) * stage_bytes, bar = full0 + uint32_t(s) * 8;
 #pragma unroll
         for (int t = 0; t < MT; ++t) {
@@ -173,7 +177,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       };
       auto load_a = [&](int kb) {
         const int s = kb % stages;
-        load(tiles + uint32_t(s) * stage_bytes + MT * w_bytes, &tmA, (kb0 + kb) * kBK, r0, full0 + uint32_t(s) * 8, a_policy);
+        const int g = kb0 + kb;
+        load(tiles + uint32_t(s) * stage_bytes + MT * w_bytes, &tmA, (g & wshift) * e.a_lo_off + (g >> wshift) * kBK, r0,
+             full0 + uint32_t(s) * 8, a_policy);
       };
       // The ring was filled with weight tiles at the start of the kernel (they do not depend on the
       // kernel before this one); only now wait for that kernel's results (the activations).
@@ -489,8 +495,8 @@ laser_status gemm_fused(laser_model* m, const __nv_bfloat16* A, const __nv_bfloa
   }
   const CUtensorMap *tw = nullptr, *ta = nullptr;
   LASER_TRY(tensor_map(st, W, N, K, 64, &tw));
-  LASER_TRY(tensor_map(st, A, m->R_pad, K, sh.NT, &ta));
-  const int total_kb = ceil_div(K, kBK), kbps = ceil_div(total_kb, splits);
+  LASER_TRY(tensor_map(st, A, m->R_pad, e.a_lo_off ? 2 * K : K, sh.NT, &ta));
+  const int total_kb = ceil_div(K, kBK) * (e.a_lo_off ? 2 : 1), kbps = ceil_div(total_kb, splits);
   const int n_groups = ceil_div(n_wtiles, mt);     // grid rows: groups of mt weight tiles
 #define LASER_GEMM_LAUNCH(E)                                                                                            \
   do {                                                                                                                  \

@@ -91,7 +91,8 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 __global__ void __launch_bounds__(256)
 embed_kernel(const int32_t* __restrict__ tokens, int R, int d, int vocab, const bf16* __restrict__ emb,
              const bf16* __restrict__ gain, float* __restrict__ resid, bf16* __restrict__ xb,
-             float* __restrict__ sumsq, const int32_t* __restrict__ n_rows, int Rs, int32_t* __restrict__ row_draft) {
+             float* __restrict__ sumsq, const int32_t* __restrict__ n_rows, int Rs, int32_t* __restrict__ row_draft,
+             int split) {
   __shared__ float red[8];
   const int r = blockIdx.x;
   const int tok = r < R ? tokens[r] : -1;
@@ -105,7 +106,14 @@ embed_kernel(const int32_t* __restrict__ tokens, int R, int d, int vocab, const 
   for (int j = threadIdx.x; j < d; j += blockDim.x) {
     const float x = ok ? __bfloat162float(emb[size_t(tok) * d + j]) : 0.f;
     resid[size_t(r) * d + j] = x;
-    xb[size_t(r) * d + j] = __float2bfloat16(x * __bfloat162float(gain[j]));
+    const float y = x * __bfloat162float(gain[j]);
+    const bf16 hi = __float2bfloat16(y);
+    if (split) {   // operand as a hi + lo pair: [hi | lo] in a row of 2 d
+      xb[size_t(r) * (2 * d) + j] = hi;
+      xb[size_t(r) * (2 * d) + d + j] = __float2bfloat16(y - __bfloat162float(hi));
+    } else {
+      xb[size_t(r) * d + j] = hi;
+    }
     ss += x * x;
   }
   ss = block_sum(ss, red);
@@ -115,8 +123,9 @@ embed_kernel(const int32_t* __restrict__ tokens, int R, int d, int vocab, const 
 // Causal attention of the step's rows over the paged cache: grid (sequence, head).
 // Scores of one row go to shared memory, softmax in fp32, then thread d accumulates
 // sum_j p_j V[j][d].
+// qf (optional): the queries in fp32 instead of q; out_split: the output as hi + lo bf16 pairs, rows of 2 H dh.
 __global__ void __launch_bounds__(128)
-attention_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ seq_ids,
+attention_kernel(const bf16* __restrict__ q, const float* __restrict__ qf, int out_split, const int32_t* __restrict__ seq_ids,
                  const int32_t* __restrict__ row_ctx, const int32_t* __restrict__ row_n, int Rs, int H,
                  int Hkv, int dh, const int32_t* __restrict__ page_table, int pages_per_seq,
                  const bf16* __restrict__ pages_layer, size_t page_elems, bf16* __restrict__ out,
@@ -132,13 +141,18 @@ attention_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ seq_ids
   const float scale = rsqrtf(float(dh));
   for (int i = 0; i < Rs; ++i) {
     const size_t r = size_t(b) * Rs + i;
-    bf16* o = out + r * H * dh + size_t(h) * dh;
+    bf16* o = out + r * H * dh * (out_split ? 2 : 1) + size_t(h) * dh;
+    bf16* o_lo = o + size_t(H) * dh;
     if (i >= nr) {
-      for (int d = tid; d < dh; d += 128) o[d] = __float2bfloat16(0.f);
+      for (int d = tid; d < dh; d += 128) {
+        o[d] = __float2bfloat16(0.f);
+        if (out_split) o_lo[d] = __float2bfloat16(0.f);
+      }
       continue;
     }
     __syncthreads();
-    for (int d = tid; d < dh; d += 128) s_q[d] = __bfloat162float(q[r * H * dh + size_t(h) * dh + d]) * scale;
+    for (int d = tid; d < dh; d += 128)
+      s_q[d] = (qf ? qf[r * H * dh + size_t(h) * dh + d] : __bfloat162float(q[r * H * dh + size_t(h) * dh + d])) * scale;
     __syncthreads();
     // chain: the cache and rows 0..i; token tree: the cache and the rows of the mask
     const int n = row_mask ? ctx + nr : ctx + i + 1;
@@ -178,7 +192,9 @@ attention_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ seq_ids
         const bf16* vp = pages_layer + size_t(pt[j / 16]) * page_elems + (size_t(Hkv) + hk) * 16 * dh + size_t(j % 16) * dh;
         acc += s_sc[j] * __bfloat162float(vp[d]);
       }
-      o[d] = __float2bfloat16(acc / sum);
+      const float y = acc / sum;
+      o[d] = __float2bfloat16(y);
+      if (out_split) o_lo[d] = __float2bfloat16(y - __bfloat162float(o[d]));
     }
   }
 }
@@ -315,10 +331,13 @@ LASER_API laser_status laser_model_create(const laser_model_cfg* cfg, const lase
   }
   const size_t Rp = size_t(m->R_pad);
   LASER_TRY(model_alloc(m, &m->resid, Rp * d));
-  LASER_TRY(model_alloc(m, &m->xn, Rp * d));
+  m->precise = cfg->precise != 0;
+  const size_t pair = m->precise ? 2 : 1;     // hi + lo parts side by side in a row
+  LASER_TRY(model_alloc(m, &m->xn, Rp * d * pair));
   LASER_TRY(model_alloc(m, &m->q, Rp * m->dq));
-  LASER_TRY(model_alloc(m, &m->attn, Rp * m->dq));
-  LASER_TRY(model_alloc(m, &m->act, Rp * f));
+  if (m->precise) LASER_TRY(model_alloc(m, &m->qf, Rp * m->dq));
+  LASER_TRY(model_alloc(m, &m->attn, Rp * m->dq * pair));
+  LASER_TRY(model_alloc(m, &m->act, Rp * f * pair));
   LASER_TRY(model_alloc(m, &m->sumsq, size_t(ceil_div(d, 128)) * Rp));
   LASER_TRY(model_alloc(m, &m->rope, Rp * (cfg->head_dim / 2) * 2));
   LASER_TRY(model_alloc(m, &m->row_pos, Rp));
@@ -522,9 +541,9 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
                                           m->rope, m->status);
   const __nv_bfloat16* first_gain = c.n_layers > 0 ? m->attn_norm[0] : m->final_norm;
   embed_kernel<<<m->R_pad, 256, 0, stream>>>(tokens, R, d, c.vocab, m->tok_emb, first_gain, m->resid, m->xn, m->sumsq, n_rows, Rs,
-                                             fused ? m->row_draft : nullptr);
+                                             fused ? m->row_draft : nullptr, m->precise ? 1 : 0);
   count_launch(2);
-  const bool use_tma_attn = attention_tma_supported(m, kv);
+  const bool use_tma_attn = !m->precise && attention_tma_supported(m, kv);   // precise: fp32 queries and probabilities
   const size_t attn_smem = (size_t(dh) + size_t(capacity) + 8) * sizeof(float);
   if (!use_tma_attn && attn_smem > 48 * 1024) {
     LASER_REQUIRE(attn_smem <= 200 * 1024, "KV capacity of %d tokens per sequence exceeds the attention kernel's limit", capacity);
@@ -536,6 +555,7 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
   base.sumsq_ld = m->R_pad;
   base.inv_d = 1.f / float(d);
   base.eps = c.rms_eps;
+  base.out_split = m->precise ? 1 : 0;
   int norm_tiles = 1;  // tile planes holding the sums of squares of the current residual
   for (int l = 0; l < c.n_layers; ++l) {
     __nv_bfloat16* pages_l = kv->pages + size_t(l) * kv->layer_elems();
@@ -545,6 +565,7 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
       e.q = m->q; e.pages_layer = pages_l; e.page_elems = kv->page_elems(); e.page_table = kv->page_table;
       e.pages_per_seq = kv->pages_per_seq; e.row_pos = m->row_pos; e.row_seq = m->row_seq; e.rope = m->rope;
       e.H = H; e.Hkv = Hkv; e.dh = dh;
+      if (m->precise) { e.a_lo_off = d; e.qf = m->qf; }
       ProfScope ps(m, 0, stream);
       LASER_TRY(gemm_fused(m, m->xn, m->wqkv[l], Rp, m->dqkv, d, EPI_QKV, e, stream));
     }
@@ -553,7 +574,7 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
       if (use_tma_attn) {
         LASER_TRY(attention_tma_launch(m, kv, l, seq_ids, B, Rs, tree, stream));
       } else {
-        attention_kernel<<<dim3(B, H), 128, attn_smem, stream>>>(m->q, seq_ids, m->row_ctx, m->row_n, Rs, H, Hkv, dh,
+        attention_kernel<<<dim3(B, H), 128, attn_smem, stream>>>(m->q, m->qf, m->precise ? 1 : 0, seq_ids, m->row_ctx, m->row_n, Rs, H, Hkv, dh,
                                                                 kv->page_table, kv->pages_per_seq, pages_l,
                                                                 kv->page_elems(), m->attn, tree ? m->row_mask : nullptr);
         count_launch();
@@ -562,6 +583,7 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
     {  // output projection; residual add; operand and statistics of the FFN norm
       GemmEpilogue e = base;
       e.resid = m->resid; e.xb = m->xn; e.gain_next = m->ffn_norm[l]; e.sumsq_out = m->sumsq;
+      if (m->precise) e.a_lo_off = m->dq;
       ProfScope ps(m, 0, stream);
       LASER_TRY(gemm_fused(m, m->attn, m->wo[l], Rp, d, m->dq, EPI_RESID, e, stream));
     }
@@ -569,6 +591,7 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
       GemmEpilogue e = base;
       e.sumsq_in = m->sumsq; e.sumsq_in_tiles = d_tiles;
       e.act = m->act; e.f = f;
+      if (m->precise) e.a_lo_off = d;
       ProfScope ps(m, 0, stream);
       LASER_TRY(gemm_fused(m, m->xn, m->wgu[l], Rp, 2 * f, d, EPI_SWIGLU, e, stream));
     }
@@ -576,6 +599,7 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
       GemmEpilogue e = base;
       e.resid = m->resid; e.xb = m->xn; e.sumsq_out = m->sumsq;
       e.gain_next = l + 1 < c.n_layers ? m->attn_norm[l + 1] : m->final_norm;
+      if (m->precise) e.a_lo_off = f;
       ProfScope ps(m, 0, stream);
       LASER_TRY(gemm_fused(m, m->act, m->wdown[l], Rp, d, f, EPI_RESID, e, stream));
     }
@@ -585,6 +609,7 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
     GemmEpilogue e = base;
     e.sumsq_in = m->sumsq; e.sumsq_in_tiles = norm_tiles;
     e.out = logits; e.ldo = c.vocab; e.R_store = R;
+    if (m->precise) e.a_lo_off = d;
     if (fused) {   // ... or into what the acceptance rule needs of every (row, vocabulary tile)
       e.row_draft = m->row_draft; e.draft_logit = m->draft_logit; e.top_val = m->top_val; e.top_idx = m->top_idx;
       e.tile_sum = fused < 0 ? m->tile_sum : nullptr;

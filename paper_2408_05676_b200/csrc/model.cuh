@@ -17,6 +17,9 @@ struct laser_model {
   float* resid = nullptr;          // [R_pad, d] residual stream, fp32
   __nv_bfloat16* xn = nullptr;     // [R_pad, d] normalised activations (GEMM operand)
   __nv_bfloat16* q = nullptr;      // [R_pad, dq] rotated queries
+  float* qf = nullptr;             // [R_pad, dq] the same in fp32 (precise mode only)
+  bool precise = false;            // activations handed to the contractions as hi + lo bf16 pairs: xn, attn, act are
+                                   // [R_pad, 2 x width] with the lo parts in the second half of a row
   __nv_bfloat16* attn = nullptr;   // [R_pad, dq] attention output
   __nv_bfloat16* act = nullptr;    // [R_pad, f] SwiGLU output
   float* sumsq = nullptr;          // [ceil(d/128)][R_pad] per-tile sums of squares of the residual
@@ -49,6 +52,9 @@ enum { EPI_PLAIN = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_QKV = 3, EPI_VERDICT = 
 
 struct GemmEpilogue {
   int R_rows = 0;                    // rows the activation / output buffers really have
+  // Operands as hi + lo bf16 pairs (the precise mode): the A operand's rows are [hi | lo] with lo starting at column
+  // a_lo_off (0 = plain bf16 operand); out_split = the bf16 activations this epilogue writes (xb, act) are pairs too
+  int a_lo_off = 0, out_split = 0;
   // RMSNorm of the A operand, applied as a per-row scale of the result: the producer left
   // x * gain in bf16 and one sum of squares per (128-feature tile, row); null = no scale
   const float* sumsq_in = nullptr;
@@ -74,8 +80,9 @@ struct GemmEpilogue {
   // EPI_SWIGLU: W is [gate rows | up rows] (f each); act[r][j] = silu(gate_j) * up_j
   __nv_bfloat16* act = nullptr;
   int f = 0;
-  // EPI_QKV: rotary embedding, Q store, K/V page write
+  // EPI_QKV: rotary embedding, Q store (bf16, or fp32 into qf when given), K/V page write
   __nv_bfloat16* q = nullptr;
+  float* qf = nullptr;
   __nv_bfloat16* pages_layer = nullptr;
   size_t page_elems = 0;
   const int32_t* page_table = nullptr;

@@ -23,7 +23,7 @@ def test_library_exports_every_declared_symbol():
 def test_binding_structs_match_header_and_names():
     ensure_built()
     from paper_2408_05676_b200 import binding as L
-    assert ctypes.sizeof(L.ModelCfg) == 12 * 4
+    assert ctypes.sizeof(L.ModelCfg) == 13 * 4
     assert ctypes.sizeof(L.Params) == 13 * 4
     assert ctypes.sizeof(L.Weights) == 12 * 8
     assert ctypes.sizeof(L.Stats) == 6 * 8 + 5 * 4 + 4
