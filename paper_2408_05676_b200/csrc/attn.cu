@@ -40,9 +40,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int DH, int TPC>
-__global__ void __launch_bounds__(kAttnThreads, kCtasPerSm)
-attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restrict__ q,
+// PR (precise mode): the queries come in fp32 (qf) and enter the score MMA as hi + lo bf16 pairs, the probabilities
+// enter the value MMA as pairs as well, and the output is written as pairs ([hi | lo] rows of 2 H DH).
+template <int DH, int TPC, bool PR>
+__global__ void __launch_bounds__(kAttnThreads, PR ? 3 : kCtasPerSm)
+attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restrict__ q, const float* __restrict__ qf,
                   const int32_t* __restrict__ seq_ids, const int32_t* __restrict__ row_ctx,
                   const int32_t* __restrict__ row_n, int Rs, int H, int Hkv,
                   const int32_t* __restrict__ page_table, int pages_per_seq, int layer_row0,
@@ -70,12 +72,16 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
   const int cta_row0 = mt * 16 * TPC;              // first row of the CTA's tiles
   const int tile = TPC == 1 ? 0 : (warp & (TPC - 1)), pgrp = TPC == 1 ? warp : (warp / TPC);
   const int row0 = cta_row0 + tile * 16;           // first row of this warp's tile
-  bf16* obase = out + (size_t(b) * Rs + cta_row0) * H * DH + size_t(h) * DH;
+  constexpr int OW = PR ? 2 : 1;                    // output row = OW x H x DH elements
+  bf16* obase = out + (size_t(b) * Rs + cta_row0) * H * DH * OW + size_t(h) * DH;
   if (cta_row0 >= nr) {  // nothing active in these tiles: zero their rows
     asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int idx = tid; idx < 16 * TPC * DH; idx += kAttnThreads) {
       const int r = idx / DH, d = idx % DH;
-      if (cta_row0 + r < Rs) obase[size_t(r) * H * DH + d] = __float2bfloat16(0.f);
+      if (cta_row0 + r < Rs) {
+        obase[size_t(r) * H * DH * OW + d] = __float2bfloat16(0.f);
+        if (PR) obase[size_t(r) * H * DH * OW + size_t(H) * DH + d] = __float2bfloat16(0.f);
+      }
     }
     return;
   }
@@ -129,11 +135,30 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
   // ---- consumers ----
   asm volatile("griddepcontrol.wait;" ::: "memory");
   // Q tiles: rows of this sequence, zero beyond the active ones
+  constexpr int QLO = 16 * TPC * QLD;             // PR: the lo parts of the Q tile follow the hi parts
   for (int idx = tid; idx < 16 * TPC * (DH / 8); idx += kConsumers * 32) {
     const int r = idx / (DH / 8), c = idx % (DH / 8);
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (cta_row0 + r < nr) v = *reinterpret_cast<const uint4*>(q + (size_t(b) * Rs + cta_row0 + r) * H * DH + size_t(h) * DH + c * 8);
+    uint4 v = make_uint4(0, 0, 0, 0), vl = v;
+    if (cta_row0 + r < nr) {
+      const size_t at = (size_t(b) * Rs + cta_row0 + r) * H * DH + size_t(h) * DH + c * 8;
+      if (PR) {
+        const float4 f0 = *reinterpret_cast<const float4*>(qf + at), f1 = *reinterpret_cast<const float4*>(qf + at + 4);
+        const float f[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
+        uint32_t hi[4], lo[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+          const __nv_bfloat162 hh = __floats2bfloat162_rn(f[2 * x], f[2 * x + 1]);
+          hi[x] = *reinterpret_cast<const uint32_t*>(&hh);
+          lo[x] = pack_bf16(f[2 * x] - __low2float(hh), f[2 * x + 1] - __high2float(hh));
+        }
+        v = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        vl = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      } else {
+        v = *reinterpret_cast<const uint4*>(q + at);
+      }
+    }
     *reinterpret_cast<uint4*>(q_ptr + r * QLD + c * 8) = v;
+    if (PR) *reinterpret_cast<uint4*>(q_ptr + QLO + r * QLD + c * 8) = vl;
   }
   asm volatile("bar.sync 1, 128;" ::: "memory");
   const int g = lane >> 2, qd = lane & 3;
@@ -168,6 +193,11 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
         ldsm_x4(kb, kbase + (ks >> 2) * SUB + key * 128 + ((c ^ (key & 7)) << 4));
         mma16816(sc[0], qa, kb[0], kb[1]);
         mma16816(sc[1], qa, kb[2], kb[3]);
+        if (PR) {
+          ldsm_x4(qa, q_frag + QLO * 2 + ks * 32);
+          mma16816(sc[0], qa, kb[0], kb[1]);
+          mma16816(sc[1], qa, kb[2], kb[3]);
+        }
       }
     }
     // causal mask, online softmax (rows g and g+8 of the tile)
@@ -195,7 +225,7 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
     const float mu0 = mn0 == -INFINITY ? 0.f : mn0, mu1 = mn1 == -INFINITY ? 0.f : mn1;
     const float al0 = exp2f((m_run[0] - mu0) * sl2), al1 = exp2f((m_run[1] - mu1) * sl2);
     m_run[0] = mn0; m_run[1] = mn1;
-    uint32_t pf[4];
+    uint32_t pf[4], pl[4] = {0u, 0u, 0u, 0u};
     float ps0 = 0.f, ps1 = 0.f;
     {
       const float p00 = exp2f((sc[0][0] - mu0) * sl2), p01 = exp2f((sc[0][1] - mu0) * sl2);
@@ -208,6 +238,14 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
       pf[1] = pack_bf16(p02, p03);   // row g+8, keys 2q..
       pf[2] = pack_bf16(p10, p11);   // row g,   keys 8+2q.. (k high)
       pf[3] = pack_bf16(p12, p13);   // row g+8, keys 8+2q..
+      if (PR) {
+        auto lo_of = [](uint32_t packed, float a, float b) {
+          const __nv_bfloat162 hh = *reinterpret_cast<const __nv_bfloat162*>(&packed);
+          return pack_bf16(a - __low2float(hh), b - __high2float(hh));
+        };
+        pl[0] = lo_of(pf[0], p00, p01); pl[1] = lo_of(pf[1], p02, p03);
+        pl[2] = lo_of(pf[2], p10, p11); pl[3] = lo_of(pf[3], p12, p13);
+      }
     }
     l_run[0] = l_run[0] * al0 + ps0;
     l_run[1] = l_run[1] * al1 + ps1;
@@ -222,6 +260,10 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
         ldsm_x4_t(vb, vbase + (j >> 2) * SUB + key * 128 + ((c ^ (key & 7)) << 4));
         mma16816(o[2 * j], pf, vb[0], vb[1]);
         mma16816(o[2 * j + 1], pf, vb[2], vb[3]);
+        if (PR) {
+          mma16816(o[2 * j], pl, vb[0], vb[1]);
+          mma16816(o[2 * j + 1], pl, vb[2], vb[3]);
+        }
       }
     }
     __syncwarp();
@@ -272,8 +314,11 @@ attn_paged_kernel(const __grid_constant__ CUtensorMap kvmap, const bf16* __restr
       acc.x += e * x.x; acc.y += e * x.y; acc.z += e * x.z; acc.w += e * x.w;
     }
     const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
-    *reinterpret_cast<uint2*>(obase + size_t(rr) * H * DH + d) =
+    *reinterpret_cast<uint2*>(obase + size_t(rr) * H * DH * OW + d) =
         make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+    if (PR)   // the part of the result that the first bf16 value leaves
+      *reinterpret_cast<uint2*>(obase + size_t(rr) * H * DH * OW + size_t(H) * DH + d) =
+          make_uint2(pack_bf16(acc.x - __low2float(lo), acc.y - __high2float(lo)), pack_bf16(acc.z - __low2float(hi), acc.w - __high2float(hi)));
   }
   if (tid == 0 && abort_flag) atomicCAS(status, 0, LASER_ERR_TIMEOUT);
 }
@@ -290,7 +335,8 @@ laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const
   const int64_t rows_per_layer = int64_t(kv->n_pages) * 2 * Hkv * 16;
   const int layer_row0 = int(rows_per_layer * layer);
   const int tiles = ceil_div(Rs, 16), tpc = tiles > 1 ? 2 : 1;   // row tiles of a sequence; tiles per CTA
-  const size_t smem = 1024 + size_t(kStages) * (2 * (dh / 64) * 16 * 128) + size_t(16) * tpc * (dh + 8) * 2;
+  const bool pr = m->precise;
+  const size_t smem = 1024 + size_t(kStages) * (2 * (dh / 64) * 16 * 128) + size_t(16) * tpc * (dh + 8) * 2 * (pr ? 2 : 1);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(unsigned(B), unsigned(H), unsigned(ceil_div(tiles, tpc)));
   cfg.blockDim = dim3(kAttnThreads, 1, 1);
@@ -304,16 +350,22 @@ laser_status attention_tma_launch(laser_model* m, laser_kv* kv, int layer, const
   const __nv_bfloat16* q = m->q;
   const int32_t *rc = m->row_ctx, *rn = m->row_n, *pt = kv->page_table;
   const unsigned long long* mask = tree ? m->row_mask : nullptr;
-#define LASER_ATTN_LAUNCH(DH_, TPC_)                                                                                     \
+  const float* qf = m->qf;
+#define LASER_ATTN_LAUNCH(DH_, TPC_, PR_)                                                                                \
   do {                                                                                                                   \
-    LASER_CUDA(cudaFuncSetAttribute(attn_paged_kernel<DH_, TPC_>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))); \
-    LASER_CUDA(cudaLaunchKernelEx(&cfg, attn_paged_kernel<DH_, TPC_>, kv->pages_map, q, seq_ids, rc, rn, Rs, H, Hkv, pt, \
+    LASER_CUDA(cudaFuncSetAttribute(attn_paged_kernel<DH_, TPC_, PR_>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))); \
+    LASER_CUDA(cudaLaunchKernelEx(&cfg, attn_paged_kernel<DH_, TPC_, PR_>, kv->pages_map, q, qf, seq_ids, rc, rn, Rs, H, Hkv, pt, \
                                   kv->pages_per_seq, layer_row0, m->attn, m->status, mask));                              \
   } while (0)
-  if (dh == 128 && tpc == 1) LASER_ATTN_LAUNCH(128, 1);
-  else if (dh == 128) LASER_ATTN_LAUNCH(128, 2);
-  else if (tpc == 1) LASER_ATTN_LAUNCH(64, 1);
-  else LASER_ATTN_LAUNCH(64, 2);
+  if (pr) {
+    if (dh == 128 && tpc == 1) LASER_ATTN_LAUNCH(128, 1, true);
+    else if (dh == 128) LASER_ATTN_LAUNCH(128, 2, true);
+    else if (tpc == 1) LASER_ATTN_LAUNCH(64, 1, true);
+    else LASER_ATTN_LAUNCH(64, 2, true);
+  } else if (dh == 128 && tpc == 1) LASER_ATTN_LAUNCH(128, 1, false);
+  else if (dh == 128) LASER_ATTN_LAUNCH(128, 2, false);
+  else if (tpc == 1) LASER_ATTN_LAUNCH(64, 1, false);
+  else LASER_ATTN_LAUNCH(64, 2, false);
 #undef LASER_ATTN_LAUNCH
   count_launch();
   LASER_CUDA(cudaGetLastError());

@@ -543,7 +543,7 @@ static laser_status verify_impl(laser_model* m, laser_kv* kv, const int32_t* seq
   embed_kernel<<<m->R_pad, 256, 0, stream>>>(tokens, R, d, c.vocab, m->tok_emb, first_gain, m->resid, m->xn, m->sumsq, n_rows, Rs,
                                              fused ? m->row_draft : nullptr, m->precise ? 1 : 0);
   count_launch(2);
-  const bool use_tma_attn = !m->precise && attention_tma_supported(m, kv);   // precise: fp32 queries and probabilities
+  const bool use_tma_attn = attention_tma_supported(m, kv);
   const size_t attn_smem = (size_t(dh) + size_t(capacity) + 8) * sizeof(float);
   if (!use_tma_attn && attn_smem > 48 * 1024) {
     LASER_REQUIRE(attn_smem <= 200 * 1024, "KV capacity of %d tokens per sequence exceeds the attention kernel's limit", capacity);

@@ -3,7 +3,7 @@ contractions and attention (the library's per-launch event brackets), and of the
 the forward against acceptance fused into the LM head.
 
     python -m paper_2408_05676_b200.step_probe [--shape 7b|13b|tiny] [--layers L] [--batch B] [--draft K]
-                                               [--ctx N] [--steps S]
+                                               [--ctx N] [--steps S] [--precise 1]
 
 Synthetic weights (seed 0) and a synthetic cache of `ctx` tokens per sequence; every sequence carries
 K + 1 active rows.  Prints one JSON line.  The tests and bench.py measure the named configurations; this
@@ -20,9 +20,9 @@ from . import binding as L
 from . import synth
 
 
-def run(shape: str, layers: int, batch: int, draft: int, ctx: int, steps: int) -> dict:
+def run(shape: str, layers: int, batch: int, draft: int, ctx: int, steps: int, precise: int = 0) -> dict:
     dev = "cuda"
-    cfg = synth.model_cfg(shape, n_layers=layers, max_draft=draft)
+    cfg = synth.model_cfg(shape, n_layers=layers, max_draft=draft, precise=precise)
     W = synth.make_weights(cfg, seed=0, device=dev)
     model = L.model_create(cfg, W, max_batch=batch)
     pages = (ctx + draft + 1 + 15) // 16 + 1
@@ -88,7 +88,7 @@ def run(shape: str, layers: int, batch: int, draft: int, ctx: int, steps: int) -
     weight_bytes = 2 * (layers * (2 * d * d + 2 * d * dkv + 3 * d * f) + d * V)
     flops = float(rows) * weight_bytes
     kv_bytes = batch * ctx * layers * 2 * dkv * 2
-    return dict(shape=shape, layers=layers, batch=batch, rows=rows, ctx=ctx, ms_per_step=e0.elapsed_time(e1) / steps,
+    return dict(shape=shape, precise=precise, layers=layers, batch=batch, rows=rows, ctx=ctx, ms_per_step=e0.elapsed_time(e1) / steps,
                 verify_then_accept_ms=ab["two"], verify_accept_fused_ms=ab["fused"],
                 contractions_ms=gemm_ms / 2, contraction_launches=n_gemm // 2, attention_ms=attn_ms / 2,
                 attention_launches=n_attn // 2, weight_gb=weight_bytes / 1e9, kv_gb=kv_bytes / 1e9,
@@ -104,5 +104,6 @@ if __name__ == "__main__":
     ap.add_argument("--draft", type=int, default=8)
     ap.add_argument("--ctx", type=int, default=512)
     ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--precise", type=int, default=0, help="1 = operands as hi + lo bf16 pairs, fp32 attention")
     a = ap.parse_args()
-    print(json.dumps(run(a.shape, a.layers, a.batch, a.draft, a.ctx, a.steps)))
+    print(json.dumps(run(a.shape, a.layers, a.batch, a.draft, a.ctx, a.steps, a.precise)))
