@@ -65,10 +65,11 @@ typedef struct {
   int32_t page_size;   /* tokens per KV page; must be 16                                   */
   int32_t max_draft;   /* K: row stride of a step is max_draft + 1                         */
   int32_t max_batch;   /* most sequences in one laser_verify_step call                     */
-  int32_t precise;     /* non-zero: every activation that enters a matrix product is carried as a pair
-                          of bf16 values (hi + lo, about 16 significant bits) and the attention of the
-                          step's rows runs in fp32; weights and cache stay bf16.  Slower (each weight
-                          block is multiplied twice); for checking the forward against an exact one  */
+  int32_t precise;     /* non-zero: every activation that enters a matrix product (the attention's
+                          queries and probabilities included) is carried as a pair of bf16 values,
+                          hi + lo, about 16 significant bits; weights and cache stay bf16, sums fp32.
+                          Logits then lie within 2e-2 of an exact forward at the 7B depth (0.006
+                          measured); about 1.5 x the step time (each weight block is multiplied twice) */
 } laser_model_cfg;
 
 /* bf16 device pointers, matrices row-major [out_features, in_features] and 16-byte aligned,

@@ -1,6 +1,6 @@
 """The precise mode of the forward (`laser_model_cfg.precise`): every activation that enters a matrix
-product travels as a pair of bf16 values (hi + lo), the attention of the step's rows runs in fp32,
-weights and cache stay bf16.  With it the logits meet the stated tolerance - 2e-2 max-abs against the
+product travels as a pair of bf16 values (hi + lo) - the attention's queries and probabilities too -
+while weights and cache stay bf16 and accumulation fp32.  With it the logits meet the stated tolerance - 2e-2 max-abs against the
 exact fp64 oracle - at the 7B width and full depth, where no forward with plain bf16 operands can
 (the pinned bf16-operand yardstick is 0.2 away there, its hi + lo form 2e-3)."""
 import numpy as np
@@ -23,14 +23,18 @@ def L():
     return binding
 
 
-@pytest.mark.parametrize("over,B,ctx", [
-    (dict(), 4, [150, 0, 170, 5]),
+@pytest.mark.parametrize("over,B,ctx,bound", [
+    (dict(), 4, [150, 0, 170, 5], TOL / 10),
     # d_ffn 1376 is no multiple of the 64-wide K block: the last block of the hi part runs into the lo part
-    (dict(n_layers=3, d_model=512, n_heads=4, n_kv_heads=4, head_dim=128, d_ffn=1376, vocab=8192), 3, [130, 16, 1]),
-    (dict(n_layers=2, d_model=256, n_heads=8, n_kv_heads=2, head_dim=32, d_ffn=256, vocab=1000, max_draft=3), 5, [9, 33, 2, 0, 17]),
-    (dict(), 30, [int(x) for x in np.random.default_rng(3).integers(0, 150, 30)]),     # two token tiles
+    (dict(n_layers=3, d_model=512, n_heads=4, n_kv_heads=4, head_dim=128, d_ffn=1376, vocab=8192), 3, [130, 16, 1], TOL / 10),
+    (dict(n_layers=2, d_model=256, n_heads=8, n_kv_heads=2, head_dim=32, d_ffn=256, vocab=1000, max_draft=3), 5, [9, 33, 2, 0, 17], TOL / 10),
+    (dict(), 30, [int(x) for x in np.random.default_rng(3).integers(0, 150, 30)], TOL / 10),     # two token tiles
+    # the 13B layer shape at two layers (K = 16: two row tiles per attention CTA).  At this width the floor is the
+    # cache's own bf16 rounding of the new rows' K and V (the oracle's hi + lo yardstick is 1.8e-3 after one layer)
+    (dict(n_layers=2, d_model=5120, n_heads=40, n_kv_heads=40, head_dim=128, d_ffn=13824, vocab=8192, max_draft=16), 5,
+     [100, 3, 0, 64, 150], TOL / 2),
 ])
-def test_small_models_are_ten_times_inside_the_tolerance(L, over, B, ctx):
+def test_logits_well_inside_the_tolerance(L, over, B, ctx, bound):
     cfg = synth.model_cfg("tiny", **dict(over, precise=1))
     Wc = synth.make_weights(cfg, seed=0, gain_jitter=0.1)
     m = L.model_create(cfg, weights_to(Wc, "cuda"), max_batch=B)
@@ -51,7 +55,7 @@ def test_small_models_are_ten_times_inside_the_tolerance(L, over, B, ctx):
             okv.ctx[b] += len(rows[b])
         L.kv_set_len(kv, seq_ids, [int(okv.ctx[s]) for s in seq_ids])
     print("precise mode, max-abs logit error %.2e" % worst)
-    assert worst <= TOL / 10
+    assert worst <= bound
 
 
 def test_7b_full_depth_meets_the_stated_tolerance(L):
