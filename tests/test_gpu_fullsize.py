@@ -222,6 +222,7 @@ def _oracle_sample(L, cfg, W, model, pool, pool_np, offs, prompts, gid, sample, 
             okv.v[l, i, :ctx[i]] = v.cpu().view(ctx[i], cfg["n_kv_heads"], cfg["head_dim"])
         okv.ctx[i] = ctx[i]
     prm = L.make_params(K=K, n_min=1, n_max=4, max_occ=64)
+    model_p = L.model_create(dict(cfg, precise=1), W, max_batch=n)     # the precise mode on the same weights and cache
     seqs = [list(map(int, x)) for x in ps]
     ids = torch.arange(n, dtype=torch.int32, device="cuda")
     d_gid = dev_i32([gid[s] for s in sample])
@@ -230,6 +231,9 @@ def _oracle_sample(L, cfg, W, model, pool, pool_np, offs, prompts, gid, sample, 
         tails = np.asarray([x[-4:] for x in seqs], np.int32)
         d, dl, _ = L.draft(pool, dev_i32(tails), dev_i32([4] * n), d_gid, prm)
         tk, nr = L.make_rows(dev_i32([x[-1] for x in seqs]), d, dl, K)
+        if step == 0:      # first, so that the default mode's K/V of the rows are what stays in the cache
+            lg_p = L.verify_step(model_p, kv2, ids, tk, nr).cpu().numpy()
+            L.check(model_p)
         logits = L.verify_step(model, kv2, ids, tk, nr)
         na, ot, no = L.accept_commit(kv2, ids, logits, tk, nr, prm)
         L.check(model)
@@ -248,6 +252,10 @@ def _oracle_sample(L, cfg, W, model, pool, pool_np, offs, prompts, gid, sample, 
                 print("   sequence %d (prompt %d tokens, %d rows): logits vs exact max %.4f, bf16-operand yardstick %.4f"
                       % (s, len(ps[i]), len(rows), err, yerr))
                 assert err <= 1.25 * yerr
+                perr = float((torch.as_tensor(lg_p[i, :len(rows)]).double() - exact).abs().max())
+                print("   the same rows in the precise mode (operands as hi + lo bf16 pairs): max %.4f (stated tolerance %.0e)"
+                      % (perr, TOL))
+                assert perr <= TOL
             a_lib, em_lib = A.accept_one(lg[i, :len(rows)], rows, len(rows), A.STRICT, 1, 0.0)
             assert na[i] == a_lib and ot[i, :no[i]].tolist() == em_lib                  # acceptance on its own logits: bit-exact
             a_or, em_or = A.accept_one(exact.float().numpy(), rows, len(rows), A.STRICT, 1, 0.0)
