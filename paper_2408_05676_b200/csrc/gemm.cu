@@ -20,6 +20,11 @@
 //              cluster barrier, all six warps sum the partial tiles of the cluster through
 //              distributed shared memory in rank order (run-to-run identical, no partial sums
 //              in global memory) for the token columns this CTA owns and apply the fused epilogue.
+// Variants chosen by the host per launch: two weight tiles per CTA (MT = 2, one CTA per SM, token
+// tiles of up to 256 rows) where several token tiles make the launch L2->SM-bound; activations as
+// hi + lo bf16 pairs (the model's precise mode: every weight block is multiplied with both parts
+// into the same accumulator); and, for the LM head, an epilogue that leaves what the acceptance
+// rule needs per (row, vocabulary tile) instead of the logits.
 // Every mbarrier wait is bounded: on expiry the CTA records LASER_ERR_TIMEOUT, drains its
 // copies, still joins the cluster barriers, frees its tensor memory and exits.
 #include <map>
