@@ -133,6 +133,25 @@ def test_strict_equals_greedy_and_oracle(L, setup):
     assert exact + near + wtol == steps and near <= max(2, steps // 20) and wtol <= MAX_WITHIN_TOL
 
 
+def test_precise_mode_follows_the_oracle_without_tolerance_flips(L, setup):
+    """The same generation with the model in its precise mode (activations as hi + lo bf16 pairs) and acceptance
+    fused into the LM head: still lossless, and under teacher forcing no decision differs from the fp64 oracle's
+    except at true near-ties (1e-3) - the "within twice the logit tolerance" class stays empty."""
+    cfg, Wc, m, kv, pool, offs, prompts = setup
+    mp = L.model_create(dict(cfg, precise=1), weights_to(Wc, "cuda"), max_batch=4)
+    kvp = L.kv_create(mp, 4, 4 * 40)
+    h = L.pool_build(pool, offs, 1, 3)
+    gid = [0, 1, 2, 3]
+    greedy = L.generate(mp, kvp, None, prompts, gid, L.make_params(K=8, max_new=64))
+    for fused in (0, 1):
+        prm = L.make_params(K=8, n_min=1, n_max=3, max_occ=0, max_new=64, fused_accept=fused)
+        spec = L.generate(mp, kvp, h, prompts, gid, prm)
+        assert spec["out"] == greedy["out"] and spec["steps"] < greedy["steps"]
+    steps, exact, near, wtol = _teacher_forced(cfg, Wc, pool, offs, prompts, gid, spec["out"], prm, A.STRICT, 1, 0.0)
+    print("precise mode, strict: steps", steps, "exact", exact, "near-tie(<1e-3)", near, "within 2x tolerance", wtol)
+    assert exact + near == steps and wtol == 0 and near <= 1
+
+
 def test_relaxed_matches_oracle_under_teacher_forcing(L, setup):
     cfg, Wc, m, kv, pool, offs, prompts = setup
     h = L.pool_build(pool, offs, 1, 3)
