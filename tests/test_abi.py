@@ -44,3 +44,5 @@ def test_argument_errors_are_reported_without_a_gpu():
     assert st == -1 and b"null" in L.lib.laser_last_error()
     st = L.lib.laser_accept_commit(None, None, None, None, None, 1, 10, ctypes.byref(p), None, None, None, None)
     assert st == -1
+    st = L.lib.laser_verify_accept(None, None, None, None, None, 1, ctypes.byref(p), 1, None, None, None, None, None)
+    assert st == -1 and b"null" in L.lib.laser_last_error()
