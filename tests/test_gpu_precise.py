@@ -58,6 +58,33 @@ def test_logits_well_inside_the_tolerance(L, over, B, ctx, bound):
     assert worst <= bound
 
 
+def test_token_tree_rows_in_the_precise_mode(L):
+    """Tree attention (ancestor mask, depth positions) through the precise kernels: 20 rows per sequence, two row
+    tiles per attention CTA."""
+    cfg = synth.model_cfg("tiny", max_draft=19, precise=1)
+    Wc = synth.make_weights(cfg, seed=0, gain_jitter=0.1)
+    B, ctx = 3, [70, 0, 33]
+    m = L.model_create(cfg, weights_to(Wc, "cuda"), max_batch=B)
+    kv = L.kv_create(m, B, B * 12)
+    okv = O.KVCache(cfg, B, 12 * 16)
+    _fill_both(L, cfg, kv, okv, list(range(B)), ctx, seed=7)
+    rng = np.random.default_rng(2)
+    Rs = cfg["max_draft"] + 1
+    n_rows = np.asarray([Rs, 7, 12], np.int32)
+    tokens = rng.integers(0, cfg["vocab"], (B, Rs)).astype(np.int32)
+    parents = np.zeros((B, Rs), np.int32)
+    for b in range(B):
+        for i in range(1, Rs):
+            parents[b, i] = int(rng.integers(0, i))          # any earlier row
+    logits = L.verify_step_tree(m, kv, dev_i32(np.arange(B)), dev_i32(tokens), dev_i32(parents), dev_i32(n_rows))
+    L.check(m)
+    want = O.forward(Wc, cfg, okv, list(range(B)), [tokens[b, :n_rows[b]] for b in range(B)],
+                     parents=[parents[b, 1:n_rows[b]] for b in range(B)])
+    err = max(float((logits[b, :n_rows[b]].cpu().double() - want[b]).abs().max()) for b in range(B))
+    print("precise mode, token tree: max-abs logit error %.2e" % err)
+    assert err <= TOL / 10
+
+
 def test_7b_full_depth_meets_the_stated_tolerance(L):
     B, K, CTX = 16, 8, 512
     cfg = synth.model_cfg("7b", precise=1)
