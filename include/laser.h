@@ -357,7 +357,7 @@ laser_status laser_accept_commit_noalloc(laser_kv* kv, const int32_t* seq_ids, c
  *           applied to stored logits; NULL is the form meant for decoding.
  *   The arg max, the rank test (Eq. 7) and so STRICT and TOPK are exact: identical to
  *   laser_accept_commit on the stored logits.  Probabilities are combined in fp64 from per-tile
- *   fp32 sums and agree with the two-pass rule to about 1e-6 relative, so a RELAXED / TOPP /
+ *   fp32 sums and agree with the two-pass rule to a few 1e-6 relative, so a RELAXED / TOPP /
  *   RELAXED_ARGMAX verdict can differ only where the draft's probability lies within that distance
  *   of p.  Rules that rank need topk <= 4 (four logits are kept per tile): UNSUPPORTED otherwise.
  * Asynchronous on `stream`.  Errors: as laser_verify_step, and INVALID_ARG / UNSUPPORTED above. */
