@@ -112,8 +112,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 #pragma unroll
       for (int t = 0; t < MT; ++t) {
         const int T = wtile * MT + t;
-        tma_load_2d_hint(dst + t * w_bytes, &tmW, wk, EPI == EPI_SWIGLU ? T * 64 : T * kBM, bar, w_policy0);
-        tma_load_2d_hint(dst + t * w_bytes + w_bytes / 2, &tmW, wk, EPI == EPI_SWIGLU ? e.f + T * 64 : T * kBM + 64, bar, w_policy0);
+        if (EPI == EPI_SWIGLU) {   // 64 gate rows and the 64 up rows of the same features (the map's box is 64 rows)
+          tma_load_2d_hint(dst + t * w_bytes, &tmW, wk, T * 64, bar, w_policy0);
+          tma_load_2d_hint(dst + t * w_bytes + w_bytes / 2, &tmW, wk, e.f + T * 64, bar, w_policy0);
+        } else {                   // 128 consecutive rows: one copy (the map's box is 128 rows)
+          tma_load_2d_hint(dst + t * w_bytes, &tmW, wk, T * kBM, bar, w_policy0);
+        }
       }
     }
     tma_prefetch_map(&tmA);
@@ -170,18 +174,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const uint64_t w_policy = make_policy_evict_first(), a_policy = make_policy_evict_last();
       auto load = [&](uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar, uint64_t pol) { tma_load_2d_hint(dst, tm, x, y, bar, pol); };
       auto expect = [&](int s) { mbar_expect_tx(smem_u32(&full_bar[s]), stage_bytes); };
-      auto load_w = [&](int kb) {
-        const int s = kb % stages, k = ((kb0 + kb) >> wshift) * kBK;
+      auto load_w = [&](int kb, int s) {
+        const int k = ((kb0 + kb) >> wshift) * kBK;
         const uint32_t dst = tiles + uint32_t(s) * stage_bytes, bar = full0 + uint32_t(s) * 8;
 #pragma unroll
         for (int t = 0; t < MT; ++t) {
           const int T = wtile * MT + t;
-          load(dst + t * w_bytes, &tmW, k, EPI == EPI_SWIGLU ? T * 64 : T * kBM, bar, w_policy);
-          load(dst + t * w_bytes + w_bytes / 2, &tmW, k, EPI == EPI_SWIGLU ? e.f + T * 64 : T * kBM + 64, bar, w_policy);
+          if (EPI == EPI_SWIGLU) {
+            load(dst + t * w_bytes, &tmW, k, T * 64, bar, w_policy);
+            load(dst + t * w_bytes + w_bytes / 2, &tmW, k, e.f + T * 64, bar, w_policy);
+          } else {
+            load(dst + t * w_bytes, &tmW, k, T * kBM, bar, w_policy);
+          }
         }
       };
-      auto load_a = [&](int kb) {
-        const int s = kb % stages;
+      auto load_a = [&](int kb, int s) {
         const int g = kb0 + kb;
         load(tiles + uint32_t(s) * stage_bytes + MT * w_bytes, &tmA, (g & wshift) * e.a_lo_off + (g >> wshift) * kBK, r0,
              full0 + uint32_t(s) * 8, a_policy);
@@ -190,16 +197,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       // kernel before this one); only now wait for that kernel's results (the activations).
       const int pre = min(stages, nkb);
       asm volatile("griddepcontrol.wait;" ::: "memory");
-      for (int kb = 0; kb < pre; ++kb) load_a(kb);
+      for (int kb = 0; kb < pre; ++kb) load_a(kb, kb);
       bool ok = true;
       int kb = pre;
-      for (; kb < nkb; ++kb) {
-        const int s = kb % stages;
-        ok = mbar_wait(smem_u32(&empty_bar[s]), ((kb / stages) - 1) & 1, &abort_flag);
+      // (slot and round are counted, not divided out: this loop is one thread, and it paces the weight stream)
+      for (int s = 0, par = 0; kb < nkb; ++kb) {
+        ok = mbar_wait(smem_u32(&empty_bar[s]), par, &abort_flag);
         if (!ok) break;
         expect(s);
-        load_w(kb);
-        load_a(kb);
+        load_w(kb, s);
+        load_a(kb, s);
+        if (++s == stages) { s = 0; par ^= 1; }
       }
       if (!ok)  // drain copies still in flight before the CTA may exit
         for (int j = max(0, kb - stages); j < kb; ++j) mbar_drain(smem_u32(&full_bar[j % stages]), (j / stages) & 1);
@@ -208,9 +216,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (lane == 0) {  // ---- MMA issuer ----
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(NT >> 3) << 17) | (uint32_t(kBM >> 4) << 24);
       bool ok = true;
-      for (int kb = 0; kb < nkb && ok; ++kb) {
-        const int s = kb % stages;
-        ok = mbar_wait(smem_u32(&full_bar[s]), (kb / stages) & 1, &abort_flag);
+      for (int kb = 0, s = 0, par = 0; kb < nkb && ok; ++kb) {
+        ok = mbar_wait(smem_u32(&full_bar[s]), par, &abort_flag);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t w_addr = tiles + uint32_t(s) * stage_bytes;
@@ -223,6 +230,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             umma_bf16(tmem_acc + uint32_t(t) * kAccCols, wdesc + uint64_t(k * 2), adesc + uint64_t(k * 2), idesc, (kb | k) != 0);
         }
         umma_commit(smem_u32(&empty_bar[s]));
+        if (++s == stages) { s = 0; par ^= 1; }
       }
       // arrives when every MMA issued so far has finished
       umma_commit(smem_u32(&acc_bar));
@@ -499,7 +507,7 @@ laser_status gemm_fused(laser_model* m, const __nv_bfloat16* A, const __nv_bfloa
     if (cost(wide) < cost(sh)) sh = wide;
   }
   const CUtensorMap *tw = nullptr, *ta = nullptr;
-  LASER_TRY(tensor_map(st, W, N, K, 64, &tw));
+  LASER_TRY(tensor_map(st, W, N, K, epi == EPI_SWIGLU ? 64 : 128, &tw));
   LASER_TRY(tensor_map(st, A, m->R_pad, e.a_lo_off ? 2 * K : K, sh.NT, &ta));
   const int total_kb = ceil_div(K, kBK) * (e.a_lo_off ? 2 : 1), kbps = ceil_div(total_kb, splits);
   const int n_groups = ceil_div(n_wtiles, mt);     // grid rows: groups of mt weight tiles
