@@ -202,7 +202,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       int kb = pre;
       // (slot and round are counted, not divided out: this loop is one thread, and it paces the weight stream)
       for (int s = 0, par = 0; kb < nkb; ++kb) {
-        ok = mbar_wait(smem_u32(&empty_bar[s]), par, &abort_flag);
+        ok = mbar_wait_hot(smem_u32(&empty_bar[s]), par, &abort_flag);
         if (!ok) break;
         expect(s);
         load_w(kb, s);
@@ -217,7 +217,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(NT >> 3) << 17) | (uint32_t(kBM >> 4) << 24);
       bool ok = true;
       for (int kb = 0, s = 0, par = 0; kb < nkb && ok; ++kb) {
-        ok = mbar_wait(smem_u32(&full_bar[s]), par, &abort_flag);
+        ok = mbar_wait_hot(smem_u32(&full_bar[s]), par, &abort_flag);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t w_addr = tiles + uint32_t(s) * stage_bytes;

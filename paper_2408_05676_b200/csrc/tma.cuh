@@ -44,6 +44,25 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (clock64() - t0 > limit_cycles) { *abort_flag = 1; return false; }
   }
 }
+// The same bounded wait for the two single-thread loops that pace a kernel (the copy producer and the MMA
+// issuer): it polls without suspending, so the thread reacts as soon as the phase completes.
+__device__ __forceinline__ bool mbar_wait_hot(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                              long long limit_cycles = kWaitCycles) {
+  auto test = [&]() {
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+  };
+  if (test()) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    for (int i = 0; i < 1024; ++i)
+      if (test()) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > limit_cycles) { *abort_flag = 1; return false; }
+  }
+}
 // Drain helper for a producer that gave up: wait (bounded) for one copy still in flight.
 // Returns whether the copy landed within the limit.
 __device__ __forceinline__ bool mbar_drain(uint32_t bar, uint32_t parity) {
